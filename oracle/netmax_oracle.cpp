@@ -1,0 +1,384 @@
+// NetMax round oracle -- TEST INFRASTRUCTURE, not the product.
+//
+// A plain, slow, sequential-in-spirit CPU statement of what one synchronous
+// NetMax round computes, written from the paper (arXiv 2009.05766):
+//
+//   * peer selection            Algorithm 2 ("select a neighbour m with probability p_im")
+//   * first-step update         Eq. 15:  x^{k+1/2} = x^k - alpha * g^k,  g = grad f + xi
+//   * second-step (pull) update Eq. 16:  x^{k+1} = x^{k+1/2} - alpha*rho*gamma_im (x^{k+1/2} - x_m^k)
+//                               with gamma_im = (d_im + d_mi) / (2 p_im)   (Section "Convergence analysis")
+//
+// Round semantics (a batching of the paper's one-worker-per-global-step process):
+// in one round EVERY worker i performs one local iteration, and every pull reads the
+// peer's replica as it was at the START of the round.  State is fp32 (the replicas'
+// storage type); all arithmetic here is IEEE double, rounded to fp32 once per stored
+// element.  Random numbers come from the Philox4x32-10 counter-based generator
+// (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", SC'11),
+// implemented here from its published definition.
+//
+// Only tests, the smoke check and the benchmark's cpu_baseline leg may use this file.
+// It shares no code with the CUDA library and includes none of its headers.
+//
+// Parity pins (see tests/): Philox against cuRAND's host generator; normals against
+// the normal law; sampler against exact threshold sweeps and chi-square; the update
+// against the M=2 closed form, D^k products, contraction and fixed points.
+// Telemetry (consensus distance, mean loss) is not defined by the paper: parity unpinned
+// by the paper; it is pinned against a direct numpy evaluation of its definition.
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <thread>
+#include <vector>
+
+namespace {
+
+// ---------------------------------------------------------------- Philox4x32-10
+// One round: two 32x32->64 products of fixed odd multipliers with counter words 0 and 2;
+// the high halves are xored with counter words 1, 3 and the round key, the low halves
+// pass through, and the words are permuted.  The key is bumped by the two Weyl constants
+// between rounds.  Ten rounds.
+constexpr uint32_t kMul0 = 0xD2511F53u;
+constexpr uint32_t kMul1 = 0xCD9E8D57u;
+constexpr uint32_t kWeyl0 = 0x9E3779B9u;  // golden ratio
+constexpr uint32_t kWeyl1 = 0xBB67AE85u;  // sqrt(3) - 1
+
+void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+  uint32_t k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    if (round > 0) {
+      k0 += kWeyl0;
+      k1 += kWeyl1;
+    }
+    const uint64_t p0 = (uint64_t)kMul0 * c0;
+    const uint64_t p1 = (uint64_t)kMul1 * c2;
+    const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+    const uint32_t n0 = hi1 ^ c1 ^ k0;
+    const uint32_t n1 = lo1;
+    const uint32_t n2 = hi0 ^ c3 ^ k1;
+    const uint32_t n3 = lo0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Stream tags: the fourth counter word separates the independent streams.
+enum : uint32_t { TAG_PEER = 1, TAG_NOISE = 2, TAG_X0 = 3, TAG_C = 4 };
+
+// Counter layout: (column group e/4, worker i, round low word, tag | round high bits << 8).
+inline void make_ctr(uint32_t group, uint32_t worker, uint64_t round, uint32_t tag, uint32_t ctr[4]) {
+  ctr[0] = group;
+  ctr[1] = worker;
+  ctr[2] = (uint32_t)round;
+  ctr[3] = tag | ((uint32_t)(round >> 32) << 8);
+}
+
+// Box-Muller on 24-bit uniforms: u1 = (top24(a) + 1/2) / 2^24 in (0,1),
+// u2 = top24(b) / 2^24 in [0,1);  z0 = sqrt(-2 ln u1) cos(2 pi u2), z1 = ... sin(2 pi u2).
+// Words (0,1) of a Philox block give the normals of lanes 0,1; words (2,3) lanes 2,3.
+inline void normal_pair(uint32_t a, uint32_t b, double* z0, double* z1) {
+  const double u1 = ((double)(a >> 8) + 0.5) * (1.0 / 16777216.0);
+  const double u2 = (double)(b >> 8) * (1.0 / 16777216.0);
+  const double rad = std::sqrt(-2.0 * std::log(u1));
+  const double ang = 6.283185307179586476925286766559 * u2;
+  *z0 = rad * std::cos(ang);
+  *z1 = rad * std::sin(ang);
+}
+
+inline void normals4(const uint32_t r[4], double z[4]) {
+  normal_pair(r[0], r[1], &z[0], &z[1]);
+  normal_pair(r[2], r[3], &z[2], &z[3]);
+}
+
+// ------------------------------------------------------------------ sampler
+// 32-bit fixed-point cumulative thresholds of one probability row:
+//   cum_j = p_0 + ... + p_j (double, summed left to right),
+//   T_j   = floor(cum_j * 2^32 + 1/2), made non-decreasing, saturated to 2^32-1 for
+//           storage, and forced to the top for j >= the last index with p > 0.
+// A draw u (uint32) selects m = min(#{j : T_j <= u}, last_nz).
+void build_threshold_row(int M, const double* p, uint32_t* T, int32_t* last_nz) {
+  int32_t last = -1;
+  for (int j = 0; j < M; ++j)
+    if (p[j] > 0.0) last = j;
+  *last_nz = last;
+  double cum = 0.0;
+  uint64_t prev = 0;
+  for (int j = 0; j < M; ++j) {
+    cum += p[j];
+    uint64_t t = (uint64_t)std::floor(cum * 4294967296.0 + 0.5);
+    if (t < prev) t = prev;
+    if (t > 0xFFFFFFFFull || j >= last) t = 0xFFFFFFFFull;
+    T[j] = (uint32_t)t;
+    prev = t;
+  }
+}
+
+inline int32_t sample_row(const uint32_t* T, int M, int32_t last_nz, uint32_t u) {
+  int32_t count = 0;
+  for (int j = 0; j < M; ++j)
+    if (T[j] <= u) ++count;
+  return std::min(count, last_nz);
+}
+
+// Pull weight  w_im = alpha * rho * gamma_im = alpha*rho*(d_im + d_mi) / (2 p_im),
+// computed in double and rounded to fp32 (the precision the replicas are updated in).
+// Entries with p_im = 0 or m = i are 0 (never used: a self-draw skips the pull).
+void build_weight_row(int M, int i, const double* P, const uint8_t* adj, double alpha, double rho, float* w) {
+  for (int m = 0; m < M; ++m) {
+    const double p = P[(size_t)i * M + m];
+    if (m == i || !(p > 0.0)) {
+      w[m] = 0.0f;
+      continue;
+    }
+    const double dsum = (double)adj[(size_t)i * M + m] + (double)adj[(size_t)m * M + i];
+    w[m] = (float)(alpha * rho * dsum / (2.0 * p));
+  }
+}
+
+// ------------------------------------------------------------------ simulator
+struct Sim {
+  int M = 0;
+  int64_t d = 0;           // logical vector length (defines the noise counters)
+  int64_t ncols = 0;       // number of simulated columns (== d, or a sample of them)
+  std::vector<int64_t> cols;  // logical element index of each simulated column
+  double alpha = 0, rho = 0, sigma = 0;  // alpha, sigma already rounded to fp32 values
+  int objective = 1;
+  uint32_t key[2] = {0, 0};
+  uint64_t round = 0;
+  std::vector<uint32_t> T;
+  std::vector<int32_t> last_nz;
+  std::vector<float> w;
+  std::vector<float> x, xn, c;  // [M][ncols]
+  std::vector<int32_t> trace;   // [round][M], all rounds since creation
+  std::vector<double> tel_consensus, tel_loss;  // per round, on the round-start state
+};
+
+void sim_set_policy(Sim* s, const double* P, const uint8_t* adj, double rho) {
+  const int M = s->M;
+  s->rho = rho;
+  s->T.assign((size_t)M * M, 0);
+  s->last_nz.assign(M, 0);
+  s->w.assign((size_t)M * M, 0.0f);
+  for (int i = 0; i < M; ++i) {
+    build_threshold_row(M, P + (size_t)i * M, s->T.data() + (size_t)i * M, &s->last_nz[i]);
+    build_weight_row(M, i, P, adj, s->alpha, rho, s->w.data() + (size_t)i * M);
+  }
+}
+
+void fill_normal(Sim* s, std::vector<float>& dst, double stddev, uint32_t tag) {
+  for (int i = 0; i < s->M; ++i)
+    for (int64_t k = 0; k < s->ncols; ++k) {
+      const int64_t e = s->cols[k];
+      uint32_t ctr[4], r[4];
+      double z[4];
+      make_ctr((uint32_t)(e >> 2), (uint32_t)i, 0, tag, ctr);
+      philox4x32_10(ctr, s->key, r);
+      normals4(r, z);
+      dst[(size_t)i * s->ncols + k] = (float)(stddev * z[e & 3]);
+    }
+}
+
+// Telemetry on the current state: consensus distance (1/M) sum_i ||x_i - xbar||^2 and
+// mean loss (1/M) sum_i 1/2 ||x_i - c_i||^2 (the two terms of the paper's Eq. 1 that the
+// simulator can observe).  Plain double sums over the simulated columns.
+void telemetry(const Sim* s, double* consensus, double* loss) {
+  const int M = s->M;
+  double cons = 0.0, ls = 0.0;
+  for (int64_t k = 0; k < s->ncols; ++k) {
+    double mean = 0.0;
+    for (int i = 0; i < M; ++i) mean += (double)s->x[(size_t)i * s->ncols + k];
+    mean /= M;
+    for (int i = 0; i < M; ++i) {
+      const double xv = (double)s->x[(size_t)i * s->ncols + k];
+      const double cv = (double)s->c[(size_t)i * s->ncols + k];
+      cons += (xv - mean) * (xv - mean);
+      ls += 0.5 * (xv - cv) * (xv - cv);
+    }
+  }
+  *consensus = cons / M;
+  *loss = ls / M;
+}
+
+void round_columns(Sim* s, const int32_t* peer, int64_t k0, int64_t k1) {
+  const int M = s->M;
+  const int64_t n = s->ncols;
+  for (int i = 0; i < M; ++i) {
+    const int m = peer[i];
+    const double w = (double)s->w[(size_t)i * M + m];
+    const float* xi = s->x.data() + (size_t)i * n;
+    const float* xm = s->x.data() + (size_t)m * n;  // round-start snapshot of the peer
+    const float* ci = s->c.data() + (size_t)i * n;
+    float* out = s->xn.data() + (size_t)i * n;
+    for (int64_t k = k0; k < k1; ++k) {
+      const int64_t e = s->cols[k];
+      const double xv = (double)xi[k];
+      double g = 0.0;
+      if (s->objective == 1) {
+        uint32_t ctr[4], r[4];
+        double z[4];
+        make_ctr((uint32_t)(e >> 2), (uint32_t)i, s->round, TAG_NOISE, ctr);
+        philox4x32_10(ctr, s->key, r);
+        normals4(r, z);
+        g = (xv - (double)ci[k]) + s->sigma * z[e & 3];  // grad of 1/2||x-c||^2, plus additive noise
+      }
+      const double h = xv - s->alpha * g;                        // Eq. 15
+      double xnew = h;
+      if (m != i) xnew = h - w * (h - (double)xm[k]);            // Eq. 16; a self-draw pulls nothing
+      out[k] = (float)xnew;
+    }
+  }
+}
+
+void sim_round(Sim* s, int threads) {
+  const int M = s->M;
+  std::vector<int32_t> peer(M);
+  for (int i = 0; i < M; ++i) {
+    uint32_t ctr[4], r[4];
+    make_ctr(0, (uint32_t)i, s->round, TAG_PEER, ctr);
+    philox4x32_10(ctr, s->key, r);
+    peer[i] = sample_row(s->T.data() + (size_t)i * M, M, s->last_nz[i], r[0]);
+  }
+  double cons, ls;
+  telemetry(s, &cons, &ls);
+  s->tel_consensus.push_back(cons);
+  s->tel_loss.push_back(ls);
+  s->trace.insert(s->trace.end(), peer.begin(), peer.end());
+
+  threads = std::max(1, threads);
+  if (threads == 1 || s->ncols < 4096) {
+    round_columns(s, peer.data(), 0, s->ncols);
+  } else {
+    std::vector<std::thread> pool;
+    const int64_t per = (s->ncols + threads - 1) / threads;
+    for (int t = 0; t < threads; ++t) {
+      const int64_t k0 = std::min<int64_t>(s->ncols, t * per), k1 = std::min<int64_t>(s->ncols, k0 + per);
+      if (k0 < k1) pool.emplace_back(round_columns, s, peer.data(), k0, k1);
+    }
+    for (auto& th : pool) th.join();
+  }
+  s->x.swap(s->xn);
+  s->round += 1;
+}
+
+}  // namespace
+
+extern "C" {
+
+void nmo_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) { philox4x32_10(ctr, key, out); }
+
+// out[4n]: blocks for counters (c0_first + j, c1, c2, c3), j = 0..n-1.
+void nmo_philox_blocks(uint64_t seed, uint32_t c0_first, uint32_t c1, uint32_t c2, uint32_t c3, int64_t n,
+                       uint32_t* out) {
+  const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  for (int64_t j = 0; j < n; ++j) {
+    const uint32_t ctr[4] = {c0_first + (uint32_t)j, c1, c2, c3};
+    philox4x32_10(ctr, key, out + 4 * j);
+  }
+}
+
+// Normals of the noise stream: z[n] for elements e0..e0+n-1 of worker i at a round.
+void nmo_noise(uint64_t seed, int32_t worker, uint64_t round, int64_t e0, int64_t n, double* z) {
+  const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  for (int64_t e = e0; e < e0 + n; ++e) {
+    uint32_t ctr[4], r[4];
+    double zz[4];
+    make_ctr((uint32_t)(e >> 2), (uint32_t)worker, round, TAG_NOISE, ctr);
+    philox4x32_10(ctr, key, r);
+    normals4(r, zz);
+    z[e - e0] = zz[e & 3];
+  }
+}
+
+void nmo_normals_from_words(const uint32_t* r4, double* z4) { normals4(r4, z4); }
+
+void nmo_build_thresholds(int32_t M, const double* P, uint32_t* T, int32_t* last_nz) {
+  for (int i = 0; i < M; ++i) build_threshold_row(M, P + (size_t)i * M, T + (size_t)i * M, last_nz + i);
+}
+
+int32_t nmo_sample(const uint32_t* Trow, int32_t M, int32_t last_nz, uint32_t u) { return sample_row(Trow, M, last_nz, u); }
+
+void nmo_build_weights(int32_t M, const double* P, const uint8_t* adj, double alpha, double rho, float* w) {
+  for (int i = 0; i < M; ++i) build_weight_row(M, i, P, adj, alpha, rho, w + (size_t)i * M);
+}
+
+// Peer draws only (no replica state): out[n_rounds][M].
+void nmo_peer_draws(int32_t M, const double* P, uint64_t seed, uint64_t first_round, int64_t n_rounds, int32_t* out) {
+  std::vector<uint32_t> T((size_t)M * M);
+  std::vector<int32_t> last(M);
+  nmo_build_thresholds(M, P, T.data(), last.data());
+  const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  for (int64_t r = 0; r < n_rounds; ++r)
+    for (int i = 0; i < M; ++i) {
+      uint32_t ctr[4], w[4];
+      make_ctr(0, (uint32_t)i, first_round + (uint64_t)r, TAG_PEER, ctr);
+      philox4x32_10(ctr, key, w);
+      out[(size_t)r * M + i] = sample_row(T.data() + (size_t)i * M, M, last[i], w[0]);
+    }
+}
+
+// cols == nullptr: simulate all d columns; else the ncols listed logical element indices.
+void* nmo_sim_create(int32_t M, int64_t d, const int64_t* cols, int64_t ncols, const double* P, const uint8_t* adj,
+                     double alpha, double rho, double sigma, int32_t objective, uint64_t seed) {
+  Sim* s = new Sim();
+  s->M = M;
+  s->d = d;
+  if (cols) {
+    s->ncols = ncols;
+    s->cols.assign(cols, cols + ncols);
+  } else {
+    s->ncols = d;
+    s->cols.resize(d);
+    for (int64_t e = 0; e < d; ++e) s->cols[e] = e;
+  }
+  s->alpha = (double)(float)alpha;  // the update runs on fp32 parameters
+  s->sigma = (double)(float)sigma;
+  s->objective = objective;
+  s->key[0] = (uint32_t)seed;
+  s->key[1] = (uint32_t)(seed >> 32);
+  s->x.assign((size_t)M * s->ncols, 0.0f);
+  s->xn.assign((size_t)M * s->ncols, 0.0f);
+  s->c.assign((size_t)M * s->ncols, 0.0f);
+  sim_set_policy(s, P, adj, rho);
+  return s;
+}
+
+void nmo_sim_destroy(void* h) { delete (Sim*)h; }
+void nmo_sim_set_policy(void* h, const double* P, const uint8_t* adj, double rho) { sim_set_policy((Sim*)h, P, adj, rho); }
+
+// x_i(0) = x0_std * z, c_i = c_std * z from the X0 / C streams (round word 0).
+void nmo_sim_init(void* h, double x0_std, double c_std) {
+  Sim* s = (Sim*)h;
+  fill_normal(s, s->x, x0_std, TAG_X0);
+  fill_normal(s, s->c, c_std, TAG_C);
+}
+
+void nmo_sim_set_x(void* h, const float* x) { Sim* s = (Sim*)h; std::memcpy(s->x.data(), x, s->x.size() * sizeof(float)); }
+void nmo_sim_set_c(void* h, const float* c) { Sim* s = (Sim*)h; std::memcpy(s->c.data(), c, s->c.size() * sizeof(float)); }
+void nmo_sim_get_x(void* h, float* x) { Sim* s = (Sim*)h; std::memcpy(x, s->x.data(), s->x.size() * sizeof(float)); }
+void nmo_sim_get_c(void* h, float* c) { Sim* s = (Sim*)h; std::memcpy(c, s->c.data(), s->c.size() * sizeof(float)); }
+
+void nmo_sim_round(void* h, int64_t n_rounds, int32_t threads) {
+  for (int64_t r = 0; r < n_rounds; ++r) sim_round((Sim*)h, threads);
+}
+
+int64_t nmo_sim_rounds_done(void* h) { return (int64_t)((Sim*)h)->round; }
+
+void nmo_sim_get_trace(void* h, int64_t first, int64_t n, int32_t* out) {
+  Sim* s = (Sim*)h;
+  std::memcpy(out, s->trace.data() + (size_t)first * s->M, (size_t)n * s->M * sizeof(int32_t));
+}
+
+void nmo_sim_get_telemetry(void* h, int64_t first, int64_t n, double* consensus, double* loss) {
+  Sim* s = (Sim*)h;
+  for (int64_t r = 0; r < n; ++r) {
+    consensus[r] = s->tel_consensus[first + r];
+    loss[r] = s->tel_loss[first + r];
+  }
+}
+
+void nmo_sim_telemetry_now(void* h, double* consensus, double* loss) { telemetry((Sim*)h, consensus, loss); }
+
+}  // extern "C"
