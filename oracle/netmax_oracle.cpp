@@ -76,11 +76,12 @@ inline void make_ctr(uint32_t group, uint32_t worker, uint64_t round, uint32_t t
   ctr[3] = tag | ((uint32_t)(round >> 32) << 8);
 }
 
-// Box-Muller on 24-bit uniforms: u1 = (top24(a) + 1/2) / 2^24 in (0,1),
+// Box-Muller on fixed-point uniforms that fp32 also represents exactly:
+// u1 = (top23(a) + 1/2) / 2^23 in (0,1)  (2*top23+1 is a 24-bit integer),
 // u2 = top24(b) / 2^24 in [0,1);  z0 = sqrt(-2 ln u1) cos(2 pi u2), z1 = ... sin(2 pi u2).
 // Words (0,1) of a Philox block give the normals of lanes 0,1; words (2,3) lanes 2,3.
 inline void normal_pair(uint32_t a, uint32_t b, double* z0, double* z1) {
-  const double u1 = ((double)(a >> 8) + 0.5) * (1.0 / 16777216.0);
+  const double u1 = ((double)(a >> 9) + 0.5) * (1.0 / 8388608.0);
   const double u2 = (double)(b >> 8) * (1.0 / 16777216.0);
   const double rad = std::sqrt(-2.0 * std::log(u1));
   const double ang = 6.283185307179586476925286766559 * u2;

@@ -10,20 +10,20 @@ from oracle import oracle
 
 # ------------------------------------------------------------------ normals
 def test_box_muller_special_angles_and_radii():
-    top = 0xFFFFFF00
-    # angle 0: z0 = radius, z1 = 0; the radius for the largest u1 = 1 - 2^-25 is sqrt(-2 ln(1-2^-25))
+    top = 0xFFFFFE00
+    # angle 0: z0 = radius, z1 = 0; the radius for the largest u1 = 1 - 2^-24 is sqrt(-2 ln(1-2^-24))
     z = oracle.normals_from_words([top, 0, 0, 0])
     assert z[1] == 0.0
-    assert z[0] == pytest.approx(math.sqrt(-2.0 * math.log1p(-2.0 ** -25)), rel=1e-9)
-    # smallest u1 = 2^-25 gives the largest radius sqrt(50 ln 2)
-    assert z[2] == pytest.approx(math.sqrt(50.0 * math.log(2.0)), rel=1e-12)
+    assert z[0] == pytest.approx(math.sqrt(-2.0 * math.log1p(-2.0 ** -24)), rel=1e-9)
+    # smallest u1 = 2^-24 gives the largest radius sqrt(48 ln 2)
+    assert z[2] == pytest.approx(math.sqrt(48.0 * math.log(2.0)), rel=1e-12)
     # a quarter turn (u2 = 1/4): z0 ~ 0, z1 = radius; half a turn: z0 = -radius
     z = oracle.normals_from_words([0x80000000, 0x40000000, 0x80000000, 0x80000000])
-    rad = math.sqrt(-2.0 * math.log((2 ** 23 + 0.5) / 2 ** 24))
+    rad = math.sqrt(-2.0 * math.log((2 ** 22 + 0.5) / 2 ** 23))
     assert abs(z[0]) < 1e-15 and z[1] == pytest.approx(rad, rel=1e-12)
     assert z[2] == pytest.approx(-rad, rel=1e-12) and abs(z[3]) < 1e-15
-    # the low 8 bits of each word are not used
-    assert (oracle.normals_from_words([0x800000FF, 0x400000FF, 0x800000FF, 0x800000FF]) == z).all()
+    # the low 9 bits of the radius words and the low 8 bits of the angle words are not used
+    assert (oracle.normals_from_words([0x800001FF, 0x400000FF, 0x800001FF, 0x800000FF]) == z).all()
 
 
 def test_noise_is_standard_normal():
