@@ -1,0 +1,199 @@
+/*
+ * netmax.h -- C ABI of the NetMax round simulator for one NVIDIA B200 (sm_100a).
+ *
+ * NetMax (arXiv 2009.05766) is decentralised consensus SGD: worker i repeatedly (a) picks a
+ * peer m with probability p_im from its row of the communication policy matrix P
+ * (Algorithm 2, "select a neighbour m with probability p_im"), (b) takes a local SGD step
+ * x_i^{k+1/2} = x_i^k - alpha g_i^k (Eq. 15), and (c) pulls the peer's parameters,
+ * x_i^{k+1} = x_i^{k+1/2} - alpha rho gamma_im (x_i^{k+1/2} - x_m^k),
+ * gamma_im = (d_im + d_mi) / (2 p_im) (Eq. 16).  This library keeps all M replicas in one
+ * GPU's memory and advances them in synchronous ROUNDS: in a round every worker does one
+ * such iteration, and every pull reads the peer's replica as it was at the start of the
+ * round.  Objectives are f_i(x) = 1/2 ||x - c_i||^2 with additive N(0, sigma^2) gradient
+ * noise (the paper's additive-noise assumption), or zero gradients.
+ *
+ * Conventions
+ *   - Every function returns NETMAX_OK (0) or a negative netmax_status; none throws,
+ *     aborts or leaves the CUDA context in a sticky error state of its own making.
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA device memory on
+ *     the context's device.  Inputs are borrowed for the duration of the call and copied;
+ *     outputs are caller-allocated and caller-owned.
+ *   - Matrices are row-major M x M; replica arrays are dense row-major M x d (no padding).
+ *   - Rounds are numbered from 0 over the life of a context.  All random numbers are
+ *     Philox4x32-10 blocks addressed by (seed, stream, worker, round, element), so splitting
+ *     netmax_round(a + b) into netmax_round(a); netmax_round(b) changes no bit.
+ *   - Work is enqueued on the context's stream.  Calls that return data to the host
+ *     synchronise that stream first.  A context is not thread-safe.
+ */
+#ifndef NETMAX_H_
+#define NETMAX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum netmax_status {
+  NETMAX_OK = 0,
+  NETMAX_INVALID_ARG = -1,    /* null pointer, size out of range, non-finite parameter        */
+  NETMAX_BAD_PROB_ROW = -2,   /* a row of P has a negative entry or does not sum to 1 (1e-9)  */
+  NETMAX_OOM = -3,            /* device or host allocation failed / workspace too small       */
+  NETMAX_CUDA_ERROR = -4,     /* a CUDA call failed; see netmax_last_error                    */
+  NETMAX_TRACE_RANGE = -5,    /* requested rounds are not (or no longer) in the ring          */
+  NETMAX_NOT_CONNECTED = -6,  /* the link graph is not connected (Assumption 1)               */
+  NETMAX_INFEASIBLE = -7      /* Algorithm 3 found no feasible (rho, t_bar) grid point        */
+} netmax_status;
+
+typedef struct netmax_ctx netmax_ctx; /* opaque; created and destroyed by the library */
+
+/*
+ * Full configuration of a context (Algorithm 2's inputs alpha, rho and P, plus what the
+ * simulator adds: sizes, the synthetic objective, the seed and where to run).
+ */
+typedef struct netmax_config {
+  int32_t M;                     /* workers, 2 <= M <= 16384                                          */
+  int64_t d;                     /* parameters per replica, 1 <= d < 2^33                              */
+  int64_t element_offset;        /* logical index of this context's first element inside a longer global
+                                    vector (a multiple of 4, offset + d < 2^33; default 0).  Only the
+                                    noise / initialisation counters use it: contexts that hold disjoint
+                                    column ranges of one problem (one per GPU) then draw the streams the
+                                    single-context run would, and never need to exchange data            */
+  const double* link_speed_gbps; /* host, M*M, symmetric, diagonal ignored; speed <= 0 means "no link"
+                                    (d_im = 0).  NULL means fully connected with equal speeds          */
+  const double* prob;            /* host, M*M, row i = P[i,:].  NULL: run Algorithm 3 on the iteration
+                                    times derived from link_speed_gbps (policy_K x policy_R grid)      */
+  double lr;                     /* alpha > 0; the update uses its fp32 rounding                       */
+  double rho;                    /* rho; <= 0: with prob given, the largest rho meeting Eq. 11 with a
+                                    1e-6 margin, min_{p_im>0} p_im / (alpha (d_im+d_mi)); with prob
+                                    NULL, the rho Algorithm 3 selects                                  */
+  double sigma;                  /* std of the gradient noise; the update uses its fp32 rounding       */
+  double x0_std, c_std;          /* x_i(0) ~ N(0, x0_std^2), c_i ~ N(0, c_std^2), drawn from the seed  */
+  int32_t objective;             /* 0: zero gradients (sigma ignored); 1: f_i = 1/2 ||x - c_i||^2      */
+  uint64_t seed;                 /* Philox key                                                         */
+  int32_t device;                /* CUDA device ordinal                                                */
+  void* stream;                  /* cudaStream_t to enqueue on (NULL: the legacy default stream)       */
+  int64_t trace_rounds;          /* capacity of the peer-trace / telemetry ring, in rounds (>= 1)      */
+  int32_t policy_K, policy_R;    /* Algorithm 3 grid sizes when prob is NULL (<= 0: 20 x 20)           */
+  void* workspace;               /* device memory for ALL of the context's device buffers, 256-byte
+                                    aligned, at least netmax_workspace_size() bytes, owned by the
+                                    caller and kept alive until netmax_destroy.  NULL: the library
+                                    allocates with cudaMalloc and frees in netmax_destroy              */
+  size_t workspace_bytes;
+} netmax_config;
+
+/* Fills *cfg with defaults: rho = 0 (automatic), sigma = 0, stds 0, objective 1, seed 0,
+ * device 0, stream NULL, trace_rounds 1024, policy grid 20 x 20, no workspace, offset 0. */
+int netmax_config_init(netmax_config* cfg);
+
+/* Device bytes a context with this M, d and trace_rounds needs (only those fields are read). */
+int netmax_workspace_size(const netmax_config* cfg, size_t* bytes);
+
+/*
+ * Creates a context: validates, builds the 32-bit cumulative-threshold table and the
+ * pull-weight table w_im = alpha rho (d_im + d_mi) / (2 p_im) (Eq. 16) on the host, uploads
+ * them, and fills x(0) and c on the device from the seed.  *out is NULL on failure.
+ */
+int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out);
+
+/* Short form: objective 1, sigma = 0, x0_std = c_std = 1, automatic rho, current device,
+ * default stream, library-allocated memory.  link_speed_gbps and prob as in netmax_config. */
+int netmax_create(int32_t M, int64_t d, const double* link_speed_gbps, const double* prob, double lr,
+                  uint64_t seed, netmax_ctx** out);
+
+void netmax_destroy(netmax_ctx* ctx);
+
+/*
+ * Replaces P, the link graph and rho between rounds (Algorithm 2: "if received new policy").
+ * Arguments as in netmax_config; prob == NULL reruns Algorithm 3; link_speed_gbps == NULL
+ * keeps the current graph.  Takes effect from the next round.
+ */
+int netmax_set_policy(netmax_ctx* ctx, const double* link_speed_gbps, const double* prob, double rho);
+
+/* Reads back the policy in force: prob_out (host, M*M) and *rho_out; either may be NULL. */
+int netmax_get_policy(netmax_ctx* ctx, double* prob_out, double* rho_out);
+
+/* Overwrite all replicas / all centres from dense host arrays of M*d floats. */
+int netmax_set_replicas(netmax_ctx* ctx, const float* host_x);
+int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
+
+/*
+ * Runs n_rounds rounds (n_rounds >= 0), asynchronously on the context's stream.  Per round:
+ * the peer of every worker is drawn (Algorithm 2), then ONE fused kernel applies Eq. 15 and
+ * Eq. 16 to every element of every replica, reading the round-start buffer and writing the
+ * other one, and reduces that round's telemetry.
+ */
+int netmax_round(netmax_ctx* ctx, int64_t n_rounds);
+
+/* Number of rounds enqueued so far. */
+int64_t netmax_rounds_done(const netmax_ctx* ctx);
+
+/* Synchronises, then copies the current replicas to host_out (M*d floats, dense). */
+int netmax_read_replicas(netmax_ctx* ctx, float* host_out);
+/* Same for the centres c_i. */
+int netmax_read_centres(netmax_ctx* ctx, float* host_out);
+
+/*
+ * Copies the values of the listed logical element indices (0 <= cols[k] < d) of every
+ * replica to host_out (M*n_cols floats, row-major): a cheap way to inspect large replicas.
+ */
+int netmax_read_columns(netmax_ctx* ctx, const int64_t* host_cols, int64_t n_cols, float* host_out);
+
+/*
+ * Peers drawn in rounds [first_round, first_round + n): host_out[(r - first_round) * M + i]
+ * is the peer of worker i in round r.  Only the last trace_rounds rounds are kept;
+ * NETMAX_TRACE_RANGE otherwise.  Synchronises.
+ */
+int netmax_peer_trace(netmax_ctx* ctx, int64_t first_round, int64_t n, int32_t* host_out);
+
+/*
+ * Telemetry of rounds [first_round, first_round + n), measured on each round's START state:
+ * consensus[r] = (1/M) sum_i ||x_i - mean_j x_j||^2 and loss[r] = (1/M) sum_i 1/2 ||x_i - c_i||^2
+ * (the two parts of the consensus objective, Eq. 1, that the simulator observes).  Either
+ * output may be NULL.  Same ring rule as netmax_peer_trace.  Synchronises.
+ */
+int netmax_telemetry(netmax_ctx* ctx, int64_t first_round, int64_t n, double* host_consensus, double* host_loss);
+
+/*
+ * Device access for callers that keep working on the GPU (for example through PyTorch):
+ * *x is the buffer holding the current replicas, row i at x + i * ld, ld >= d floats,
+ * valid until the next netmax_round / netmax_set_* call; nothing is synchronised.
+ */
+int netmax_replicas_device(netmax_ctx* ctx, const float** x, int64_t* ld);
+
+/*
+ * Peer draws alone (the sampler of Algorithm 2), for n_rounds rounds starting at
+ * first_round, written to device_out (device, n_rounds*M int32), asynchronously on the
+ * context's stream; does not advance the context's round counter.
+ */
+int netmax_sample_peers(netmax_ctx* ctx, int64_t first_round, int64_t n_rounds, int32_t* device_out);
+
+/*
+ * Host control plane.  Iteration-time model (Section II-B: t_im = max{C_i, N_im}):
+ * N_im = 32 d / (s_im 1e9) s, C_i = min N / 4, t_ii = C_i.  t_out (M*M) and adj_out (M*M,
+ * 0/1) are host arrays.
+ */
+int netmax_iteration_times(int32_t M, int64_t d, const double* link_speed_gbps, double* t_out, uint8_t* adj_out);
+
+/*
+ * Algorithm 3 (communication policy generation): searches K values of rho and, for each,
+ * R values of the average iteration time t_bar; at every grid point solves the row-wise LP
+ * (Eq. 14 under Eq. 10-13), forms Y_P = E[D^T D] (Eq. 22), and keeps the point minimising
+ * t_bar ln(eps) / ln(lambda_2).  All arrays are host memory; prob_out is M*M.  info_out,
+ * if not NULL, receives {lambda_2, t_bar, t_convergence (eps = 1e-3), k, r}.
+ */
+int netmax_policy_generate(int32_t M, const double* t_iter, const uint8_t* adj, double lr, int32_t K, int32_t R,
+                           double* prob_out, double* rho_out, double* info_out /* 5 doubles */);
+
+/* Counters for benchmarks: kernels launched by this context so far. */
+int64_t netmax_kernel_launches(const netmax_ctx* ctx);
+
+/* Message of the last failure on this context ("" if none); ctx == NULL: the last failure
+ * of a call that had no context (creation).  The string is owned by the library. */
+const char* netmax_last_error(const netmax_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NETMAX_H_ */

@@ -1,0 +1,700 @@
+// C-ABI implementation of the NetMax round simulator (see include/netmax.h).
+//
+// Host side: validation, the 32-bit cumulative-threshold and pull-weight tables, buffer
+// layout, launches.  Every step of a round runs in the kernels of netmax_kernels.cuh.
+#include "../../include/netmax.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "netmax_kernels.cuh"
+#include "netmax_policy.h"
+
+using namespace netmax;
+
+namespace {
+
+thread_local std::string g_error;  // failures of calls that have no context
+
+constexpr int kThreads = 256;
+constexpr int64_t kMaxM = 16384;
+constexpr int64_t kMaxD = (int64_t)1 << 33;
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { prev = -1; }
+    if (prev != dev) ok = (cudaSetDevice(dev) == cudaSuccess);
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+struct Layout {
+  int64_t ld = 0, ldq = 0, nq = 0;
+  size_t off_x0 = 0, off_x1 = 0, off_c = 0, off_thr = 0, off_last = 0, off_w = 0, off_trace = 0, off_tel = 0,
+         off_partials = 0, off_ticket = 0, total = 0;
+};
+
+constexpr int kMaxGrid = 148 * 16;  // upper bound on resident CTAs of the round kernel
+
+Layout make_layout(int64_t M, int64_t d, int64_t trace_rounds) {
+  Layout L;
+  L.ld = (int64_t)align_up((size_t)d, 32);  // rows start on 128-byte boundaries
+  L.ldq = L.ld / 4;
+  L.nq = (d + 3) / 4;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  const size_t plane = (size_t)M * L.ld * sizeof(float);
+  L.off_x0 = take(plane);
+  L.off_x1 = take(plane);
+  L.off_c = take(plane);
+  L.off_thr = take((size_t)M * M * sizeof(uint32_t));
+  L.off_last = take((size_t)M * sizeof(int32_t));
+  L.off_w = take((size_t)M * M * sizeof(float));
+  L.off_trace = take((size_t)trace_rounds * M * sizeof(int32_t));
+  L.off_tel = take((size_t)trace_rounds * 2 * sizeof(double));
+  L.off_partials = take((size_t)kMaxGrid * 2 * sizeof(double));
+  L.off_ticket = take(256);
+  L.total = o;
+  return L;
+}
+
+}  // namespace
+
+namespace netmax {
+void set_global_error(const std::string& msg) { g_error = msg; }
+}  // namespace netmax
+
+struct netmax_ctx {
+  int32_t M = 0;
+  int64_t d = 0;
+  uint32_t q_offset = 0;  // element_offset / 4: added to the column-group word of the counters
+  Layout L;
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  bool own_memory = false;
+  unsigned char* base = nullptr;
+  float *x[2] = {nullptr, nullptr}, *c = nullptr;
+  uint32_t* thr = nullptr;
+  int32_t* last_nz = nullptr;
+  float* wtab = nullptr;
+  int32_t* trace = nullptr;
+  double* tel = nullptr;
+  double* partials = nullptr;
+  unsigned int* ticket = nullptr;
+  int cur = 0;  // index of the buffer holding the current replicas
+  int64_t rounds = 0;
+  int64_t trace_rounds = 0;
+  double alpha = 0, rho = 0, sigma = 0;
+  int objective = 1;
+  uint64_t seed = 0;
+  int policy_K = 20, policy_R = 20;
+  PhiloxKeys keys;
+  std::vector<double> P;      // policy in force
+  std::vector<uint8_t> adj;   // link graph in force
+  int sm_count = 148;
+  int64_t launches = 0;
+  std::string error;
+};
+
+namespace {
+
+int fail(netmax_ctx* ctx, int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (ctx) ctx->error = buf; else g_error = buf;
+  return code;
+}
+
+#define NM_CUDA(ctx, call)                                                                         \
+  do {                                                                                             \
+    cudaError_t e_ = (call);                                                                       \
+    if (e_ != cudaSuccess)                                                                         \
+      return fail(ctx, e_ == cudaErrorMemoryAllocation ? NETMAX_OOM : NETMAX_CUDA_ERROR, "%s: %s", \
+                  #call, cudaGetErrorString(e_));                                                  \
+  } while (0)
+
+// Link graph from speeds: d_im = 1 iff i != m and the speed is positive (symmetrised).
+int build_adjacency(netmax_ctx* ctx, int32_t M, const double* speed, std::vector<uint8_t>& adj) {
+  adj.assign((size_t)M * M, 0);
+  for (int i = 0; i < M; ++i)
+    for (int m = 0; m < M; ++m) {
+      if (i == m) continue;
+      if (!speed) { adj[(size_t)i * M + m] = 1; continue; }
+      const double a = speed[(size_t)i * M + m], b = speed[(size_t)m * M + i];
+      if (!std::isfinite(a) || !std::isfinite(b)) return fail(ctx, NETMAX_INVALID_ARG, "link speed (%d,%d) is not finite", i, m);
+      adj[(size_t)i * M + m] = (a > 0.0 && b > 0.0) ? 1 : 0;
+    }
+  // connectivity (Assumption 1) by a depth-first walk from worker 0
+  std::vector<int> stack{0};
+  std::vector<uint8_t> seen(M, 0);
+  seen[0] = 1;
+  int count = 1;
+  while (!stack.empty()) {
+    const int v = stack.back();
+    stack.pop_back();
+    for (int m = 0; m < M; ++m)
+      if (adj[(size_t)v * M + m] && !seen[m]) { seen[m] = 1; ++count; stack.push_back(m); }
+  }
+  if (count != M) return fail(ctx, NETMAX_NOT_CONNECTED, "link graph is not connected (%d of %d workers reachable)", count, M);
+  return NETMAX_OK;
+}
+
+int validate_policy(netmax_ctx* ctx, int32_t M, const double* P, const std::vector<uint8_t>& adj) {
+  for (int i = 0; i < M; ++i) {
+    double sum = 0.0;
+    for (int m = 0; m < M; ++m) {
+      const double p = P[(size_t)i * M + m];
+      if (!(p >= 0.0) || !std::isfinite(p)) return fail(ctx, NETMAX_BAD_PROB_ROW, "P[%d,%d] = %g is negative or not finite", i, m, p);
+      if (p > 0.0 && m != i && !adj[(size_t)i * M + m])
+        return fail(ctx, NETMAX_BAD_PROB_ROW, "P[%d,%d] > 0 on a missing link (Eq. 12)", i, m);
+      sum += p;
+    }
+    if (std::fabs(sum - 1.0) > 1e-9) return fail(ctx, NETMAX_BAD_PROB_ROW, "row %d of P sums to %.12g", i, sum);
+  }
+  return NETMAX_OK;
+}
+
+// rho <= 0: the largest rho that keeps Eq. 11 (p_im > alpha rho (d_im + d_mi)) with a 1e-6 margin.
+double default_rho(int32_t M, const double* P, const std::vector<uint8_t>& adj, double alpha) {
+  double best = INFINITY;
+  for (int i = 0; i < M; ++i)
+    for (int m = 0; m < M; ++m) {
+      const double p = P[(size_t)i * M + m];
+      if (i == m || !(p > 0.0)) continue;
+      const double dsum = (double)adj[(size_t)i * M + m] + (double)adj[(size_t)m * M + i];
+      best = std::min(best, p / (alpha * dsum));
+    }
+  return std::isfinite(best) ? (1.0 - 1e-6) * best : 0.0;
+}
+
+// T_j = floor(cum_j 2^32 + 1/2) over the left-to-right double prefix sums of the row,
+// non-decreasing, saturated, and pinned to the top from the last positive entry on.
+void build_tables(int32_t M, const double* P, const std::vector<uint8_t>& adj, double alpha32, double rho,
+                  std::vector<uint32_t>& thr, std::vector<int32_t>& last_nz, std::vector<float>& w) {
+  thr.resize((size_t)M * M);
+  last_nz.resize(M);
+  w.resize((size_t)M * M);
+  for (int i = 0; i < M; ++i) {
+    const double* p = P + (size_t)i * M;
+    int32_t last = -1;
+    for (int j = 0; j < M; ++j) if (p[j] > 0.0) last = j;
+    last_nz[i] = last;
+    double cum = 0.0;
+    uint64_t prev = 0;
+    for (int j = 0; j < M; ++j) {
+      cum += p[j];
+      uint64_t t = (uint64_t)std::floor(cum * 4294967296.0 + 0.5);
+      t = std::max(t, prev);
+      if (t > 0xFFFFFFFFull || j >= last) t = 0xFFFFFFFFull;
+      thr[(size_t)i * M + j] = (uint32_t)t;
+      prev = t;
+      float wv = 0.0f;
+      if (j != i && p[j] > 0.0) {
+        const double dsum = (double)adj[(size_t)i * M + j] + (double)adj[(size_t)j * M + i];
+        wv = (float)(alpha32 * rho * dsum / (2.0 * p[j]));   // alpha rho gamma_im   (Eq. 16)
+      }
+      w[(size_t)i * M + j] = wv;
+    }
+  }
+}
+
+int upload_policy(netmax_ctx* ctx) {
+  std::vector<uint32_t> thr;
+  std::vector<int32_t> last;
+  std::vector<float> w;
+  build_tables(ctx->M, ctx->P.data(), ctx->adj, (double)(float)ctx->alpha, ctx->rho, thr, last, w);
+  // pageable sources: the copies are complete (staged) when these calls return
+  NM_CUDA(ctx, cudaMemcpyAsync(ctx->thr, thr.data(), thr.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));
+  NM_CUDA(ctx, cudaMemcpyAsync(ctx->last_nz, last.data(), last.size() * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
+  NM_CUDA(ctx, cudaMemcpyAsync(ctx->wtab, w.data(), w.size() * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
+  NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  return NETMAX_OK;
+}
+
+// Chooses P and rho: the caller's, or Algorithm 3's.
+int resolve_policy(netmax_ctx* ctx, const double* speed, const double* prob, double rho) {
+  const int32_t M = ctx->M;
+  if (prob) {
+    int rc = validate_policy(ctx, M, prob, ctx->adj);
+    if (rc) return rc;
+    ctx->P.assign(prob, prob + (size_t)M * M);
+    ctx->rho = rho > 0.0 ? rho : default_rho(M, prob, ctx->adj, ctx->alpha);
+    return NETMAX_OK;
+  }
+  std::vector<double> t((size_t)M * M), flat;
+  std::vector<uint8_t> adj2((size_t)M * M);
+  if (!speed) {
+    flat.assign((size_t)M * M, 1.0);
+    speed = flat.data();
+  }
+  int rc = netmax_iteration_times(M, ctx->d, speed, t.data(), adj2.data());
+  if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
+  ctx->P.assign((size_t)M * M, 0.0);
+  double rho_sel = 0.0;
+  rc = netmax_policy_generate(M, t.data(), adj2.data(), ctx->alpha, ctx->policy_K, ctx->policy_R, ctx->P.data(), &rho_sel, nullptr);
+  if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
+  ctx->rho = rho > 0.0 ? rho : rho_sel;
+  return NETMAX_OK;
+}
+
+int launch_init(netmax_ctx* ctx, float* dst, double stddev, uint32_t tag) {
+  NM_CUDA(ctx, cudaMemsetAsync(dst, 0, (size_t)ctx->M * ctx->L.ld * sizeof(float), ctx->stream));
+  if (stddev == 0.0) return NETMAX_OK;
+  InitParams p;
+  p.dst = reinterpret_cast<float4*>(dst);
+  p.ldq = ctx->L.ldq;
+  p.nq = ctx->L.nq;
+  p.M = ctx->M;
+  p.tail = (int32_t)(ctx->d % 4);
+  p.stddev = (float)stddev;
+  p.tag = tag;
+  p.q_offset = ctx->q_offset;
+  p.keys = ctx->keys;
+  const int64_t total = (int64_t)ctx->M * ctx->L.nq;
+  const int grid = (int)std::min<int64_t>((total + kThreads - 1) / kThreads, (int64_t)ctx->sm_count * 16);
+  init_normal_kernel<<<grid, kThreads, 0, ctx->stream>>>(p);
+  ctx->launches += 1;
+  NM_CUDA(ctx, cudaGetLastError());
+  return NETMAX_OK;
+}
+
+int launch_sampler(netmax_ctx* ctx, uint64_t first_round, int64_t n_rounds, int32_t* out, int64_t slot0, int64_t ring) {
+  if (n_rounds <= 0) return NETMAX_OK;
+  SampleParams p;
+  p.thresholds = ctx->thr;
+  p.last_nz = ctx->last_nz;
+  p.out = out;
+  p.slot0 = slot0;
+  p.ring = ring;
+  p.first_round = first_round;
+  p.n_rounds = n_rounds;
+  p.M = ctx->M;
+  p.keys = ctx->keys;
+  const int64_t total = n_rounds * (int64_t)ctx->M;
+  const int grid = (int)std::min<int64_t>((total + kThreads - 1) / kThreads, (int64_t)ctx->sm_count * 32);
+  sample_peers_kernel<<<grid, kThreads, 0, ctx->stream>>>(p);
+  ctx->launches += 1;
+  NM_CUDA(ctx, cudaGetLastError());
+  return NETMAX_OK;
+}
+
+struct RoundPlan {
+  int cg = kThreads, rl = 1;
+  int grid = 1;
+  size_t smem = 0;
+  int64_t n_tiles = 0;
+};
+
+using RoundKernel = void (*)(const RoundParams);
+
+RoundKernel pick_kernel(int objective) {
+  return objective == 1 ? round_kernel<1, true, 4> : round_kernel<0, true, 4>;
+}
+
+// Tile shape: all M rows x cg column groups.  cg is the largest power of two (<= 256
+// threads' worth) that keeps the tile's share of x near 48 KB, so that a row fetched for
+// its own update is still close by in cache when another row pulls it as a peer; it is
+// reduced further while that leaves SMs without a tile.
+int plan_round(netmax_ctx* ctx, RoundPlan& plan) {
+  const int64_t M = ctx->M, nq = ctx->L.nq;
+  int cg = kThreads;
+  while (cg > 2 && (int64_t)cg * 16 * M > 48 * 1024) cg >>= 1;
+  while (cg > 2 && (nq + cg - 1) / cg < 2 * (int64_t)ctx->sm_count) cg >>= 1;
+  plan.cg = cg;
+  plan.rl = kThreads / cg;
+  plan.n_tiles = (nq + cg - 1) / cg;
+  plan.smem = align_up((size_t)M * 8, 16) + (plan.rl > 1 ? (size_t)kThreads * 32 : 0) + 64 * sizeof(double);
+  RoundKernel k = pick_kernel(ctx->objective);
+  if (plan.smem > 48 * 1024)
+    NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
+  int per_sm = 0;
+  NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, plan.smem));
+  if (per_sm < 1) return fail(ctx, NETMAX_CUDA_ERROR, "round kernel does not fit on an SM (smem %zu)", plan.smem);
+  plan.grid = (int)std::min<int64_t>(plan.n_tiles, std::min<int64_t>((int64_t)per_sm * ctx->sm_count, kMaxGrid));
+  return NETMAX_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int netmax_config_init(netmax_config* cfg) {
+  if (!cfg) return fail(nullptr, NETMAX_INVALID_ARG, "cfg is NULL");
+  std::memset(cfg, 0, sizeof *cfg);
+  cfg->objective = 1;
+  cfg->trace_rounds = 1024;
+  cfg->policy_K = 20;
+  cfg->policy_R = 20;
+  return NETMAX_OK;
+}
+
+static int check_sizes(const netmax_config* cfg) {
+  if (!cfg) return fail(nullptr, NETMAX_INVALID_ARG, "cfg is NULL");
+  if (cfg->M < 2 || cfg->M > kMaxM) return fail(nullptr, NETMAX_INVALID_ARG, "M = %d outside [2, %lld]", cfg->M, (long long)kMaxM);
+  if (cfg->d < 1 || cfg->d >= kMaxD) return fail(nullptr, NETMAX_INVALID_ARG, "d = %lld outside [1, 2^33)", (long long)cfg->d);
+  if (cfg->element_offset < 0 || cfg->element_offset % 4 != 0 || cfg->element_offset + cfg->d >= kMaxD)
+    return fail(nullptr, NETMAX_INVALID_ARG, "element_offset = %lld must be a non-negative multiple of 4 with offset + d < 2^33", (long long)cfg->element_offset);
+  if (cfg->trace_rounds < 1) return fail(nullptr, NETMAX_INVALID_ARG, "trace_rounds = %lld < 1", (long long)cfg->trace_rounds);
+  return NETMAX_OK;
+}
+
+int netmax_workspace_size(const netmax_config* cfg, size_t* bytes) {
+  int rc = check_sizes(cfg);
+  if (rc) return rc;
+  if (!bytes) return fail(nullptr, NETMAX_INVALID_ARG, "bytes is NULL");
+  *bytes = make_layout(cfg->M, cfg->d, cfg->trace_rounds).total;
+  return NETMAX_OK;
+}
+
+int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
+  if (!out) return fail(nullptr, NETMAX_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  int rc = check_sizes(cfg);
+  if (rc) return rc;
+  if (!(cfg->lr > 0.0) || !std::isfinite(cfg->lr)) return fail(nullptr, NETMAX_INVALID_ARG, "lr = %g must be positive and finite", cfg->lr);
+  if (!(cfg->sigma >= 0.0) || !std::isfinite(cfg->sigma)) return fail(nullptr, NETMAX_INVALID_ARG, "sigma = %g must be >= 0 and finite", cfg->sigma);
+  if (!(cfg->x0_std >= 0.0) || !std::isfinite(cfg->x0_std) || !(cfg->c_std >= 0.0) || !std::isfinite(cfg->c_std))
+    return fail(nullptr, NETMAX_INVALID_ARG, "x0_std and c_std must be >= 0 and finite");
+  if (!std::isfinite(cfg->rho)) return fail(nullptr, NETMAX_INVALID_ARG, "rho is not finite");
+  if (cfg->objective != 0 && cfg->objective != 1) return fail(nullptr, NETMAX_INVALID_ARG, "objective = %d is not 0 or 1", cfg->objective);
+  if (cfg->device < 0) return fail(nullptr, NETMAX_INVALID_ARG, "device = %d", cfg->device);
+
+  netmax_ctx* ctx = new (std::nothrow) netmax_ctx();
+  if (!ctx) return fail(nullptr, NETMAX_OOM, "host allocation failed");
+  auto bail = [&](int code) {
+    g_error = ctx->error;
+    netmax_destroy(ctx);
+    return code;
+  };
+  ctx->M = cfg->M;
+  ctx->d = cfg->d;
+  ctx->q_offset = (uint32_t)(cfg->element_offset / 4);
+  ctx->device = cfg->device;
+  ctx->stream = (cudaStream_t)cfg->stream;
+  ctx->trace_rounds = cfg->trace_rounds;
+  ctx->alpha = cfg->lr;
+  ctx->sigma = cfg->sigma;
+  ctx->objective = cfg->objective;
+  ctx->seed = cfg->seed;
+  ctx->policy_K = cfg->policy_K > 0 ? cfg->policy_K : 20;
+  ctx->policy_R = cfg->policy_R > 0 ? cfg->policy_R : 20;
+  ctx->keys = make_philox_keys(cfg->seed);
+  ctx->L = make_layout(cfg->M, cfg->d, cfg->trace_rounds);
+
+  rc = build_adjacency(ctx, cfg->M, cfg->link_speed_gbps, ctx->adj);
+  if (rc) return bail(rc);
+  rc = resolve_policy(ctx, cfg->link_speed_gbps, cfg->prob, cfg->rho);
+  if (rc) return bail(rc);
+
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+    cudaGetLastError();
+    ctx->error = "no CUDA device is available";
+    return bail(NETMAX_CUDA_ERROR);
+  }
+  if (cfg->device >= ndev) { ctx->error = "device ordinal out of range"; return bail(NETMAX_INVALID_ARG); }
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) { ctx->error = "cudaSetDevice failed"; return bail(NETMAX_CUDA_ERROR); }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, cfg->device) == cudaSuccess) ctx->sm_count = prop.multiProcessorCount;
+  if (cfg->workspace) {
+    if (((uintptr_t)cfg->workspace & 255) != 0) { ctx->error = "workspace is not 256-byte aligned"; return bail(NETMAX_INVALID_ARG); }
+    if (cfg->workspace_bytes < ctx->L.total) {
+      char buf[128];
+      snprintf(buf, sizeof buf, "workspace holds %zu bytes, %zu needed", cfg->workspace_bytes, ctx->L.total);
+      ctx->error = buf;
+      return bail(NETMAX_OOM);
+    }
+    ctx->base = (unsigned char*)cfg->workspace;
+  } else {
+    void* ptr = nullptr;
+    cudaError_t e = cudaMalloc(&ptr, ctx->L.total);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      char buf[160];
+      snprintf(buf, sizeof buf, "cudaMalloc of %zu bytes failed: %s", ctx->L.total, cudaGetErrorString(e));
+      ctx->error = buf;
+      return bail(NETMAX_OOM);
+    }
+    ctx->base = (unsigned char*)ptr;
+    ctx->own_memory = true;
+  }
+  const Layout& L = ctx->L;
+  ctx->x[0] = (float*)(ctx->base + L.off_x0);
+  ctx->x[1] = (float*)(ctx->base + L.off_x1);
+  ctx->c = (float*)(ctx->base + L.off_c);
+  ctx->thr = (uint32_t*)(ctx->base + L.off_thr);
+  ctx->last_nz = (int32_t*)(ctx->base + L.off_last);
+  ctx->wtab = (float*)(ctx->base + L.off_w);
+  ctx->trace = (int32_t*)(ctx->base + L.off_trace);
+  ctx->tel = (double*)(ctx->base + L.off_tel);
+  ctx->partials = (double*)(ctx->base + L.off_partials);
+  ctx->ticket = (unsigned int*)(ctx->base + L.off_ticket);
+
+  auto step = [&](cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return true;
+    ctx->error = std::string(what) + ": " + cudaGetErrorString(e);
+    return false;
+  };
+  if (!step(cudaMemsetAsync(ctx->ticket, 0, 256, ctx->stream), "cudaMemsetAsync(ticket)")) return bail(NETMAX_CUDA_ERROR);
+  if (!step(cudaMemsetAsync(ctx->x[1], 0, (size_t)ctx->M * L.ld * sizeof(float), ctx->stream), "cudaMemsetAsync(x)")) return bail(NETMAX_CUDA_ERROR);
+  if (!step(cudaMemsetAsync(ctx->tel, 0, (size_t)ctx->trace_rounds * 2 * sizeof(double), ctx->stream), "cudaMemsetAsync(tel)")) return bail(NETMAX_CUDA_ERROR);
+  rc = upload_policy(ctx);
+  if (rc) return bail(rc);
+  rc = launch_init(ctx, ctx->x[0], cfg->x0_std, kTagX0);
+  if (rc) return bail(rc);
+  rc = launch_init(ctx, ctx->c, cfg->c_std, kTagC);
+  if (rc) return bail(rc);
+  if (!step(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize")) return bail(NETMAX_CUDA_ERROR);
+  *out = ctx;
+  return NETMAX_OK;
+}
+
+int netmax_create(int32_t M, int64_t d, const double* link_speed_gbps, const double* prob, double lr, uint64_t seed,
+                  netmax_ctx** out) {
+  netmax_config cfg;
+  netmax_config_init(&cfg);
+  cfg.M = M;
+  cfg.d = d;
+  cfg.link_speed_gbps = link_speed_gbps;
+  cfg.prob = prob;
+  cfg.lr = lr;
+  cfg.seed = seed;
+  cfg.x0_std = 1.0;
+  cfg.c_std = 1.0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cfg.device = dev; else cudaGetLastError();
+  return netmax_create_ex(&cfg, out);
+}
+
+void netmax_destroy(netmax_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->own_memory && ctx->base) {
+    DeviceGuard guard(ctx->device);
+    cudaStreamSynchronize(ctx->stream);
+    cudaFree(ctx->base);
+    cudaGetLastError();
+  }
+  delete ctx;
+}
+
+int netmax_set_policy(netmax_ctx* ctx, const double* link_speed_gbps, const double* prob, double rho) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (!std::isfinite(rho)) return fail(ctx, NETMAX_INVALID_ARG, "rho is not finite");
+  DeviceGuard guard(ctx->device);
+  std::vector<uint8_t> old_adj = ctx->adj;
+  std::vector<double> old_P = ctx->P;
+  const double old_rho = ctx->rho;
+  int rc = NETMAX_OK;
+  if (link_speed_gbps) rc = build_adjacency(ctx, ctx->M, link_speed_gbps, ctx->adj);
+  if (!rc) rc = resolve_policy(ctx, link_speed_gbps, prob, rho);
+  if (rc) {  // leave the policy in force untouched
+    ctx->adj.swap(old_adj);
+    ctx->P.swap(old_P);
+    ctx->rho = old_rho;
+    return rc;
+  }
+  // rounds already enqueued still read the old tables: wait for them before overwriting
+  NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  return upload_policy(ctx);
+}
+
+int netmax_get_policy(netmax_ctx* ctx, double* prob_out, double* rho_out) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (prob_out) std::memcpy(prob_out, ctx->P.data(), ctx->P.size() * sizeof(double));
+  if (rho_out) *rho_out = ctx->rho;
+  return NETMAX_OK;
+}
+
+static int copy_in(netmax_ctx* ctx, float* dst, const float* host) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (!host) return fail(ctx, NETMAX_INVALID_ARG, "host pointer is NULL");
+  DeviceGuard guard(ctx->device);
+  NM_CUDA(ctx, cudaMemcpy2DAsync(dst, (size_t)ctx->L.ld * sizeof(float), host, (size_t)ctx->d * sizeof(float),
+                                 (size_t)ctx->d * sizeof(float), (size_t)ctx->M, cudaMemcpyHostToDevice, ctx->stream));
+  return NETMAX_OK;
+}
+
+static int copy_out(netmax_ctx* ctx, const float* src, float* host) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (!host) return fail(ctx, NETMAX_INVALID_ARG, "host pointer is NULL");
+  DeviceGuard guard(ctx->device);
+  NM_CUDA(ctx, cudaMemcpy2DAsync(host, (size_t)ctx->d * sizeof(float), src, (size_t)ctx->L.ld * sizeof(float),
+                                 (size_t)ctx->d * sizeof(float), (size_t)ctx->M, cudaMemcpyDeviceToHost, ctx->stream));
+  NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  return NETMAX_OK;
+}
+
+int netmax_set_replicas(netmax_ctx* ctx, const float* host_x) { return copy_in(ctx, ctx ? ctx->x[ctx->cur] : nullptr, host_x); }
+int netmax_set_centres(netmax_ctx* ctx, const float* host_c) { return copy_in(ctx, ctx ? ctx->c : nullptr, host_c); }
+int netmax_read_replicas(netmax_ctx* ctx, float* host_out) { return copy_out(ctx, ctx ? ctx->x[ctx->cur] : nullptr, host_out); }
+int netmax_read_centres(netmax_ctx* ctx, float* host_out) { return copy_out(ctx, ctx ? ctx->c : nullptr, host_out); }
+
+int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (n_rounds < 0) return fail(ctx, NETMAX_INVALID_ARG, "n_rounds = %lld < 0", (long long)n_rounds);
+  if (n_rounds == 0) return NETMAX_OK;
+  if ((uint64_t)(ctx->rounds + n_rounds) >= ((uint64_t)1 << 56)) return fail(ctx, NETMAX_INVALID_ARG, "round counter would exceed 2^56");
+  DeviceGuard guard(ctx->device);
+  RoundPlan plan;
+  int rc = plan_round(ctx, plan);
+  if (rc) return rc;
+  RoundKernel kernel = pick_kernel(ctx->objective);
+
+  RoundParams p;
+  p.c = reinterpret_cast<const float4*>(ctx->c);
+  p.wtab = ctx->wtab;
+  p.partials = ctx->partials;
+  p.ticket = ctx->ticket;
+  p.ldq = ctx->L.ldq;
+  p.nq = ctx->L.nq;
+  p.n_tiles = plan.n_tiles;
+  p.M = ctx->M;
+  p.tail = (int32_t)(ctx->d % 4);
+  p.cg = plan.cg;
+  p.rl = plan.rl;
+  p.alpha = (float)ctx->alpha;
+  p.sigma = (float)ctx->sigma;
+  p.inv_M = 1.0f / (float)ctx->M;
+  p.q_offset = ctx->q_offset;
+  p.keys = ctx->keys;
+
+  int64_t done = 0;
+  while (done < n_rounds) {
+    // peers of a batch of rounds in one launch (counter-based draws do not depend on x),
+    // at most one lap of the ring at a time
+    const int64_t batch = std::min<int64_t>(n_rounds - done, ctx->trace_rounds);
+    rc = launch_sampler(ctx, (uint64_t)ctx->rounds, batch, ctx->trace, ctx->rounds % ctx->trace_rounds, ctx->trace_rounds);
+    if (rc) return rc;
+    for (int64_t b = 0; b < batch; ++b) {
+      const uint64_t r = (uint64_t)ctx->rounds;
+      const int64_t slot = (int64_t)(r % (uint64_t)ctx->trace_rounds);
+      p.x_cur = reinterpret_cast<const float4*>(ctx->x[ctx->cur]);
+      p.x_nxt = reinterpret_cast<float4*>(ctx->x[ctx->cur ^ 1]);
+      p.peers = ctx->trace + slot * ctx->M;
+      p.tel_out = ctx->tel + 2 * slot;
+      p.round_lo = (uint32_t)r;
+      p.ctr3 = philox_ctr3(kTagNoise, r);
+      kernel<<<plan.grid, kThreads, plan.smem, ctx->stream>>>(p);
+      ctx->launches += 1;
+      ctx->cur ^= 1;
+      ctx->rounds += 1;
+    }
+    NM_CUDA(ctx, cudaGetLastError());
+    done += batch;
+  }
+  return NETMAX_OK;
+}
+
+int64_t netmax_rounds_done(const netmax_ctx* ctx) { return ctx ? ctx->rounds : -1; }
+
+int netmax_read_columns(netmax_ctx* ctx, const int64_t* host_cols, int64_t n_cols, float* host_out) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (n_cols < 0 || (n_cols > 0 && (!host_cols || !host_out))) return fail(ctx, NETMAX_INVALID_ARG, "bad column list");
+  if (n_cols == 0) return NETMAX_OK;
+  for (int64_t k = 0; k < n_cols; ++k)
+    if (host_cols[k] < 0 || host_cols[k] >= ctx->d) return fail(ctx, NETMAX_INVALID_ARG, "cols[%lld] = %lld outside [0, d)", (long long)k, (long long)host_cols[k]);
+  DeviceGuard guard(ctx->device);
+  int64_t* d_cols = nullptr;
+  float* d_out = nullptr;
+  NM_CUDA(ctx, cudaMalloc(&d_cols, (size_t)n_cols * sizeof(int64_t)));
+  cudaError_t e = cudaMalloc(&d_out, (size_t)n_cols * ctx->M * sizeof(float));
+  if (e != cudaSuccess) { cudaFree(d_cols); cudaGetLastError(); return fail(ctx, NETMAX_OOM, "cudaMalloc failed: %s", cudaGetErrorString(e)); }
+  int rc = NETMAX_OK;
+  const int64_t total = n_cols * ctx->M;
+  const int grid = (int)std::min<int64_t>((total + kThreads - 1) / kThreads, 4096);
+  e = cudaMemcpyAsync(d_cols, host_cols, (size_t)n_cols * sizeof(int64_t), cudaMemcpyHostToDevice, ctx->stream);
+  if (e == cudaSuccess) {
+    gather_columns_kernel<<<grid, kThreads, 0, ctx->stream>>>(ctx->x[ctx->cur], ctx->L.ld, ctx->M, d_cols, n_cols, d_out);
+    ctx->launches += 1;
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(host_out, d_out, (size_t)total * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) rc = fail(ctx, NETMAX_CUDA_ERROR, "read_columns: %s", cudaGetErrorString(e));
+  cudaFree(d_cols);
+  cudaFree(d_out);
+  return rc;
+}
+
+static int ring_range(netmax_ctx* ctx, int64_t first, int64_t n) {
+  if (first < 0 || n < 0 || first + n > ctx->rounds || first < ctx->rounds - ctx->trace_rounds)
+    return fail(ctx, NETMAX_TRACE_RANGE, "rounds [%lld, %lld) are not in the ring (rounds done %lld, capacity %lld)",
+                (long long)first, (long long)(first + n), (long long)ctx->rounds, (long long)ctx->trace_rounds);
+  return NETMAX_OK;
+}
+
+int netmax_peer_trace(netmax_ctx* ctx, int64_t first_round, int64_t n, int32_t* host_out) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  int rc = ring_range(ctx, first_round, n);
+  if (rc) return rc;
+  if (n == 0) return NETMAX_OK;
+  if (!host_out) return fail(ctx, NETMAX_INVALID_ARG, "host_out is NULL");
+  DeviceGuard guard(ctx->device);
+  NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  const size_t row = (size_t)ctx->M * sizeof(int32_t);
+  int64_t r = first_round;
+  while (r < first_round + n) {  // at most two contiguous pieces of the ring
+    const int64_t slot = r % ctx->trace_rounds;
+    const int64_t piece = std::min<int64_t>(first_round + n - r, ctx->trace_rounds - slot);
+    NM_CUDA(ctx, cudaMemcpy(host_out + (size_t)(r - first_round) * ctx->M, ctx->trace + (size_t)slot * ctx->M, piece * row, cudaMemcpyDeviceToHost));
+    r += piece;
+  }
+  return NETMAX_OK;
+}
+
+int netmax_telemetry(netmax_ctx* ctx, int64_t first_round, int64_t n, double* host_consensus, double* host_loss) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  int rc = ring_range(ctx, first_round, n);
+  if (rc) return rc;
+  if (n == 0) return NETMAX_OK;
+  DeviceGuard guard(ctx->device);
+  NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  std::vector<double> ring((size_t)ctx->trace_rounds * 2);
+  NM_CUDA(ctx, cudaMemcpy(ring.data(), ctx->tel, ring.size() * sizeof(double), cudaMemcpyDeviceToHost));
+  for (int64_t k = 0; k < n; ++k) {
+    const int64_t slot = (first_round + k) % ctx->trace_rounds;
+    if (host_consensus) host_consensus[k] = ring[2 * slot];
+    if (host_loss) host_loss[k] = ring[2 * slot + 1];
+  }
+  return NETMAX_OK;
+}
+
+int netmax_replicas_device(netmax_ctx* ctx, const float** x, int64_t* ld) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (!x || !ld) return fail(ctx, NETMAX_INVALID_ARG, "output pointer is NULL");
+  *x = ctx->x[ctx->cur];
+  *ld = ctx->L.ld;
+  return NETMAX_OK;
+}
+
+int netmax_sample_peers(netmax_ctx* ctx, int64_t first_round, int64_t n_rounds, int32_t* device_out) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (first_round < 0 || n_rounds < 0 || (n_rounds > 0 && !device_out)) return fail(ctx, NETMAX_INVALID_ARG, "bad range or NULL output");
+  DeviceGuard guard(ctx->device);
+  return launch_sampler(ctx, (uint64_t)first_round, n_rounds, device_out, 0, INT64_MAX);
+}
+
+int64_t netmax_kernel_launches(const netmax_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+const char* netmax_last_error(const netmax_ctx* ctx) { return ctx ? ctx->error.c_str() : g_error.c_str(); }
+
+}  // extern "C"

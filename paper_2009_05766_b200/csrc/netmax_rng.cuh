@@ -1,0 +1,107 @@
+// Device-side random numbers of the NetMax round simulator: Philox4x32-10 (Salmon, Moraes,
+// Dror, Shaw, SC'11) and a Box-Muller transform on fixed-point uniforms.
+//
+// The paper only assumes additive gradient noise with zero mean and bounded variance
+// (Assumption 1); the generator, the counter layout and the uniform-to-normal map are this
+// library's choice and are documented in the C header's conventions.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace netmax {
+
+constexpr uint32_t kPhiloxMul0 = 0xD2511F53u;
+constexpr uint32_t kPhiloxMul1 = 0xCD9E8D57u;
+constexpr uint32_t kPhiloxWeyl0 = 0x9E3779B9u;
+constexpr uint32_t kPhiloxWeyl1 = 0xBB67AE85u;
+
+// Streams (fourth counter word, low byte).
+constexpr uint32_t kTagPeer = 1, kTagNoise = 2, kTagX0 = 3, kTagC = 4;
+
+// The ten round keys of one seed, expanded once on the host (the key schedule does not
+// depend on the counter, so every thread shares it).
+struct PhiloxKeys {
+  uint32_t k0[10];
+  uint32_t k1[10];
+};
+
+inline PhiloxKeys make_philox_keys(uint64_t seed) {
+  PhiloxKeys k;
+  uint32_t a = (uint32_t)seed, b = (uint32_t)(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    k.k0[r] = a;
+    k.k1[r] = b;
+    a += kPhiloxWeyl0;
+    b += kPhiloxWeyl1;
+  }
+  return k;
+}
+
+// Counter layout: (column group e/4, worker, round low word, tag | round high bits << 8).
+__host__ __device__ __forceinline__ uint32_t philox_ctr3(uint32_t tag, uint64_t round) {
+  return tag | ((uint32_t)(round >> 32) << 8);
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               const PhiloxKeys& keys) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(kPhiloxMul0, c0), lo0 = kPhiloxMul0 * c0;
+    const uint32_t hi1 = __umulhi(kPhiloxMul1, c2), lo1 = kPhiloxMul1 * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ keys.k0[r];
+    const uint32_t n2 = hi0 ^ c3 ^ keys.k1[r];
+    c0 = n0;
+    c1 = lo1;
+    c2 = n2;
+    c3 = lo0;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+// u1 = (top23(a) + 1/2) / 2^23 in (0,1), exactly representable in fp32:
+// bits 0x3F800000 | top23 are the float 1 + top23 / 2^23; subtracting 1 - 2^-24 is exact.
+__device__ __forceinline__ float radius_uniform(uint32_t a) {
+  return __uint_as_float(0x3F800000u | (a >> 9)) - 0.99999994039535522461f;
+}
+
+// Fast pair: hardware log2 / sin / cos / sqrt approximations.  The absolute error of each
+// normal is about 2e-7 for typical radii and is bounded by 6e-4 for radii below 1e-3
+// (probability 5e-7), far inside the replica tolerance after scaling by alpha*sigma.
+__device__ __forceinline__ void normal_pair_fast(uint32_t a, uint32_t b, float& z0, float& z1) {
+  const float u1 = radius_uniform(a);
+  // angle = 2 pi u2 with u2 = top24(b)/2^24 taken modulo 1 into [-1/2, 1/2)
+  const float ang = (float)((int32_t)b >> 8) * 3.74507028e-07f;  // 2 pi / 2^24
+  const float r2 = fmaxf(-1.38629436111989f * __log2f(u1), 0.0f);  // -2 ln 2 * log2(u1)
+  float rad;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(r2));
+  float s, c;
+  __sincosf(ang, &s, &c);
+  z0 = rad * c;
+  z1 = rad * s;
+}
+
+// Accurate pair (library logf / sincospif / sqrtf): used where speed does not matter.
+__device__ __forceinline__ void normal_pair_accurate(uint32_t a, uint32_t b, float& z0, float& z1) {
+  const float u1 = radius_uniform(a);
+  const float turns2 = (float)((int32_t)b >> 8) * 1.1920928955078125e-07f;  // 2 u2 in [-1, 1)
+  const float rad = sqrtf(-2.0f * logf(u1));
+  float s, c;
+  sincospif(turns2, &s, &c);
+  z0 = rad * c;
+  z1 = rad * s;
+}
+
+template <bool kFast>
+__device__ __forceinline__ float4 normals4(uint4 r) {
+  float4 z;
+  if (kFast) {
+    normal_pair_fast(r.x, r.y, z.x, z.y);
+    normal_pair_fast(r.z, r.w, z.z, z.w);
+  } else {
+    normal_pair_accurate(r.x, r.y, z.x, z.y);
+    normal_pair_accurate(r.z, r.w, z.z, z.w);
+  }
+  return z;
+}
+
+}  // namespace netmax

@@ -1,0 +1,126 @@
+"""CPU-side checks of the CUDA library: it loads, exports what the header declares, its host
+control plane (iteration times, Algorithm 3, validation) agrees with the oracle.  No kernel runs."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import policy as opolicy
+from paper_2009_05766_b200 import binding, workloads
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "netmax.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = sorted(set(re.findall(r"\b(netmax_[a-z_]+)\s*\(", header)))
+    assert len(declared) >= 20
+    L = binding.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+    assert sorted(binding.EXPORTS) == declared
+
+
+def test_iteration_times_match_oracle():
+    for idx in (1, 2, 3, 4):
+        w = workloads.config(idx)
+        s = w.link_speeds(0)
+        t, adj = binding.netmax_iteration_times(s, w.d)
+        t0, adj0 = opolicy.iteration_times(s, w.d)
+        np.testing.assert_allclose(t, t0, rtol=1e-15)
+        assert (adj == adj0).all()
+
+
+def _policy_case(name):
+    if name.startswith("cfg"):
+        w = workloads.config(int(name[3]))
+        K, R = {1: (20, 20), 2: (10, 10), 3: (6, 6), 4: (3, 3)}[w.index]
+        return opolicy.iteration_times(w.link_speeds(1 if w.index == 3 else 0), w.d) + (w.lr, K, R)
+    rng = np.random.default_rng(5)
+    M = 7
+    s = np.triu(np.exp(rng.uniform(np.log(1.0), np.log(50.0), (M, M))), 1)
+    s[0, 4] = s[1, 5] = s[2, 6] = 0.0
+    return opolicy.iteration_times(s + s.T, 1_000_000) + (0.05, 8, 8)
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4", "sparse7"])
+def test_policy_generator_matches_oracle(name):
+    t, adj, lr, K, R = _policy_case(name)
+    P, rho, info = binding.netmax_policy_generate(t, adj, lr, K, R)
+    P0, rho0, info0 = opolicy.generate_policy(t, adj, lr, K, R)
+    assert (info["k"], info["r"]) == (info0["k"], info0["r"])
+    assert rho == pytest.approx(rho0, rel=1e-14)
+    np.testing.assert_allclose(P, P0, atol=1e-9)
+    assert info["lam2"] == pytest.approx(info0["lam2"], abs=1e-9)
+    assert info["t_conv"] == pytest.approx(info0["t_conv"], rel=1e-6)
+    np.testing.assert_allclose(P.sum(axis=1), 1.0, atol=1e-12)
+
+
+def test_lanczos_path_of_the_library_agrees_with_dense_eigenvalues():
+    """M > 96 switches the library's lambda_2 to Lanczos; the oracle uses a dense solver."""
+    M = 128
+    rng = np.random.default_rng(9)
+    s = np.triu(np.exp(rng.uniform(np.log(1.0), np.log(100.0), (M, M))), 1)
+    t, adj = opolicy.iteration_times(s + s.T, 1_000_000)
+    P, rho, info = binding.netmax_policy_generate(t, adj, 0.05, 2, 2)
+    Y = opolicy.y_matrix(P, opolicy.node_probabilities(P, t, adj), adj, 0.05, rho)
+    assert info["lam2"] == pytest.approx(np.linalg.eigvalsh(Y)[-2], abs=1e-9)
+
+
+def test_policy_generate_rejects_bad_arguments():
+    t, adj = opolicy.iteration_times(np.ones((3, 3)) - np.eye(3), 100)
+    with pytest.raises(binding.NetmaxError) as e:
+        binding.netmax_policy_generate(t, adj, -0.1, 4, 4)
+    assert e.value.code == -1
+    lone = adj.copy()
+    lone[0, :] = lone[:, 0] = 0
+    with pytest.raises(binding.NetmaxError) as e:
+        binding.netmax_policy_generate(t, lone, 0.1, 4, 4)
+    assert e.value.code == -6
+    with pytest.raises(binding.NetmaxError) as e:
+        binding.netmax_iteration_times(np.zeros((3, 3)), 10)
+    assert e.value.code == -6
+
+
+def test_create_validates_before_touching_the_gpu():
+    M = 3
+    good = np.array([[0, .5, .5], [.5, 0, .5], [.5, .5, 0]])
+    cases = [
+        (dict(M=1, d=8, lr=0.1, prob=None), -1),
+        (dict(M=M, d=0, lr=0.1, prob=good), -1),
+        (dict(M=M, d=8, lr=0.0, prob=good), -1),
+        (dict(M=M, d=8, lr=0.1, prob=good, sigma=-1.0), -1),
+        (dict(M=M, d=8, lr=0.1, prob=good, objective=2), -1),
+        (dict(M=M, d=8, lr=0.1, prob=good, trace_rounds=0), -1),
+        (dict(M=M, d=8, lr=0.1, prob=good * 0.9), -2),
+        (dict(M=M, d=8, lr=0.1, prob=np.array([[0, 1.5, -.5], [.5, 0, .5], [.5, .5, 0]])), -2),
+        (dict(M=M, d=8, lr=0.1, prob=good, link_speed_gbps=np.array([[0, 1, 0], [1, 0, 1], [0, 1, 0.]])), -2),
+        (dict(M=M, d=8, lr=0.1, prob=None, link_speed_gbps=np.array([[0, 1, 0], [1, 0, 0], [0, 0, 0.]])), -6),
+    ]
+    for kw, code in cases:
+        with pytest.raises(binding.NetmaxError) as e:
+            binding.Netmax(**kw)
+        assert e.value.code == code, (kw, str(e.value))
+
+
+def test_null_context_calls_return_errors_not_crashes():
+    L = binding.lib()
+    assert L.netmax_round(None, 1) == -1
+    assert L.netmax_read_replicas(None, None) == -1
+    assert L.netmax_rounds_done(None) == -1
+    assert L.netmax_create_ex(None, None) == -1
+    L.netmax_destroy(None)
+    size = binding.Netmax.workspace_size(8, 1000, 16)
+    assert size >= 3 * 8 * 1024 * 4 and size % 256 == 0
+
+
+def test_product_path_fails_loudly_without_a_gpu(gpu_available):
+    if gpu_available:
+        pytest.skip("a GPU is present")
+    good = np.array([[0, 1.0], [1.0, 0]])
+    with pytest.raises(binding.NetmaxError) as e:
+        binding.Netmax(M=2, d=8, lr=0.1, prob=good)
+    assert e.value.code == -4
