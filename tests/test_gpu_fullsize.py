@@ -68,7 +68,7 @@ def test_full_size_configs_on_sampled_columns(nm, idx):
         P, rho, _ = opolicy.generate_policy(t, adj, w.lr, w.K if idx != 4 else 4, w.R if idx != 4 else 4)
         if g is None:
             g = nm.Netmax(M=w.M, d=w.d, lr=w.lr, link_speed_gbps=s, prob=P, rho=rho, sigma=w.sigma,
-                          x0_std=w.x0_std, c_std=w.c_std, objective=1, seed=w.seed, trace_rounds=w.rounds)
+                          x0_std=w.x0_std, c_std=w.c_std, objective=1, seed=w.seed, trace_rounds=w.rounds + 1)
             o = oracle.Sim(w.M, w.d, P, adj, alpha=w.lr, rho=rho, sigma=w.sigma, objective=1, seed=w.seed, cols=cols)
             o.init(w.x0_std, w.c_std)
         else:
@@ -100,7 +100,7 @@ def test_full_size_sampling_stress_config(nm):
     P = s / s.sum(axis=1, keepdims=True)      # dense heterogeneous rows: an input, not Algorithm 3
     cols = workloads.sample_columns(w.d, 40, w.seed)
     g = nm.Netmax(M=w.M, d=w.d, lr=w.lr, prob=P, sigma=w.sigma, x0_std=w.x0_std, c_std=w.c_std, objective=1,
-                  seed=w.seed, trace_rounds=rounds)
+                  seed=w.seed, trace_rounds=rounds + 1)
     _, rho = g.get_policy()
     o = oracle.Sim(w.M, w.d, P, (1 - np.eye(w.M)).astype(np.uint8), alpha=w.lr, rho=rho, sigma=w.sigma, objective=1,
                    seed=w.seed, cols=cols)
