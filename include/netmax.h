@@ -141,6 +141,38 @@ int netmax_read_centres(netmax_ctx* ctx, float* host_out);
 int netmax_read_columns(netmax_ctx* ctx, const int64_t* host_cols, int64_t n_cols, float* host_out);
 
 /*
+ * netmax_read_columns without any allocation.  (The paper has no counterpart: this is a
+ * convenience of the library, like netmax_read_columns itself.)
+ *
+ * netmax_read_columns stages the column list and the gathered values in temporaries that it
+ * cudaMallocs and frees on every call.  Some callers must not do that: a process whose
+ * device memory is entirely handed to a pool allocator (the reason netmax_config.workspace
+ * exists) can see cudaMalloc fail or take memory the pool counts on; a monitoring loop that
+ * polls a few parameters between rounds does not want the device-wide synchronisation that
+ * cudaMalloc / cudaFree imply; and code that runs where the CUDA runtime forbids allocation
+ * cannot call it at all.  This variant runs the same gather kernel, but stages through a
+ * fixed array that lives in the library image (a file-scope __device__ array of
+ * NETMAX_STATIC_MAX_COLS * 8 + NETMAX_STATIC_MAX_VALUES * 4 bytes, about 1.03 MB, present on
+ * every GPU that loads the library until the process exits).  It calls no cudaMalloc,
+ * cudaFree or other allocating routine.
+ *
+ * Arguments and result are those of netmax_read_columns.  Limits: n_cols <=
+ * NETMAX_STATIC_MAX_COLS and M * n_cols <= NETMAX_STATIC_MAX_VALUES; beyond either the call
+ * returns NETMAX_INVALID_ARG and touches nothing (split the list and call again).
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress,
+ * once per device, cached); make that first call before any stream capture begins.  All
+ * calls, from every context on the device, share the one array: it still holds the previous
+ * call's data (nothing in it needs to start at zero, every slot that is read back is
+ * written first), and two calls whose GPU work overlaps -- different streams, or different
+ * host threads -- race on it.  Calls on one stream are ordered and safe.  Synchronises the
+ * context's stream before returning, like netmax_read_columns.
+ */
+#define NETMAX_STATIC_MAX_COLS 4096
+#define NETMAX_STATIC_MAX_VALUES 262144
+int netmax_read_columns_static(netmax_ctx* ctx, const int64_t* host_cols, int64_t n_cols, float* host_out);
+
+/*
  * Peers drawn in rounds [first_round, first_round + n): host_out[(r - first_round) * M + i]
  * is the peer of worker i in round r.  Only the last trace_rounds rounds are kept;
  * NETMAX_TRACE_RANGE otherwise.  Synchronises.

@@ -22,6 +22,7 @@ EXPORTS = [
     "netmax_config_init", "netmax_workspace_size", "netmax_create_ex", "netmax_create", "netmax_destroy",
     "netmax_set_policy", "netmax_get_policy", "netmax_set_replicas", "netmax_set_centres", "netmax_round",
     "netmax_rounds_done", "netmax_read_replicas", "netmax_read_centres", "netmax_read_columns",
+    "netmax_read_columns_static",
     "netmax_peer_trace", "netmax_telemetry", "netmax_replicas_device", "netmax_sample_peers",
     "netmax_iteration_times", "netmax_policy_generate", "netmax_kernel_launches", "netmax_last_error",
 ]
@@ -74,6 +75,7 @@ def lib():
             "netmax_read_replicas": ([vp, vp], C.c_int),
             "netmax_read_centres": ([vp, vp], C.c_int),
             "netmax_read_columns": ([vp, vp, i64, vp], C.c_int),
+            "netmax_read_columns_static": ([vp, vp, i64, vp], C.c_int),
             "netmax_peer_trace": ([vp, i64, i64, vp], C.c_int),
             "netmax_telemetry": ([vp, i64, i64, vp, vp], C.c_int),
             "netmax_replicas_device": ([vp, vp, vp], C.c_int),
@@ -233,6 +235,14 @@ class Netmax:
         cols = np.ascontiguousarray(cols, dtype=np.int64)
         out = np.empty((self.M, cols.shape[0]), dtype=np.float32)
         _check(lib().netmax_read_columns(self._h, _p(cols), cols.shape[0], _p(out)), self._h)
+        return out
+
+    def read_columns_static(self, cols):
+        """netmax_read_columns_static: the same read-back through the library's fixed staging
+        array, for callers that must not allocate device memory (limits in the C header)."""
+        cols = np.ascontiguousarray(cols, dtype=np.int64)
+        out = np.empty((self.M, cols.shape[0]), dtype=np.float32)
+        _check(lib().netmax_read_columns_static(self._h, _p(cols), cols.shape[0], _p(out)), self._h)
         return out
 
     def peer_trace(self, first_round: int = 0, n: Optional[int] = None):

@@ -9,6 +9,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -633,6 +634,63 @@ int netmax_read_columns(netmax_ctx* ctx, const int64_t* host_cols, int64_t n_col
   cudaFree(d_cols);
   cudaFree(d_out);
   return rc;
+}
+
+// ---- sampled read-back that allocates nothing -------------------------------------------
+// Staging area of netmax_read_columns_static: the column list, then the gathered values.
+// It is part of the library image, so every device that loads the library holds it.
+struct StaticGatherScratch {
+  int64_t cols[NETMAX_STATIC_MAX_COLS];
+  float values[NETMAX_STATIC_MAX_VALUES];
+};
+static __device__ __align__(256) unsigned char g_gather_scratch[sizeof(StaticGatherScratch)];
+
+// In host code g_gather_scratch is only a stand-in for the symbol; the address a kernel or a
+// copy can use comes from cudaGetSymbolAddress, looked up once per device (that device
+// current) and cached here.
+static std::mutex g_gather_mu;
+static StaticGatherScratch* g_gather_ptr[64] = {};
+
+static int gather_scratch_address(netmax_ctx* ctx, StaticGatherScratch** out) {
+  std::lock_guard<std::mutex> lock(g_gather_mu);
+  const bool cached = ctx->device >= 0 && ctx->device < 64;
+  if (cached && g_gather_ptr[ctx->device]) {
+    *out = g_gather_ptr[ctx->device];
+    return NETMAX_OK;
+  }
+  void* ptr = nullptr;
+  NM_CUDA(ctx, cudaGetSymbolAddress(&ptr, g_gather_scratch));
+  if (!ptr) return fail(ctx, NETMAX_CUDA_ERROR, "cudaGetSymbolAddress returned a null address");
+  if (cached) g_gather_ptr[ctx->device] = (StaticGatherScratch*)ptr;
+  *out = (StaticGatherScratch*)ptr;
+  return NETMAX_OK;
+}
+
+int netmax_read_columns_static(netmax_ctx* ctx, const int64_t* host_cols, int64_t n_cols, float* host_out) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (n_cols < 0 || (n_cols > 0 && (!host_cols || !host_out))) return fail(ctx, NETMAX_INVALID_ARG, "bad column list");
+  if (n_cols > NETMAX_STATIC_MAX_COLS)
+    return fail(ctx, NETMAX_INVALID_ARG, "read_columns_static: n_cols = %lld exceeds the fixed staging area (%d columns); split the list",
+                (long long)n_cols, NETMAX_STATIC_MAX_COLS);
+  if (n_cols * (int64_t)ctx->M > NETMAX_STATIC_MAX_VALUES)
+    return fail(ctx, NETMAX_INVALID_ARG, "read_columns_static: M * n_cols = %lld exceeds the fixed staging area (%d values); split the list",
+                (long long)(n_cols * (int64_t)ctx->M), NETMAX_STATIC_MAX_VALUES);
+  if (n_cols == 0) return NETMAX_OK;
+  for (int64_t k = 0; k < n_cols; ++k)
+    if (host_cols[k] < 0 || host_cols[k] >= ctx->d) return fail(ctx, NETMAX_INVALID_ARG, "cols[%lld] = %lld outside [0, d)", (long long)k, (long long)host_cols[k]);
+  DeviceGuard guard(ctx->device);
+  StaticGatherScratch* scratch = nullptr;
+  int rc = gather_scratch_address(ctx, &scratch);
+  if (rc) return rc;
+  const int64_t total = n_cols * ctx->M;
+  const int grid = (int)std::min<int64_t>((total + kThreads - 1) / kThreads, 4096);
+  NM_CUDA(ctx, cudaMemcpyAsync(scratch->cols, host_cols, (size_t)n_cols * sizeof(int64_t), cudaMemcpyHostToDevice, ctx->stream));
+  gather_columns_kernel<<<grid, kThreads, 0, ctx->stream>>>(ctx->x[ctx->cur], ctx->L.ld, ctx->M, scratch->cols, n_cols, scratch->values);
+  ctx->launches += 1;
+  NM_CUDA(ctx, cudaGetLastError());
+  NM_CUDA(ctx, cudaMemcpyAsync(host_out, scratch->values, (size_t)total * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+  NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  return NETMAX_OK;
 }
 
 static int ring_range(netmax_ctx* ctx, int64_t first, int64_t n) {
