@@ -347,12 +347,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="cfg2", help="cfg1..cfg5 (default: the ResNet18-sized cfg2)")
+    ap.add_argument("--d", type=int, default=0, help="override the workload's vector length (profiling on a smaller case)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     w = workloads.config(int(args.workload.replace("cfg", "")))
+    if args.d > 0:
+        w = w.scaled(d=args.d)
     if args.impl == "reference":
         run_reference(args, w)
     else:

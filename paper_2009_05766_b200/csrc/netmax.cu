@@ -307,7 +307,7 @@ struct RoundPlan {
 using RoundKernel = void (*)(const RoundParams);
 
 RoundKernel pick_kernel(int objective) {
-  return objective == 1 ? round_kernel<1, true, 4> : round_kernel<0, true, 4>;
+  return objective == 1 ? round_kernel<1, true, NETMAX_ROUND_UNROLL> : round_kernel<0, true, NETMAX_ROUND_UNROLL>;
 }
 
 // Tile shape: all M rows x cg column groups.  cg is the largest power of two (<= 256

@@ -99,8 +99,17 @@ __device__ __forceinline__ float4 update_group(const RoundParams& p, uint32_t q,
 // tile and the rows rli, rli + rl, ...; tiles are taken round-robin by the resident CTAs.
 // Dynamic shared memory: int32 peer[M], float w[M], then (rl > 1) 2 * blockDim float4 of
 // column-sum scratch, then 2 * 32 doubles for the block reduction.
+// Tuning constants of round_kernel: rows whose loads are in flight together per thread, and
+// the CTAs per SM the register allocation must leave room for.
+#ifndef NETMAX_ROUND_UNROLL
+#define NETMAX_ROUND_UNROLL 1
+#endif
+#ifndef NETMAX_ROUND_MIN_CTAS
+#define NETMAX_ROUND_MIN_CTAS 4
+#endif
+
 template <int kObjective, bool kFastNoise, int kUnroll>
-__global__ void __launch_bounds__(256) round_kernel(const RoundParams p) {
+__global__ void __launch_bounds__(256, NETMAX_ROUND_MIN_CTAS) round_kernel(const RoundParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   int32_t* s_peer = reinterpret_cast<int32_t*>(smem_raw);
   float* s_w = reinterpret_cast<float*>(s_peer + p.M);
