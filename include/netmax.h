@@ -54,9 +54,9 @@ typedef struct netmax_ctx netmax_ctx; /* opaque; created and destroyed by the li
  */
 typedef struct netmax_config {
   int32_t M;                     /* workers, 2 <= M <= 16384                                          */
-  int64_t d;                     /* parameters per replica, 1 <= d < 2^33                              */
+  int64_t d;                     /* parameters per replica, 1 <= d < 2^30 - 32                        */
   int64_t element_offset;        /* logical index of this context's first element inside a longer global
-                                    vector (a multiple of 4, offset + d < 2^33; default 0).  Only the
+                                    vector (a multiple of 4, offset + d < 2^30 - 32; default 0).  Only the
                                     noise / initialisation counters use it: contexts that hold disjoint
                                     column ranges of one problem (one per GPU) then draw the streams the
                                     single-context run would, and never need to exchange data            */

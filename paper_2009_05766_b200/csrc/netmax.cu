@@ -27,7 +27,7 @@ thread_local std::string g_error;  // failures of calls that have no context
 
 constexpr int kThreads = 256;
 constexpr int64_t kMaxM = 16384;
-constexpr int64_t kMaxD = (int64_t)1 << 33;
+constexpr int64_t kMaxD = ((int64_t)1 << 30) - 32;  // a padded row stays below 2^32 bytes
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -307,17 +307,18 @@ struct RoundPlan {
 using RoundKernel = void (*)(const RoundParams);
 
 RoundKernel pick_kernel(int objective) {
-  return objective == 1 ? round_kernel<1, true, NETMAX_ROUND_UNROLL> : round_kernel<0, true, NETMAX_ROUND_UNROLL>;
+  return objective == 1 ? round_kernel<1, true> : round_kernel<0, true>;
 }
 
 // Tile shape: all M rows x cg column groups.  cg is the largest power of two (<= 256
-// threads' worth) that keeps the tile's share of x near 48 KB, so that a row fetched for
-// its own update is still close by in cache when another row pulls it as a peer; it is
-// reduced further while that leaves SMs without a tile.
+// threads' worth, i.e. 4 KB of a row) that keeps the tile's share of x within 96 KB, so that
+// a row fetched for its own update is still in cache when another row pulls it as a peer
+// (measured optimum on cfg 2-4: wider tiles stream better until the peer reads start to
+// miss); it is reduced further while that leaves SMs without a tile.
 int plan_round(netmax_ctx* ctx, RoundPlan& plan) {
   const int64_t M = ctx->M, nq = ctx->L.nq;
   int cg = kThreads;
-  while (cg > 2 && (int64_t)cg * 16 * M > 48 * 1024) cg >>= 1;
+  while (cg > 2 && (int64_t)cg * 16 * M > 96 * 1024) cg >>= 1;
   while (cg > 2 && (nq + cg - 1) / cg < 2 * (int64_t)ctx->sm_count) cg >>= 1;
   plan.cg = cg;
   plan.rl = kThreads / cg;
@@ -350,9 +351,9 @@ int netmax_config_init(netmax_config* cfg) {
 static int check_sizes(const netmax_config* cfg) {
   if (!cfg) return fail(nullptr, NETMAX_INVALID_ARG, "cfg is NULL");
   if (cfg->M < 2 || cfg->M > kMaxM) return fail(nullptr, NETMAX_INVALID_ARG, "M = %d outside [2, %lld]", cfg->M, (long long)kMaxM);
-  if (cfg->d < 1 || cfg->d >= kMaxD) return fail(nullptr, NETMAX_INVALID_ARG, "d = %lld outside [1, 2^33)", (long long)cfg->d);
+  if (cfg->d < 1 || cfg->d >= kMaxD) return fail(nullptr, NETMAX_INVALID_ARG, "d = %lld outside [1, 2^30 - 32)", (long long)cfg->d);
   if (cfg->element_offset < 0 || cfg->element_offset % 4 != 0 || cfg->element_offset + cfg->d >= kMaxD)
-    return fail(nullptr, NETMAX_INVALID_ARG, "element_offset = %lld must be a non-negative multiple of 4 with offset + d < 2^33", (long long)cfg->element_offset);
+    return fail(nullptr, NETMAX_INVALID_ARG, "element_offset = %lld must be a non-negative multiple of 4 with offset + d < 2^30 - 32", (long long)cfg->element_offset);
   if (cfg->trace_rounds < 1) return fail(nullptr, NETMAX_INVALID_ARG, "trace_rounds = %lld < 1", (long long)cfg->trace_rounds);
   return NETMAX_OK;
 }
@@ -566,6 +567,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   p.partials = ctx->partials;
   p.ticket = ctx->ticket;
   p.ldq = ctx->L.ldq;
+  p.row_bytes = (uint32_t)(ctx->L.ld * sizeof(float));
   p.nq = ctx->L.nq;
   p.n_tiles = plan.n_tiles;
   p.M = ctx->M;

@@ -58,6 +58,7 @@ struct RoundParams {
   unsigned int* ticket;  // last-CTA-done counter (0 between launches)
   double* tel_out;       // [2] this round's (consensus, loss)
   int64_t ldq;           // row stride, in float4
+  uint32_t row_bytes;    // row stride, in bytes (< 2^32)
   int64_t nq;            // column groups per row = ceil(d / 4)
   int64_t n_tiles;       // ceil(nq / cg)
   int32_t M;
@@ -71,138 +72,67 @@ struct RoundParams {
   PhiloxKeys keys;
 };
 
-__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
-__device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
+// Per-thread telemetry accumulators of one column group (4 columns as two fp32 pairs):
+// sum (x - pivot), sum (x - pivot)^2 and sum (x - c)^2 over the rows the thread has seen.
+struct RowAcc {
+  pair_t s1a = 0ull, s1b = 0ull, s2a = 0ull, s2b = 0ull, la = 0ull, lb = 0ull;  // +0.0f pairs
+};
 
+// Eq. 15 and Eq. 16 on one column group of one worker, on packed fp32 pairs:
+//   g = (x - c) + sigma z,  h = x - alpha g                                       (Eq. 15)
+//   x' = h - w (h - x_m),   w = alpha rho gamma_im  (w = 0 on a self-draw)          (Eq. 16)
+// q32 is the global column-group index (first Philox counter word), tail > 0 marks the ragged
+// last group of a row whose padding lanes must stay zero.
 template <int kObjective, bool kFastNoise>
-__device__ __forceinline__ float4 update_group(const RoundParams& p, uint32_t q, uint32_t worker, float4 x, float4 c,
-                                               float4 xm, float w) {
-  float4 h = x;
+__device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t q32, uint32_t worker, ulonglong2 xv,
+                                                 ulonglong2 cv, ulonglong2 xm, ulonglong2 pivot, float w, bool ragged,
+                                                 RowAcc& acc) {
+  const pair_t neg1 = pack2(-1.0f, -1.0f);
+  const pair_t nw2 = pack2(-w, -w);
+  const pair_t ta = fma2(cv.x, neg1, xv.x), tb = fma2(cv.y, neg1, xv.y);  // x - c
+  pair_t ha = xv.x, hb = xv.y;
   if (kObjective == 1) {
-    const float4 z = normals4<kFastNoise>(philox4x32_10(q, worker, p.round_lo, p.ctr3, p.keys));
-    // g = (x - c) + sigma z ;  h = x - alpha g                                    (Eq. 15)
-    h.x = fmaf(-p.alpha, fmaf(p.sigma, z.x, x.x - c.x), x.x);
-    h.y = fmaf(-p.alpha, fmaf(p.sigma, z.y, x.y - c.y), x.y);
-    h.z = fmaf(-p.alpha, fmaf(p.sigma, z.z, x.z - c.z), x.z);
-    h.w = fmaf(-p.alpha, fmaf(p.sigma, z.w, x.w - c.w), x.w);
+    const pair_t sig2 = pack2(p.sigma, p.sigma);
+    const pair_t nalpha2 = pack2(-p.alpha, -p.alpha);
+    const uint4 rnd = philox4x32_10(q32, worker, p.round_lo, p.ctr3, p.keys);
+    pair_t za, zb;
+    if (kFastNoise) {
+      za = normal_pair_fast_packed(rnd.x, rnd.y);
+      zb = normal_pair_fast_packed(rnd.z, rnd.w);
+    } else {
+      const float4 z = normals4<false>(rnd);
+      za = pack2(z.x, z.y);
+      zb = pack2(z.z, z.w);
+    }
+    ha = fma2(nalpha2, fma2(sig2, za, ta), xv.x);
+    hb = fma2(nalpha2, fma2(sig2, zb, tb), xv.y);
   }
-  // x' = h - w (h - x_m)  with w = alpha rho gamma_im; w = 0 on a self-draw          (Eq. 16)
-  float4 o;
-  o.x = fmaf(-w, h.x - xm.x, h.x);
-  o.y = fmaf(-w, h.y - xm.y, h.y);
-  o.z = fmaf(-w, h.z - xm.z, h.z);
-  o.w = fmaf(-w, h.w - xm.w, h.w);
-  return o;
+  pair_t oa = fma2(nw2, fma2(xm.x, neg1, ha), ha);
+  pair_t ob = fma2(nw2, fma2(xm.y, neg1, hb), hb);
+  if (ragged) {  // keep the padding lanes of the last group at zero
+    float o0, o1, o2, o3;
+    unpack2(oa, o0, o1);
+    unpack2(ob, o2, o3);
+    if (p.tail < 2) o1 = 0.f;
+    if (p.tail < 3) o2 = 0.f;
+    oa = pack2(o0, o1);
+    ob = pack2(o2, 0.f);
+  }
+  const pair_t da = fma2(pivot.x, neg1, xv.x), db = fma2(pivot.y, neg1, xv.y);  // x - pivot
+  acc.s1a = add2(acc.s1a, da);
+  acc.s1b = add2(acc.s1b, db);
+  acc.s2a = fma2(da, da, acc.s2a);
+  acc.s2b = fma2(db, db, acc.s2b);
+  acc.la = fma2(ta, ta, acc.la);
+  acc.lb = fma2(tb, tb, acc.lb);
+  return make_ulonglong2(oa, ob);
 }
 
-// One tile = all M rows x cg column groups.  Thread (cgi, rli) owns column group cgi of the
-// tile and the rows rli, rli + rl, ...; tiles are taken round-robin by the resident CTAs.
-// Dynamic shared memory: int32 peer[M], float w[M], then (rl > 1) 2 * blockDim float4 of
-// column-sum scratch, then 2 * 32 doubles for the block reduction.
-// Tuning constants of round_kernel: rows whose loads are in flight together per thread, and
-// the CTAs per SM the register allocation must leave room for.
-#ifndef NETMAX_ROUND_UNROLL
-#define NETMAX_ROUND_UNROLL 1
-#endif
-#ifndef NETMAX_ROUND_MIN_CTAS
-#define NETMAX_ROUND_MIN_CTAS 4
-#endif
-
-template <int kObjective, bool kFastNoise, int kUnroll>
-__global__ void __launch_bounds__(256, NETMAX_ROUND_MIN_CTAS) round_kernel(const RoundParams p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  int32_t* s_peer = reinterpret_cast<int32_t*>(smem_raw);
-  float* s_w = reinterpret_cast<float*>(s_peer + p.M);
-  const size_t head = (((size_t)p.M * 8) + 15) & ~(size_t)15;
-  float4* s_col = reinterpret_cast<float4*>(smem_raw + head);
-  double* s_red = reinterpret_cast<double*>(smem_raw + head + (p.rl > 1 ? (size_t)blockDim.x * 32 : 0));
-
+// Block reduction of a CTA's two telemetry sums; the last CTA of the grid to arrive then adds
+// all CTA partials in index order (deterministic) and publishes the round's telemetry.
+// s_red: 64 doubles of shared memory.  Every thread of the CTA must call this.
+__device__ __forceinline__ void finalize_telemetry(const RoundParams& p, double acc_cons, double acc_loss, double* s_red) {
   const int tid = threadIdx.x;
-  for (int i = tid; i < p.M; i += blockDim.x) {
-    const int32_t m = __ldg(p.peers + i);
-    s_peer[i] = m;
-    s_w[i] = (m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * p.M + m);
-  }
-  __syncthreads();
-
-  const int cgi = tid & (p.cg - 1);
-  const int rli = tid / p.cg;
-  const int M = p.M;
-  const int step = p.rl;
-  double acc_cons = 0.0, acc_loss = 0.0;
-
-  for (int64_t tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x) {
-    const int64_t q = tile * p.cg + cgi;
-    const bool live = q < p.nq;
-    const bool ragged = (p.tail != 0) && (q == p.nq - 1);
-    float4 s1 = make_float4(0.f, 0.f, 0.f, 0.f), s2 = s1;
-    float loss = 0.f;
-    if (live) {
-      const float4 pivot = __ldg(p.x_cur + q);  // row 0: pivot of the one-pass variance
-      for (int i0 = rli; i0 < M; i0 += step * kUnroll) {
-        float4 xv[kUnroll], cv[kUnroll], xm[kUnroll];
-        float wv[kUnroll];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-          const int i = i0 + u * step;
-          if (i < M) {
-            const int m = s_peer[i];
-            wv[u] = s_w[i];
-            xv[u] = __ldg(p.x_cur + (size_t)i * p.ldq + q);
-            xm[u] = __ldg(p.x_cur + (size_t)m * p.ldq + q);
-            cv[u] = ld_stream(p.c + (size_t)i * p.ldq + q);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-          const int i = i0 + u * step;
-          if (i < M) {
-            float4 o = update_group<kObjective, kFastNoise>(p, (uint32_t)q + p.q_offset, (uint32_t)i, xv[u], cv[u], xm[u], wv[u]);
-            if (ragged) {  // keep the padding lanes of the last group at zero
-              if (p.tail < 2) o.y = 0.f;
-              if (p.tail < 3) o.z = 0.f;
-              o.w = 0.f;
-            }
-            st_stream(p.x_nxt + (size_t)i * p.ldq + q, o);
-            const float dx = xv[u].x - pivot.x, dy = xv[u].y - pivot.y, dz = xv[u].z - pivot.z, dw = xv[u].w - pivot.w;
-            s1.x += dx; s1.y += dy; s1.z += dz; s1.w += dw;
-            s2.x = fmaf(dx, dx, s2.x); s2.y = fmaf(dy, dy, s2.y); s2.z = fmaf(dz, dz, s2.z); s2.w = fmaf(dw, dw, s2.w);
-            const float ex = xv[u].x - cv[u].x, ey = xv[u].y - cv[u].y, ez = xv[u].z - cv[u].z, ew = xv[u].w - cv[u].w;
-            loss = fmaf(ex, ex, fmaf(ey, ey, fmaf(ez, ez, fmaf(ew, ew, loss))));
-          }
-        }
-      }
-    }
-    if (p.rl > 1) {  // sum the column statistics over the row lanes (stride cg in tid)
-      s_col[tid] = s1;
-      s_col[blockDim.x + tid] = s2;
-      __syncthreads();
-      for (int s = blockDim.x >> 1; s >= p.cg; s >>= 1) {
-        if (tid < s) {
-          float4 a = s_col[tid], b = s_col[tid + s];
-          a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-          s_col[tid] = a;
-          a = s_col[blockDim.x + tid]; b = s_col[blockDim.x + tid + s];
-          a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-          s_col[blockDim.x + tid] = a;
-        }
-        __syncthreads();
-      }
-      s1 = s_col[cgi];
-      s2 = s_col[blockDim.x + cgi];
-      __syncthreads();
-    }
-    if (rli == 0) {
-      // sum_i (x_i - xbar)^2 = sum_i (x_i - a)^2 - (sum_i (x_i - a))^2 / M   per column
-      const float cons = (s2.x - s1.x * s1.x * p.inv_M) + (s2.y - s1.y * s1.y * p.inv_M) +
-                         (s2.z - s1.z * s1.z * p.inv_M) + (s2.w - s1.w * s1.w * p.inv_M);
-      acc_cons += (double)cons;
-    }
-    acc_loss += (double)loss;
-  }
-
-  // block reduction of the two doubles, then the last CTA to finish sums all partials in
-  // index order (deterministic) and publishes the round's telemetry.
   acc_loss *= 0.5;
   for (int off = 16; off > 0; off >>= 1) {
     acc_cons += __shfl_down_sync(0xffffffffu, acc_cons, off);
@@ -257,6 +187,101 @@ __global__ void __launch_bounds__(256, NETMAX_ROUND_MIN_CTAS) round_kernel(const
       *p.ticket = 0u;
     }
   }
+}
+
+// Direct-load round kernel (any M).  One tile = all M rows x cg column groups.  Thread
+// (cgi, rli) owns column group cgi of the tile and the rows rli, rli + rl, ...; tiles are
+// taken round-robin by the resident CTAs.  All accesses are plain cacheable 128-bit loads and
+// stores: the peer read (a row this tile reads anyway) then hits L1/L2, and streaming hints on
+// c and on the output measured slower.
+// Dynamic shared memory: (peer, weight) int2[M], then (rl > 1) 2 * blockDim float4 of
+// column-sum scratch, then 64 doubles for the block reduction.
+#ifndef NETMAX_ROUND_MIN_CTAS
+#define NETMAX_ROUND_MIN_CTAS 4  // CTAs per SM the register allocation leaves room for
+#endif
+
+template <int kObjective, bool kFastNoise>
+__global__ void __launch_bounds__(256, NETMAX_ROUND_MIN_CTAS) round_kernel(const RoundParams p) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  int2* s_pw = reinterpret_cast<int2*>(smem_raw);  // (peer, bits of the pull weight) per worker
+  const size_t head = (((size_t)p.M * 8) + 15) & ~(size_t)15;
+  float4* s_col = reinterpret_cast<float4*>(smem_raw + head);
+  double* s_red = reinterpret_cast<double*>(smem_raw + head + (p.rl > 1 ? (size_t)blockDim.x * 32 : 0));
+
+  const int tid = threadIdx.x;
+  for (int i = tid; i < p.M; i += blockDim.x) {
+    const int32_t m = __ldg(p.peers + i);
+    s_pw[i] = make_int2(m, __float_as_int((m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * p.M + m)));
+  }
+  __syncthreads();
+
+  const int cgi = tid & (p.cg - 1);
+  const int rli = tid / p.cg;
+  const int M = p.M;
+  const int step = p.rl;
+  double acc_cons = 0.0, acc_loss = 0.0;
+
+  for (int64_t tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x) {
+    const int64_t q = tile * p.cg + cgi;
+    const bool live = q < p.nq;
+    const bool ragged = (p.tail != 0) && (q == p.nq - 1);
+    float4 s1 = make_float4(0.f, 0.f, 0.f, 0.f), s2 = s1;
+    float loss = 0.f;
+    if (live) {
+      // byte pointers to this thread's column group in row 0; row i is i * row_bytes further
+      const char* xq = reinterpret_cast<const char*>(p.x_cur + q);
+      const char* cq = reinterpret_cast<const char*>(p.c + q);
+      char* oq = reinterpret_cast<char*>(p.x_nxt + q);
+      const uint32_t q32 = (uint32_t)q + p.q_offset;
+      const ulonglong2 pivot = __ldg(reinterpret_cast<const ulonglong2*>(xq));  // row 0: pivot of the one-pass variance
+      RowAcc acc;
+      for (int i = rli; i < M; i += step) {
+        const int2 pw = s_pw[i];
+        const uint64_t row = (uint64_t)(uint32_t)i * p.row_bytes;
+        const ulonglong2 xv = __ldg(reinterpret_cast<const ulonglong2*>(xq + row));
+        const ulonglong2 xm = __ldg(reinterpret_cast<const ulonglong2*>(xq + (uint64_t)(uint32_t)pw.x * p.row_bytes));
+        const ulonglong2 cv = __ldg(reinterpret_cast<const ulonglong2*>(cq + row));
+        const ulonglong2 o = row_update<kObjective, kFastNoise>(p, q32, (uint32_t)i, xv, cv, xm, pivot,
+                                                                __int_as_float(pw.y), ragged, acc);
+        *reinterpret_cast<ulonglong2*>(oq + row) = o;
+      }
+      unpack2(acc.s1a, s1.x, s1.y);
+      unpack2(acc.s1b, s1.z, s1.w);
+      unpack2(acc.s2a, s2.x, s2.y);
+      unpack2(acc.s2b, s2.z, s2.w);
+      float l0, l1, l2, l3;
+      unpack2(acc.la, l0, l1);
+      unpack2(acc.lb, l2, l3);
+      loss = (l0 + l1) + (l2 + l3);
+    }
+    if (p.rl > 1) {  // sum the column statistics over the row lanes (stride cg in tid)
+      s_col[tid] = s1;
+      s_col[blockDim.x + tid] = s2;
+      __syncthreads();
+      for (int s = blockDim.x >> 1; s >= p.cg; s >>= 1) {
+        if (tid < s) {
+          float4 a = s_col[tid], b = s_col[tid + s];
+          a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+          s_col[tid] = a;
+          a = s_col[blockDim.x + tid]; b = s_col[blockDim.x + tid + s];
+          a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+          s_col[blockDim.x + tid] = a;
+        }
+        __syncthreads();
+      }
+      s1 = s_col[cgi];
+      s2 = s_col[blockDim.x + cgi];
+      __syncthreads();
+    }
+    if (rli == 0) {
+      // sum_i (x_i - xbar)^2 = sum_i (x_i - a)^2 - (sum_i (x_i - a))^2 / M   per column
+      const float cons = (s2.x - s1.x * s1.x * p.inv_M) + (s2.y - s1.y * s1.y * p.inv_M) +
+                         (s2.z - s1.z * s1.z * p.inv_M) + (s2.w - s1.w * s1.w * p.inv_M);
+      acc_cons += (double)cons;
+    }
+    acc_loss += (double)loss;
+  }
+  finalize_telemetry(p, acc_cons, acc_loss, s_red);
 }
 
 // ------------------------------------------------------------------------- init / IO

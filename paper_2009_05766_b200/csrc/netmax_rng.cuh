@@ -46,14 +46,14 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
                                                const PhiloxKeys& keys) {
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(kPhiloxMul0, c0), lo0 = kPhiloxMul0 * c0;
-    const uint32_t hi1 = __umulhi(kPhiloxMul1, c2), lo1 = kPhiloxMul1 * c2;
-    const uint32_t n0 = hi1 ^ c1 ^ keys.k0[r];
-    const uint32_t n2 = hi0 ^ c3 ^ keys.k1[r];
+    const uint64_t p0 = (uint64_t)kPhiloxMul0 * c0;  // one 32x32->64 multiply each
+    const uint64_t p1 = (uint64_t)kPhiloxMul1 * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ keys.k0[r];
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ keys.k1[r];
     c0 = n0;
-    c1 = lo1;
+    c1 = (uint32_t)p1;
     c2 = n2;
-    c3 = lo0;
+    c3 = (uint32_t)p0;
   }
   return make_uint4(c0, c1, c2, c3);
 }
@@ -89,6 +89,45 @@ __device__ __forceinline__ void normal_pair_accurate(uint32_t a, uint32_t b, flo
   sincospif(turns2, &s, &c);
   z0 = rad * c;
   z1 = rad * s;
+}
+
+// ---- packed fp32x2 arithmetic (sm_100: two IEEE fp32 operations per instruction) ----------
+typedef unsigned long long pair_t;  // two floats in one 64-bit register: (low lane, high lane)
+
+__device__ __forceinline__ pair_t pack2(float lo, float hi) {
+  pair_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(pair_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ pair_t fma2(pair_t a, pair_t b, pair_t c) {
+  pair_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ pair_t mul2(pair_t a, pair_t b) {
+  pair_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ pair_t add2(pair_t a, pair_t b) {
+  pair_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// The two normals of one Box-Muller pair, packed (fast path; same arithmetic as normal_pair_fast).
+__device__ __forceinline__ pair_t normal_pair_fast_packed(uint32_t a, uint32_t b) {
+  const float u1 = radius_uniform(a);
+  const float ang = (float)((int32_t)b >> 8) * 3.74507028e-07f;
+  const float r2 = fmaxf(-1.38629436111989f * __log2f(u1), 0.0f);
+  float rad;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(r2));
+  float s, c;
+  __sincosf(ang, &s, &c);
+  return mul2(pack2(rad, rad), pack2(c, s));
 }
 
 template <bool kFast>

@@ -294,3 +294,4 @@ def test_many_workers_small_vectors(nm):
     np.testing.assert_allclose(gc, oc, rtol=1e-4)
     np.testing.assert_allclose(gl, ol, rtol=1e-4)
     g.close()
+
