@@ -295,3 +295,34 @@ def test_many_workers_small_vectors(nm):
     np.testing.assert_allclose(gl, ol, rtol=1e-4)
     g.close()
 
+
+def test_column_shards_match_the_unsharded_problem(nm):
+    """Two contexts holding disjoint column ranges (element_offset) of one problem reproduce the
+    oracle's run of the whole problem: same peers, same noise streams, no exchange."""
+    M, d, rounds = 5, 3001, 15
+    d4 = (d + 3) // 4 * 4
+    rng = np.random.default_rng(23)
+    P = random_policy(M, rng)
+    parts = []
+    for rank in range(2):
+        g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, seed=41,
+                      element_offset=rank * d4)
+        g.round(rounds)
+        parts.append(g)
+    rho = parts[0].get_policy()[1]
+    cols = np.concatenate([rank * d4 + np.arange(d, dtype=np.int64) for rank in range(2)])
+    o = oracle.Sim(M, 2 * d4, P, full_adj(M), alpha=0.05, rho=rho, sigma=0.1, objective=1, seed=41, cols=cols)
+    o.init(1.0, 1.0)
+    o.round(rounds)
+    got = np.concatenate([g.read_replicas() for g in parts], axis=1)
+    assert_replicas_close(got, o.x())
+    assert (parts[0].peer_trace() == o.trace()).all() and (parts[1].peer_trace() == o.trace()).all()
+    oc, ol = o.telemetry()
+    gc = parts[0].telemetry()[0] + parts[1].telemetry()[0]
+    gl = parts[0].telemetry()[1] + parts[1].telemetry()[1]
+    np.testing.assert_allclose(gc, oc, rtol=1e-4)
+    np.testing.assert_allclose(gl, ol, rtol=1e-4)
+    with pytest.raises(nm.NetmaxError):
+        nm.Netmax(M=M, d=d, lr=0.05, prob=P, element_offset=2)
+    for g in parts:
+        g.close()
