@@ -304,6 +304,21 @@ def run_ours(args, w):
         e2e_ms = float(tmax.item())
     e2e_value = BYTES_PER_ELEMENT * elements * world * e2e_steps / (e2e_ms / 1e3) / 1e9
 
+    # the sampler alone: one batched launch of 1024 rounds x M draws (Algorithm 2's peer selection)
+    batch = 1024
+    draws = torch.empty((batch, w.M), dtype=torch.int32, device="cuda")
+    for _ in range(3):
+        g.sample_peers(0, batch, draws.data_ptr())
+    barrier()
+    with torch.cuda.stream(stream):
+        start.record()
+    for rep in range(10):
+        g.sample_peers(rep * batch, batch, draws.data_ptr())
+    with torch.cuda.stream(stream):
+        stop.record()
+    stop.synchronize()
+    sampler_draws_per_s = 10 * batch * w.M / (start.elapsed_time(stop) / 1e3)
+
     cons, loss = g.telemetry(g.rounds_done - 1, 1)
     peak, peak_kind = measured_peak()
     per_launch_ms = ms / args.steps
@@ -317,7 +332,8 @@ def run_ours(args, w):
                    "sigma": w.sigma, "policy": f"Algorithm 3, K={w.K}, R={w.R}, rho={rho:.6g}",
                    "sharding": "columns, no exchange" if world > 1 else "none",
                    "l2": "inputs larger than L2: each of x, x', c is %.0f MB" % (elements * 4 / 1e6)},
-        "rounds_per_s": args.steps / sec, "peer_draws_per_s": w.M * args.steps / sec,
+        "rounds_per_s": args.steps / sec, "peer_draws_per_s": w.M * world * args.steps / sec,
+        "sampler_only_draws_per_s": sampler_draws_per_s,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "round_kernel",
                      "bytes_per_launch": BYTES_PER_ELEMENT * elements,

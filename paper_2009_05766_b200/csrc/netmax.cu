@@ -47,10 +47,11 @@ struct DeviceGuard {
 struct Layout {
   int64_t ld = 0, ldq = 0, nq = 0;
   size_t off_x0 = 0, off_x1 = 0, off_c = 0, off_thr = 0, off_last = 0, off_w = 0, off_trace = 0, off_tel = 0,
-         off_partials = 0, off_ticket = 0, total = 0;
+         off_partials = 0, off_ticket = 0, off_colpart = 0, off_coltick = 0, total = 0;
 };
 
 constexpr int kMaxGrid = 148 * 16;  // upper bound on resident CTAs of the round kernel
+constexpr size_t kColPartBytes = (size_t)8 << 20;  // column partials of the row-split (short vector) shape
 
 Layout make_layout(int64_t M, int64_t d, int64_t trace_rounds) {
   Layout L;
@@ -70,6 +71,8 @@ Layout make_layout(int64_t M, int64_t d, int64_t trace_rounds) {
   L.off_tel = take((size_t)trace_rounds * 2 * sizeof(double));
   L.off_partials = take((size_t)kMaxGrid * 2 * sizeof(double));
   L.off_ticket = take(256);
+  L.off_colpart = take(kColPartBytes);
+  L.off_coltick = take((size_t)kMaxGrid * sizeof(unsigned int));
   L.total = o;
   return L;
 }
@@ -97,6 +100,8 @@ struct netmax_ctx {
   double* tel = nullptr;
   double* partials = nullptr;
   unsigned int* ticket = nullptr;
+  float4* colpart = nullptr;
+  unsigned int* coltick = nullptr;
   int cur = 0;  // index of the buffer holding the current replicas
   int64_t rounds = 0;
   int64_t trace_rounds = 0;
@@ -298,7 +303,8 @@ int launch_sampler(netmax_ctx* ctx, uint64_t first_round, int64_t n_rounds, int3
 }
 
 struct RoundPlan {
-  int cg = kThreads, rl = 1;
+  int cg = kThreads, rl = 1, rg = 1, rows_per_group = 0;
+  bool short_vectors = false;  // fewer than two streaming tiles per SM: the L2-resident shape
   int grid = 1;
   size_t smem = 0;
   int64_t n_tiles = 0;
@@ -306,25 +312,56 @@ struct RoundPlan {
 
 using RoundKernel = void (*)(const RoundParams);
 
-RoundKernel pick_kernel(int objective) {
-  return objective == 1 ? round_kernel<1, true> : round_kernel<0, true>;
+RoundKernel pick_kernel(int objective, bool short_vectors) {
+  if (short_vectors) return objective == 1 ? round_kernel<1, true, 4> : round_kernel<0, true, 4>;
+  return objective == 1 ? round_kernel<1, true, 1> : round_kernel<0, true, 1>;
 }
 
-// Tile shape: all M rows x cg column groups.  cg is the largest power of two (<= 256
-// threads' worth, i.e. 4 KB of a row) that keeps the tile's share of x within 96 KB, so that
-// a row fetched for its own update is still in cache when another row pulls it as a peer
-// (measured optimum on cfg 2-4: wider tiles stream better until the peer reads start to
-// miss); it is reduced further while that leaves SMs without a tile.
+int floor_pow2(int64_t v) {
+  int r = 1;
+  while ((int64_t)r * 2 <= v) r *= 2;
+  return r;
+}
+
+// Tile shape.  Long vectors: all M rows x cg column groups, cg the largest power of two
+// (<= 256 threads' worth, i.e. 4 KB of a row) that keeps the tile's share of x within 96 KB, so
+// that a row fetched for its own update is still in cache when another row pulls it as a peer
+// (measured optimum on cfg 2-4: wider tiles stream better until the peer reads start to miss).
+// Short vectors (fewer than two such tiles per SM; everything is L2-resident then): 128-byte
+// column segments where M allows, no idle row lanes, and the rows split into rg groups so that
+// about two CTAs per SM have work.
 int plan_round(netmax_ctx* ctx, RoundPlan& plan) {
   const int64_t M = ctx->M, nq = ctx->L.nq;
+  const int64_t target = 2 * (int64_t)ctx->sm_count;  // the short-vector kernel runs 2 CTAs per SM
   int cg = kThreads;
-  while (cg > 2 && (int64_t)cg * 16 * M > 96 * 1024) cg >>= 1;
-  while (cg > 2 && (nq + cg - 1) / cg < 2 * (int64_t)ctx->sm_count) cg >>= 1;
+  while (cg > 1 && (int64_t)cg * 16 * M > 96 * 1024) cg >>= 1;
+  int rg = 1;
+  if ((nq + cg - 1) / cg < 2 * (int64_t)ctx->sm_count || kThreads / cg > M) {
+    plan.short_vectors = true;
+    static const int order[] = {8, 4, 2, 16, 32, 64, 128, 256, 1};
+    int64_t best_score = -1;
+    for (int cand : order) {
+      const int rl = kThreads / cand;
+      if (rl > M && cand != kThreads) continue;  // row lanes without rows
+      const int64_t nct = (nq + cand - 1) / cand;
+      int g = (int)std::min<int64_t>(std::min<int64_t>(32, std::max<int64_t>(1, M / rl)), floor_pow2(std::max<int64_t>(1, target / nct)));
+      while (g > 1 && (size_t)nct * g * cand * 32 > kColPartBytes) g >>= 1;
+      if (nct * g > kMaxGrid) continue;
+      const int64_t score = std::min<int64_t>(nct * g, target);
+      if (score > best_score) {
+        best_score = score;
+        cg = cand;
+        rg = g;
+      }
+    }
+  }
   plan.cg = cg;
   plan.rl = kThreads / cg;
-  plan.n_tiles = (nq + cg - 1) / cg;
+  plan.rg = rg;
+  plan.rows_per_group = (int)((M + rg - 1) / rg);
+  plan.n_tiles = (nq + cg - 1) / cg * rg;
   plan.smem = align_up((size_t)M * 8, 16) + (plan.rl > 1 ? (size_t)kThreads * 32 : 0) + 64 * sizeof(double);
-  RoundKernel k = pick_kernel(ctx->objective);
+  RoundKernel k = pick_kernel(ctx->objective, plan.short_vectors);
   if (plan.smem > 48 * 1024)
     NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
   int per_sm = 0;
@@ -450,6 +487,8 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   ctx->tel = (double*)(ctx->base + L.off_tel);
   ctx->partials = (double*)(ctx->base + L.off_partials);
   ctx->ticket = (unsigned int*)(ctx->base + L.off_ticket);
+  ctx->colpart = (float4*)(ctx->base + L.off_colpart);
+  ctx->coltick = (unsigned int*)(ctx->base + L.off_coltick);
 
   auto step = [&](cudaError_t e, const char* what) {
     if (e == cudaSuccess) return true;
@@ -457,6 +496,7 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
     return false;
   };
   if (!step(cudaMemsetAsync(ctx->ticket, 0, 256, ctx->stream), "cudaMemsetAsync(ticket)")) return bail(NETMAX_CUDA_ERROR);
+  if (!step(cudaMemsetAsync(ctx->coltick, 0, (size_t)kMaxGrid * sizeof(unsigned int), ctx->stream), "cudaMemsetAsync(coltick)")) return bail(NETMAX_CUDA_ERROR);
   if (!step(cudaMemsetAsync(ctx->x[1], 0, (size_t)ctx->M * L.ld * sizeof(float), ctx->stream), "cudaMemsetAsync(x)")) return bail(NETMAX_CUDA_ERROR);
   if (!step(cudaMemsetAsync(ctx->tel, 0, (size_t)ctx->trace_rounds * 2 * sizeof(double), ctx->stream), "cudaMemsetAsync(tel)")) return bail(NETMAX_CUDA_ERROR);
   rc = upload_policy(ctx);
@@ -559,7 +599,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   RoundPlan plan;
   int rc = plan_round(ctx, plan);
   if (rc) return rc;
-  RoundKernel kernel = pick_kernel(ctx->objective);
+  RoundKernel kernel = pick_kernel(ctx->objective, plan.short_vectors);
 
   RoundParams p;
   p.c = reinterpret_cast<const float4*>(ctx->c);
@@ -574,6 +614,10 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   p.tail = (int32_t)(ctx->d % 4);
   p.cg = plan.cg;
   p.rl = plan.rl;
+  p.rg = plan.rg;
+  p.rows_per_group = plan.rows_per_group;
+  p.colpart = ctx->colpart;
+  p.coltick = ctx->coltick;
   p.alpha = (float)ctx->alpha;
   p.sigma = (float)ctx->sigma;
   p.inv_M = 1.0f / (float)ctx->M;

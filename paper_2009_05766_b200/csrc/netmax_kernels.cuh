@@ -65,6 +65,10 @@ struct RoundParams {
   int32_t tail;          // d % 4: live lanes of the last column group (0 = all four)
   int32_t cg;            // column groups per tile   (cg * rl == blockDim.x, both powers of two)
   int32_t rl;            // row lanes per tile
+  int32_t rg;            // row groups: tile t covers column tile t / rg, rows of group t % rg
+  int32_t rows_per_group;  // ceil(M / rg)
+  float4* colpart;       // rg > 1: per tile, per column group: (sum, sum of squares) partials
+  unsigned int* coltick; // rg > 1: arrivals per column tile (0 between launches)
   float alpha, sigma;
   float inv_M;
   uint32_t round_lo, ctr3;
@@ -189,9 +193,10 @@ __device__ __forceinline__ void finalize_telemetry(const RoundParams& p, double 
   }
 }
 
-// Direct-load round kernel (any M).  One tile = all M rows x cg column groups.  Thread
-// (cgi, rli) owns column group cgi of the tile and the rows rli, rli + rl, ...; tiles are
-// taken round-robin by the resident CTAs.  All accesses are plain cacheable 128-bit loads and
+// Direct-load round kernel (any M).  One tile = all M rows (or, for short vectors with many
+// workers, one of rg row groups) x cg column groups.  Thread (cgi, rli) owns column group cgi
+// of the tile and the rows rli, rli + rl, ... of its row group; tiles are taken round-robin by
+// the resident CTAs.  All accesses are plain cacheable 128-bit loads and
 // stores: the peer read (a row this tile reads anyway) then hits L1/L2, and streaming hints on
 // c and on the output measured slower.
 // Dynamic shared memory: (peer, weight) int2[M], then (rl > 1) 2 * blockDim float4 of
@@ -200,8 +205,11 @@ __device__ __forceinline__ void finalize_telemetry(const RoundParams& p, double 
 #define NETMAX_ROUND_MIN_CTAS 4  // CTAs per SM the register allocation leaves room for
 #endif
 
-template <int kObjective, bool kFastNoise>
-__global__ void __launch_bounds__(256, NETMAX_ROUND_MIN_CTAS) round_kernel(const RoundParams p) {
+// kRowsInFlight = 1 (64 registers, 4 CTAs/SM) is the streaming shape for long vectors, where
+// occupancy hides the HBM latency; kRowsInFlight = 4 (2 CTAs/SM) serves short, L2-resident
+// problems, where a thread's chain of dependent row loads is what takes the time.
+template <int kObjective, bool kFastNoise, int kRowsInFlight>
+__global__ void __launch_bounds__(256, kRowsInFlight == 1 ? NETMAX_ROUND_MIN_CTAS : 2) round_kernel(const RoundParams p) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   int2* s_pw = reinterpret_cast<int2*>(smem_raw);  // (peer, bits of the pull weight) per worker
   const size_t head = (((size_t)p.M * 8) + 15) & ~(size_t)15;
@@ -209,11 +217,18 @@ __global__ void __launch_bounds__(256, NETMAX_ROUND_MIN_CTAS) round_kernel(const
   double* s_red = reinterpret_cast<double*>(smem_raw + head + (p.rl > 1 ? (size_t)blockDim.x * 32 : 0));
 
   const int tid = threadIdx.x;
-  for (int i = tid; i < p.M; i += blockDim.x) {
-    const int32_t m = __ldg(p.peers + i);
-    s_pw[i] = make_int2(m, __float_as_int((m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * p.M + m)));
+  const int G = p.rg;
+  auto load_draws = [&](int r0, int r1) {  // this round's (peer, weight) of workers [r0, r1)
+    for (int i = r0 + tid; i < r1; i += blockDim.x) {
+      const int32_t m = __ldg(p.peers + i);
+      s_pw[i] = make_int2(m, __float_as_int((m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * p.M + m)));
+    }
+  };
+  if (G == 1) {
+    load_draws(0, p.M);
+    __syncthreads();
   }
-  __syncthreads();
+  __shared__ bool s_lastcol;
 
   const int cgi = tid & (p.cg - 1);
   const int rli = tid / p.cg;
@@ -222,7 +237,15 @@ __global__ void __launch_bounds__(256, NETMAX_ROUND_MIN_CTAS) round_kernel(const
   double acc_cons = 0.0, acc_loss = 0.0;
 
   for (int64_t tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x) {
-    const int64_t q = tile * p.cg + cgi;
+    const int64_t ct = G == 1 ? tile : tile / G;      // column tile
+    const int grp = G == 1 ? 0 : (int)(tile - ct * G);  // row group
+    const int r0 = grp * p.rows_per_group, r1 = min(M, r0 + p.rows_per_group);
+    if (G > 1) {
+      __syncthreads();  // the previous tile's readers of s_pw are done
+      load_draws(r0, r1);
+      __syncthreads();
+    }
+    const int64_t q = ct * p.cg + cgi;
     const bool live = q < p.nq;
     const bool ragged = (p.tail != 0) && (q == p.nq - 1);
     float4 s1 = make_float4(0.f, 0.f, 0.f, 0.f), s2 = s1;
@@ -235,15 +258,29 @@ __global__ void __launch_bounds__(256, NETMAX_ROUND_MIN_CTAS) round_kernel(const
       const uint32_t q32 = (uint32_t)q + p.q_offset;
       const ulonglong2 pivot = __ldg(reinterpret_cast<const ulonglong2*>(xq));  // row 0: pivot of the one-pass variance
       RowAcc acc;
-      for (int i = rli; i < M; i += step) {
-        const int2 pw = s_pw[i];
-        const uint64_t row = (uint64_t)(uint32_t)i * p.row_bytes;
-        const ulonglong2 xv = __ldg(reinterpret_cast<const ulonglong2*>(xq + row));
-        const ulonglong2 xm = __ldg(reinterpret_cast<const ulonglong2*>(xq + (uint64_t)(uint32_t)pw.x * p.row_bytes));
-        const ulonglong2 cv = __ldg(reinterpret_cast<const ulonglong2*>(cq + row));
-        const ulonglong2 o = row_update<kObjective, kFastNoise>(p, q32, (uint32_t)i, xv, cv, xm, pivot,
-                                                                __int_as_float(pw.y), ragged, acc);
-        *reinterpret_cast<ulonglong2*>(oq + row) = o;
+      for (int i0 = r0 + rli; i0 < r1; i0 += step * kRowsInFlight) {
+        ulonglong2 xv[kRowsInFlight], xm[kRowsInFlight], cv[kRowsInFlight];
+        int2 pw[kRowsInFlight];
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {  // issue the loads of kRowsInFlight rows
+          const int i = i0 + u * step;
+          if (kRowsInFlight == 1 || i < r1) {
+            pw[u] = s_pw[i];
+            const uint64_t row = (uint64_t)(uint32_t)i * p.row_bytes;
+            xv[u] = __ldg(reinterpret_cast<const ulonglong2*>(xq + row));
+            xm[u] = __ldg(reinterpret_cast<const ulonglong2*>(xq + (uint64_t)(uint32_t)pw[u].x * p.row_bytes));
+            cv[u] = __ldg(reinterpret_cast<const ulonglong2*>(cq + row));
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+          const int i = i0 + u * step;
+          if (kRowsInFlight == 1 || i < r1) {
+            const ulonglong2 o = row_update<kObjective, kFastNoise>(p, q32, (uint32_t)i, xv[u], cv[u], xm[u], pivot,
+                                                                    __int_as_float(pw[u].y), ragged, acc);
+            *reinterpret_cast<ulonglong2*>(oq + (uint64_t)(uint32_t)i * p.row_bytes) = o;
+          }
+        }
       }
       unpack2(acc.s1a, s1.x, s1.y);
       unpack2(acc.s1b, s1.z, s1.w);
@@ -273,7 +310,36 @@ __global__ void __launch_bounds__(256, NETMAX_ROUND_MIN_CTAS) round_kernel(const
       s2 = s_col[blockDim.x + cgi];
       __syncthreads();
     }
-    if (rli == 0) {
+    bool owner = true;  // does this CTA hold the complete column sums of the tile?
+    if (G > 1) {
+      // rows are split over rg CTAs: publish this CTA's column partials; the last of the rg
+      // CTAs of a column tile to arrive adds them up in group order (deterministic)
+      if (rli == 0) {
+        p.colpart[((size_t)tile * p.cg + cgi) * 2] = s1;
+        p.colpart[((size_t)tile * p.cg + cgi) * 2 + 1] = s2;
+      }
+      __threadfence();
+      __syncthreads();
+      if (tid == 0) {
+        const unsigned int t = atomicAdd(p.coltick + ct, 1u);
+        s_lastcol = (t == (unsigned int)G - 1);
+        if (s_lastcol) p.coltick[ct] = 0u;
+      }
+      __syncthreads();
+      owner = s_lastcol;
+      if (owner && rli == 0) {
+        __threadfence();
+        s1 = make_float4(0.f, 0.f, 0.f, 0.f);
+        s2 = s1;
+        for (int gg = 0; gg < G; ++gg) {
+          const float4 a = __ldcg(p.colpart + (((size_t)ct * G + gg) * p.cg + cgi) * 2);
+          const float4 b = __ldcg(p.colpart + (((size_t)ct * G + gg) * p.cg + cgi) * 2 + 1);
+          s1.x += a.x; s1.y += a.y; s1.z += a.z; s1.w += a.w;
+          s2.x += b.x; s2.y += b.y; s2.z += b.z; s2.w += b.w;
+        }
+      }
+    }
+    if (rli == 0 && owner) {
       // sum_i (x_i - xbar)^2 = sum_i (x_i - a)^2 - (sum_i (x_i - a))^2 / M   per column
       const float cons = (s2.x - s1.x * s1.x * p.inv_M) + (s2.y - s1.y * s1.y * p.inv_M) +
                          (s2.z - s1.z * s1.z * p.inv_M) + (s2.w - s1.w * s1.w * p.inv_M);
