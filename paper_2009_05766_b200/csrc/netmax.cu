@@ -51,6 +51,7 @@ struct Layout {
 };
 
 constexpr int kMaxGrid = 148 * 16;  // upper bound on resident CTAs of the round kernel
+constexpr int64_t kMaxRoundsPerLaunch = 4096;  // rounds one cooperative launch runs at most
 constexpr size_t kColPartBytes = (size_t)8 << 20;  // column partials of the row-split (short vector) shape
 
 Layout make_layout(int64_t M, int64_t d, int64_t trace_rounds) {
@@ -69,7 +70,7 @@ Layout make_layout(int64_t M, int64_t d, int64_t trace_rounds) {
   L.off_w = take((size_t)M * M * sizeof(float));
   L.off_trace = take((size_t)trace_rounds * M * sizeof(int32_t));
   L.off_tel = take((size_t)trace_rounds * 2 * sizeof(double));
-  L.off_partials = take((size_t)kMaxGrid * 2 * sizeof(double));
+  L.off_partials = take((size_t)kMaxGrid * 2 * sizeof(double) * 2);  // two sets: multi-round launches alternate
   L.off_ticket = take(256);
   L.off_colpart = take(kColPartBytes);
   L.off_coltick = take((size_t)kMaxGrid * sizeof(unsigned int));
@@ -101,6 +102,9 @@ struct netmax_ctx {
   double* partials = nullptr;
   unsigned int* ticket = nullptr;
   float4* colpart = nullptr;
+  unsigned int* grid_barrier = nullptr;  // arrival counter of multi-round launches
+  unsigned int* dev_error = nullptr;     // raised by a kernel whose bounded wait gave up
+  bool cooperative = false;              // device supports cooperative launches
   unsigned int* coltick = nullptr;
   int cur = 0;  // index of the buffer holding the current replicas
   int64_t rounds = 0;
@@ -317,6 +321,12 @@ RoundKernel pick_kernel(int objective, bool short_vectors) {
   return objective == 1 ? round_kernel<1, true, 1> : round_kernel<0, true, 1>;
 }
 
+using MultiRoundKernel = void (*)(const MultiRoundParams);
+
+MultiRoundKernel pick_multi_kernel(int objective) {
+  return objective == 1 ? multi_round_kernel<1, true> : multi_round_kernel<0, true>;
+}
+
 int floor_pow2(int64_t v) {
   int r = 1;
   while ((int64_t)r * 2 <= v) r *= 2;
@@ -367,6 +377,15 @@ int plan_round(netmax_ctx* ctx, RoundPlan& plan) {
   int per_sm = 0;
   NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, plan.smem));
   if (per_sm < 1) return fail(ctx, NETMAX_CUDA_ERROR, "round kernel does not fit on an SM (smem %zu)", plan.smem);
+  if (plan.short_vectors && ctx->cooperative) {  // the multi-round kernel needs all of its CTAs resident
+    MultiRoundKernel mk = pick_multi_kernel(ctx->objective);
+    if (plan.smem > 48 * 1024)
+      NM_CUDA(ctx, cudaFuncSetAttribute(mk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
+    int per_sm_multi = 0;
+    NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm_multi, mk, kThreads, plan.smem));
+    per_sm = std::min(per_sm, per_sm_multi);
+    if (per_sm < 1) return fail(ctx, NETMAX_CUDA_ERROR, "multi-round kernel does not fit on an SM (smem %zu)", plan.smem);
+  }
   plan.grid = (int)std::min<int64_t>(plan.n_tiles, std::min<int64_t>((int64_t)per_sm * ctx->sm_count, kMaxGrid));
   return NETMAX_OK;
 }
@@ -453,7 +472,10 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   DeviceGuard guard(cfg->device);
   if (!guard.ok) { ctx->error = "cudaSetDevice failed"; return bail(NETMAX_CUDA_ERROR); }
   cudaDeviceProp prop;
-  if (cudaGetDeviceProperties(&prop, cfg->device) == cudaSuccess) ctx->sm_count = prop.multiProcessorCount;
+  if (cudaGetDeviceProperties(&prop, cfg->device) == cudaSuccess) {
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->cooperative = prop.cooperativeLaunch != 0;
+  }
   if (cfg->workspace) {
     if (((uintptr_t)cfg->workspace & 255) != 0) { ctx->error = "workspace is not 256-byte aligned"; return bail(NETMAX_INVALID_ARG); }
     if (cfg->workspace_bytes < ctx->L.total) {
@@ -488,6 +510,8 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   ctx->partials = (double*)(ctx->base + L.off_partials);
   ctx->ticket = (unsigned int*)(ctx->base + L.off_ticket);
   ctx->colpart = (float4*)(ctx->base + L.off_colpart);
+  ctx->grid_barrier = ctx->ticket + 16;
+  ctx->dev_error = ctx->ticket + 32;
   ctx->coltick = (unsigned int*)(ctx->base + L.off_coltick);
 
   auto step = [&](cudaError_t e, const char* what) {
@@ -566,6 +590,15 @@ int netmax_get_policy(netmax_ctx* ctx, double* prob_out, double* rho_out) {
   return NETMAX_OK;
 }
 
+// After a synchronisation: has a kernel's bounded wait given up since the last check?
+static int check_device_error(netmax_ctx* ctx) {
+  unsigned int flag = 0;
+  NM_CUDA(ctx, cudaMemcpy(&flag, ctx->dev_error, sizeof flag, cudaMemcpyDeviceToHost));
+  if (flag == 0) return NETMAX_OK;
+  cudaMemset(ctx->dev_error, 0, sizeof flag);
+  return fail(ctx, NETMAX_CUDA_ERROR, "a multi-round launch gave up waiting at its grid barrier; replicas are not valid");
+}
+
 static int copy_in(netmax_ctx* ctx, float* dst, const float* host) {
   if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
   if (!host) return fail(ctx, NETMAX_INVALID_ARG, "host pointer is NULL");
@@ -582,7 +615,7 @@ static int copy_out(netmax_ctx* ctx, const float* src, float* host) {
   NM_CUDA(ctx, cudaMemcpy2DAsync(host, (size_t)ctx->d * sizeof(float), src, (size_t)ctx->L.ld * sizeof(float),
                                  (size_t)ctx->d * sizeof(float), (size_t)ctx->M, cudaMemcpyDeviceToHost, ctx->stream));
   NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-  return NETMAX_OK;
+  return check_device_error(ctx);
 }
 
 int netmax_set_replicas(netmax_ctx* ctx, const float* host_x) { return copy_in(ctx, ctx ? ctx->x[ctx->cur] : nullptr, host_x); }
@@ -631,6 +664,38 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
     const int64_t batch = std::min<int64_t>(n_rounds - done, ctx->trace_rounds);
     rc = launch_sampler(ctx, (uint64_t)ctx->rounds, batch, ctx->trace, ctx->rounds % ctx->trace_rounds, ctx->trace_rounds);
     if (rc) return rc;
+    if (plan.short_vectors && ctx->cooperative && batch >= 2) {
+      // short, L2-resident problem: all rounds of the batch in cooperative launches
+      int64_t b = 0;
+      while (b < batch) {
+        const int64_t chunk = std::min<int64_t>(batch - b, kMaxRoundsPerLaunch);
+        MultiRoundParams mp;
+        mp.r = p;
+        mp.r.x_cur = reinterpret_cast<const float4*>(ctx->x[ctx->cur]);
+        mp.r.x_nxt = reinterpret_cast<float4*>(ctx->x[ctx->cur ^ 1]);
+        mp.r.peers = nullptr;
+        mp.r.tel_out = nullptr;
+        mp.trace = ctx->trace;
+        mp.tel = ctx->tel;
+        mp.partials2 = ctx->partials;
+        mp.barrier = ctx->grid_barrier;
+        mp.error = ctx->dev_error;
+        mp.slot0 = ctx->rounds % ctx->trace_rounds;
+        mp.ring = ctx->trace_rounds;
+        mp.first_round = (uint64_t)ctx->rounds;
+        mp.n_rounds = (int32_t)chunk;
+        NM_CUDA(ctx, cudaMemsetAsync(ctx->grid_barrier, 0, sizeof(unsigned int), ctx->stream));
+        void* args[] = {&mp};
+        NM_CUDA(ctx, cudaLaunchCooperativeKernel((const void*)pick_multi_kernel(ctx->objective), dim3(plan.grid), dim3(kThreads),
+                                                 args, plan.smem, ctx->stream));
+        ctx->launches += 1;
+        ctx->cur ^= (int)(chunk & 1);
+        ctx->rounds += chunk;
+        b += chunk;
+      }
+      done += batch;
+      continue;
+    }
     for (int64_t b = 0; b < batch; ++b) {
       const uint64_t r = (uint64_t)ctx->rounds;
       const int64_t slot = (int64_t)(r % (uint64_t)ctx->trace_rounds);
@@ -754,6 +819,8 @@ int netmax_peer_trace(netmax_ctx* ctx, int64_t first_round, int64_t n, int32_t* 
   if (!host_out) return fail(ctx, NETMAX_INVALID_ARG, "host_out is NULL");
   DeviceGuard guard(ctx->device);
   NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  rc = check_device_error(ctx);
+  if (rc) return rc;
   const size_t row = (size_t)ctx->M * sizeof(int32_t);
   int64_t r = first_round;
   while (r < first_round + n) {  // at most two contiguous pieces of the ring
@@ -772,6 +839,8 @@ int netmax_telemetry(netmax_ctx* ctx, int64_t first_round, int64_t n, double* ho
   if (n == 0) return NETMAX_OK;
   DeviceGuard guard(ctx->device);
   NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  rc = check_device_error(ctx);
+  if (rc) return rc;
   std::vector<double> ring((size_t)ctx->trace_rounds * 2);
   NM_CUDA(ctx, cudaMemcpy(ring.data(), ctx->tel, ring.size() * sizeof(double), cudaMemcpyDeviceToHost));
   for (int64_t k = 0; k < n; ++k) {

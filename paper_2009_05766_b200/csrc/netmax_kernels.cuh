@@ -88,9 +88,9 @@ struct RowAcc {
 // q32 is the global column-group index (first Philox counter word), tail > 0 marks the ragged
 // last group of a row whose padding lanes must stay zero.
 template <int kObjective, bool kFastNoise>
-__device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t q32, uint32_t worker, ulonglong2 xv,
-                                                 ulonglong2 cv, ulonglong2 xm, ulonglong2 pivot, float w, bool ragged,
-                                                 RowAcc& acc) {
+__device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t round_lo, uint32_t ctr3, uint32_t q32,
+                                                 uint32_t worker, ulonglong2 xv, ulonglong2 cv, ulonglong2 xm,
+                                                 ulonglong2 pivot, float w, bool ragged, RowAcc& acc) {
   const pair_t neg1 = pack2(-1.0f, -1.0f);
   const pair_t nw2 = pack2(-w, -w);
   const pair_t ta = fma2(cv.x, neg1, xv.x), tb = fma2(cv.y, neg1, xv.y);  // x - c
@@ -98,7 +98,7 @@ __device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t 
   if (kObjective == 1) {
     const pair_t sig2 = pack2(p.sigma, p.sigma);
     const pair_t nalpha2 = pack2(-p.alpha, -p.alpha);
-    const uint4 rnd = philox4x32_10(q32, worker, p.round_lo, p.ctr3, p.keys);
+    const uint4 rnd = philox4x32_10(q32, worker, round_lo, ctr3, p.keys);
     pair_t za, zb;
     if (kFastNoise) {
       za = normal_pair_fast_packed(rnd.x, rnd.y);
@@ -132,10 +132,9 @@ __device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t 
   return make_ulonglong2(oa, ob);
 }
 
-// Block reduction of a CTA's two telemetry sums; the last CTA of the grid to arrive then adds
-// all CTA partials in index order (deterministic) and publishes the round's telemetry.
+// Block reduction of a CTA's two telemetry sums into partials[2 * blockIdx.x ..].
 // s_red: 64 doubles of shared memory.  Every thread of the CTA must call this.
-__device__ __forceinline__ void finalize_telemetry(const RoundParams& p, double acc_cons, double acc_loss, double* s_red) {
+__device__ __forceinline__ void block_partials(double* partials, double acc_cons, double acc_loss, double* s_red) {
   const int tid = threadIdx.x;
   acc_loss *= 0.5;
   for (int off = 16; off > 0; off >>= 1) {
@@ -143,20 +142,60 @@ __device__ __forceinline__ void finalize_telemetry(const RoundParams& p, double 
     acc_loss += __shfl_down_sync(0xffffffffu, acc_loss, off);
   }
   const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
+  __syncthreads();  // s_red may still be read by an earlier call
   if (lane == 0) {
     s_red[warp] = acc_cons;
     s_red[32 + warp] = acc_loss;
   }
   __syncthreads();
-  __shared__ bool s_last;
   if (tid == 0) {
     double a = 0.0, b = 0.0;
     for (int wi = 0; wi < nwarps; ++wi) {
       a += s_red[wi];
       b += s_red[32 + wi];
     }
-    p.partials[2 * (size_t)blockIdx.x] = a;
-    p.partials[2 * (size_t)blockIdx.x + 1] = b;
+    partials[2 * (size_t)blockIdx.x] = a;
+    partials[2 * (size_t)blockIdx.x + 1] = b;
+  }
+}
+
+// Adds all CTA partials in index order (deterministic) and writes the round's telemetry.
+// Every thread of the (one) calling CTA must call this.
+__device__ __forceinline__ void sum_partials(const double* partials, double inv_M, double* tel_out, double* s_red) {
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
+  double a = 0.0, b = 0.0;
+  for (unsigned int j = tid; j < gridDim.x; j += blockDim.x) {
+    a += __ldcg(partials + 2 * (size_t)j);
+    b += __ldcg(partials + 2 * (size_t)j + 1);
+  }
+  for (int off = 16; off > 0; off >>= 1) {
+    a += __shfl_down_sync(0xffffffffu, a, off);
+    b += __shfl_down_sync(0xffffffffu, b, off);
+  }
+  __syncthreads();
+  if (lane == 0) {
+    s_red[warp] = a;
+    s_red[32 + warp] = b;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    a = 0.0;
+    b = 0.0;
+    for (int wi = 0; wi < nwarps; ++wi) {
+      a += s_red[wi];
+      b += s_red[32 + wi];
+    }
+    tel_out[0] = a * inv_M;
+    tel_out[1] = b * inv_M;
+  }
+}
+
+// One launch per round: the last CTA of the grid to publish its partials sums them.
+__device__ __forceinline__ void finalize_telemetry(const RoundParams& p, double acc_cons, double acc_loss, double* s_red) {
+  block_partials(p.partials, acc_cons, acc_loss, s_red);
+  __shared__ bool s_last;
+  if (threadIdx.x == 0) {
     __threadfence();
     const unsigned int t = atomicAdd(p.ticket, 1u);
     s_last = (t == gridDim.x - 1);
@@ -164,32 +203,8 @@ __device__ __forceinline__ void finalize_telemetry(const RoundParams& p, double 
   __syncthreads();
   if (s_last) {
     __threadfence();
-    double a = 0.0, b = 0.0;
-    for (unsigned int j = tid; j < gridDim.x; j += blockDim.x) {
-      a += __ldcg(p.partials + 2 * (size_t)j);
-      b += __ldcg(p.partials + 2 * (size_t)j + 1);
-    }
-    for (int off = 16; off > 0; off >>= 1) {
-      a += __shfl_down_sync(0xffffffffu, a, off);
-      b += __shfl_down_sync(0xffffffffu, b, off);
-    }
-    __syncthreads();
-    if (lane == 0) {
-      s_red[warp] = a;
-      s_red[32 + warp] = b;
-    }
-    __syncthreads();
-    if (tid == 0) {
-      a = 0.0;
-      b = 0.0;
-      for (int wi = 0; wi < nwarps; ++wi) {
-        a += s_red[wi];
-        b += s_red[32 + wi];
-      }
-      p.tel_out[0] = a * (double)p.inv_M;
-      p.tel_out[1] = b * (double)p.inv_M;
-      *p.ticket = 0u;
-    }
+    sum_partials(p.partials, (double)p.inv_M, p.tel_out, s_red);
+    if (threadIdx.x == 0) *p.ticket = 0u;
   }
 }
 
@@ -208,33 +223,39 @@ __device__ __forceinline__ void finalize_telemetry(const RoundParams& p, double 
 // kRowsInFlight = 1 (64 registers, 4 CTAs/SM) is the streaming shape for long vectors, where
 // occupancy hides the HBM latency; kRowsInFlight = 4 (2 CTAs/SM) serves short, L2-resident
 // problems, where a thread's chain of dependent row loads is what takes the time.
-template <int kObjective, bool kFastNoise, int kRowsInFlight>
-__global__ void __launch_bounds__(256, kRowsInFlight == 1 ? NETMAX_ROUND_MIN_CTAS : 2) round_kernel(const RoundParams p) {
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  int2* s_pw = reinterpret_cast<int2*>(smem_raw);  // (peer, bits of the pull weight) per worker
-  const size_t head = (((size_t)p.M * 8) + 15) & ~(size_t)15;
-  float4* s_col = reinterpret_cast<float4*>(smem_raw + head);
-  double* s_red = reinterpret_cast<double*>(smem_raw + head + (p.rl > 1 ? (size_t)blockDim.x * 32 : 0));
+// this round's (peer, weight) of workers [r0, r1) into shared memory
+__device__ __forceinline__ void load_draws(const RoundParams& p, const int32_t* peers, int2* s_pw, int r0, int r1) {
+  for (int i = r0 + threadIdx.x; i < r1; i += blockDim.x) {
+    const int32_t m = __ldg(peers + i);
+    s_pw[i] = make_int2(m, __float_as_int((m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * p.M + m)));
+  }
+}
 
+// Loads of replica data.  Inside one launch per round the round-start buffer is read-only
+// (non-coherent path); a launch that runs several rounds reads what other SMs wrote a round
+// earlier and must bypass L1.
+template <bool kCoherent>
+__device__ __forceinline__ ulonglong2 ld_x(const char* ptr) {
+  return kCoherent ? __ldcg(reinterpret_cast<const ulonglong2*>(ptr)) : __ldg(reinterpret_cast<const ulonglong2*>(ptr));
+}
+
+// All tiles of this CTA for one round.  Every thread of the CTA must call this.
+template <int kObjective, bool kFastNoise, int kRowsInFlight, bool kCoherent>
+__device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* x_cur, float4* x_nxt, const int32_t* peers,
+                                            uint32_t round_lo, uint32_t ctr3, int2* s_pw, float4* s_col,
+                                            double& acc_cons, double& acc_loss) {
   const int tid = threadIdx.x;
   const int G = p.rg;
-  auto load_draws = [&](int r0, int r1) {  // this round's (peer, weight) of workers [r0, r1)
-    for (int i = r0 + tid; i < r1; i += blockDim.x) {
-      const int32_t m = __ldg(p.peers + i);
-      s_pw[i] = make_int2(m, __float_as_int((m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * p.M + m)));
-    }
-  };
-  if (G == 1) {
-    load_draws(0, p.M);
-    __syncthreads();
-  }
   __shared__ bool s_lastcol;
-
   const int cgi = tid & (p.cg - 1);
   const int rli = tid / p.cg;
   const int M = p.M;
   const int step = p.rl;
-  double acc_cons = 0.0, acc_loss = 0.0;
+  if (G == 1) {
+    __syncthreads();  // readers of the previous round's draws are done
+    load_draws(p, peers, s_pw, 0, M);
+    __syncthreads();
+  }
 
   for (int64_t tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x) {
     const int64_t ct = G == 1 ? tile : tile / G;      // column tile
@@ -242,7 +263,7 @@ __global__ void __launch_bounds__(256, kRowsInFlight == 1 ? NETMAX_ROUND_MIN_CTA
     const int r0 = grp * p.rows_per_group, r1 = min(M, r0 + p.rows_per_group);
     if (G > 1) {
       __syncthreads();  // the previous tile's readers of s_pw are done
-      load_draws(r0, r1);
+      load_draws(p, peers, s_pw, r0, r1);
       __syncthreads();
     }
     const int64_t q = ct * p.cg + cgi;
@@ -252,11 +273,11 @@ __global__ void __launch_bounds__(256, kRowsInFlight == 1 ? NETMAX_ROUND_MIN_CTA
     float loss = 0.f;
     if (live) {
       // byte pointers to this thread's column group in row 0; row i is i * row_bytes further
-      const char* xq = reinterpret_cast<const char*>(p.x_cur + q);
+      const char* xq = reinterpret_cast<const char*>(x_cur + q);
       const char* cq = reinterpret_cast<const char*>(p.c + q);
-      char* oq = reinterpret_cast<char*>(p.x_nxt + q);
+      char* oq = reinterpret_cast<char*>(x_nxt + q);
       const uint32_t q32 = (uint32_t)q + p.q_offset;
-      const ulonglong2 pivot = __ldg(reinterpret_cast<const ulonglong2*>(xq));  // row 0: pivot of the one-pass variance
+      const ulonglong2 pivot = ld_x<kCoherent>(xq);  // row 0: pivot of the one-pass variance
       RowAcc acc;
       for (int i0 = r0 + rli; i0 < r1; i0 += step * kRowsInFlight) {
         ulonglong2 xv[kRowsInFlight], xm[kRowsInFlight], cv[kRowsInFlight];
@@ -267,8 +288,8 @@ __global__ void __launch_bounds__(256, kRowsInFlight == 1 ? NETMAX_ROUND_MIN_CTA
           if (kRowsInFlight == 1 || i < r1) {
             pw[u] = s_pw[i];
             const uint64_t row = (uint64_t)(uint32_t)i * p.row_bytes;
-            xv[u] = __ldg(reinterpret_cast<const ulonglong2*>(xq + row));
-            xm[u] = __ldg(reinterpret_cast<const ulonglong2*>(xq + (uint64_t)(uint32_t)pw[u].x * p.row_bytes));
+            xv[u] = ld_x<kCoherent>(xq + row);
+            xm[u] = ld_x<kCoherent>(xq + (uint64_t)(uint32_t)pw[u].x * p.row_bytes);
             cv[u] = __ldg(reinterpret_cast<const ulonglong2*>(cq + row));
           }
         }
@@ -276,8 +297,8 @@ __global__ void __launch_bounds__(256, kRowsInFlight == 1 ? NETMAX_ROUND_MIN_CTA
         for (int u = 0; u < kRowsInFlight; ++u) {
           const int i = i0 + u * step;
           if (kRowsInFlight == 1 || i < r1) {
-            const ulonglong2 o = row_update<kObjective, kFastNoise>(p, q32, (uint32_t)i, xv[u], cv[u], xm[u], pivot,
-                                                                    __int_as_float(pw[u].y), ragged, acc);
+            const ulonglong2 o = row_update<kObjective, kFastNoise>(p, round_lo, ctr3, q32, (uint32_t)i, xv[u], cv[u],
+                                                                    xm[u], pivot, __int_as_float(pw[u].y), ragged, acc);
             *reinterpret_cast<ulonglong2*>(oq + (uint64_t)(uint32_t)i * p.row_bytes) = o;
           }
         }
@@ -347,7 +368,94 @@ __global__ void __launch_bounds__(256, kRowsInFlight == 1 ? NETMAX_ROUND_MIN_CTA
     }
     acc_loss += (double)loss;
   }
+}
+
+// kRowsInFlight = 1 (64 registers, 4 CTAs/SM) is the streaming shape for long vectors, where
+// occupancy hides the HBM latency; kRowsInFlight = 4 (2 CTAs/SM) serves short, L2-resident
+// problems, where a thread's chain of dependent row loads is what takes the time.
+template <int kObjective, bool kFastNoise, int kRowsInFlight>
+__global__ void __launch_bounds__(256, kRowsInFlight == 1 ? NETMAX_ROUND_MIN_CTAS : 2) round_kernel(const RoundParams p) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  int2* s_pw = reinterpret_cast<int2*>(smem_raw);  // (peer, bits of the pull weight) per worker
+  const size_t head = (((size_t)p.M * 8) + 15) & ~(size_t)15;
+  float4* s_col = reinterpret_cast<float4*>(smem_raw + head);
+  double* s_red = reinterpret_cast<double*>(smem_raw + head + (p.rl > 1 ? (size_t)blockDim.x * 32 : 0));
+  double acc_cons = 0.0, acc_loss = 0.0;
+  round_tiles<kObjective, kFastNoise, kRowsInFlight, false>(p, p.x_cur, p.x_nxt, p.peers, p.round_lo, p.ctr3, s_pw, s_col,
+                                                            acc_cons, acc_loss);
   finalize_telemetry(p, acc_cons, acc_loss, s_red);
+}
+
+// ---- several rounds in one launch (short, L2-resident problems) ------------------------------
+// For problems of a few microseconds per round the launch and the chain of dependent global
+// round trips are what take the time.  This kernel is launched cooperatively (all CTAs
+// resident), runs n_rounds rounds back to back and separates them with a grid-wide barrier: an
+// arrival counter in global memory that every CTA polls a bounded number of times.  A CTA
+// whose wait runs out raises *error and leaves; the others then run out as well.
+struct MultiRoundParams {
+  RoundParams r;          // x_cur / x_nxt: the buffers of the first round; peers, tel_out, round_lo, ctr3 unused
+  const int32_t* trace;   // peer-trace ring [ring][M], filled for these rounds by sample_peers_kernel
+  double* tel;            // telemetry ring [ring][2]
+  double* partials2;      // [2][gridDim.x][2]: CTA partials, alternating by round
+  unsigned int* barrier;  // arrival counter, 0 at launch
+  unsigned int* error;    // raised when a barrier wait gave up
+  int64_t slot0, ring;    // ring slot of the first round
+  uint64_t first_round;
+  int32_t n_rounds;
+};
+
+constexpr uint32_t kBarrierSpinLimit = 1u << 21;
+
+// Grid-wide barrier number `epoch` (1, 2, ...).  Returns false if the wait gave up.
+__device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int epoch, unsigned int* error) {
+  __shared__ int s_ok;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();  // this CTA's writes of the round are visible before it is counted
+    atomicAdd(counter, 1u);
+    const unsigned int target = epoch * gridDim.x;
+    int ok = 0;
+    for (uint32_t it = 0; it < kBarrierSpinLimit; ++it) {
+      if (*reinterpret_cast<volatile unsigned int*>(counter) >= target) {
+        ok = 1;
+        break;
+      }
+      __nanosleep(32);
+    }
+    if (!ok) atomicExch(error, 1u);
+    __threadfence();
+    s_ok = ok;
+  }
+  __syncthreads();
+  return s_ok != 0;
+}
+
+template <int kObjective, bool kFastNoise>
+__global__ void __launch_bounds__(256, 2) multi_round_kernel(const MultiRoundParams mp) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const RoundParams& p = mp.r;
+  int2* s_pw = reinterpret_cast<int2*>(smem_raw);
+  const size_t head = (((size_t)p.M * 8) + 15) & ~(size_t)15;
+  float4* s_col = reinterpret_cast<float4*>(smem_raw + head);
+  double* s_red = reinterpret_cast<double*>(smem_raw + head + (p.rl > 1 ? (size_t)blockDim.x * 32 : 0));
+  const float4* x_cur = p.x_cur;
+  float4* x_nxt = p.x_nxt;
+  for (int k = 0; k < mp.n_rounds; ++k) {
+    const uint64_t round = mp.first_round + (uint64_t)k;
+    const int64_t slot = (mp.slot0 + k) % mp.ring;
+    double* partials = mp.partials2 + (size_t)(k & 1) * 2 * gridDim.x;
+    double acc_cons = 0.0, acc_loss = 0.0;
+    round_tiles<kObjective, kFastNoise, 4, true>(p, x_cur, x_nxt, mp.trace + slot * p.M, (uint32_t)round,
+                                                 philox_ctr3(kTagNoise, round), s_pw, s_col, acc_cons, acc_loss);
+    block_partials(partials, acc_cons, acc_loss, s_red);
+    if (!grid_barrier(mp.barrier, (unsigned int)(k + 1), mp.error)) return;
+    // round k is complete everywhere: one CTA publishes its telemetry while the rest move on
+    // (partials alternate, so round k+1 cannot overwrite what is being summed here)
+    if (blockIdx.x == 0) sum_partials(partials, (double)p.inv_M, mp.tel + 2 * slot, s_red);
+    const float4* t = x_cur;
+    x_cur = x_nxt;
+    x_nxt = const_cast<float4*>(t);
+  }
 }
 
 // ------------------------------------------------------------------------- init / IO
