@@ -16,6 +16,11 @@
 // (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", SC'11),
 // implemented here from its published definition.
 //
+// A second mode follows the paper's own process (Section II-B, Eq. 17): workers run
+// asynchronously on simulated clocks, an iteration of worker i with peer m lasts t_im, and at
+// every global step exactly ONE worker -- the one whose iteration finishes next -- updates
+// its replica from the peer's CURRENT replica (nmo_async_*).
+//
 // Only tests, the smoke check and the benchmark's cpu_baseline leg may use this file.
 // It shares no code with the CUDA library and includes none of its headers.
 //
@@ -155,6 +160,19 @@ struct Sim {
   std::vector<float> x, xn, c;  // [M][ncols]
   std::vector<int32_t> trace;   // [round][M], all rounds since creation
   std::vector<double> tel_consensus, tel_loss;  // per round, on the round-start state
+  // asynchronous timeline
+  bool async_on = false;
+  double beta = 0.0;
+  std::vector<double> t_iter;          // [M][M] iteration times, t_ii = compute-only
+  std::vector<int64_t> local_n;        // [M] local iteration index n of the pending iteration
+  std::vector<int32_t> pending_peer;   // [M] peer drawn for the pending iteration
+  std::vector<double> finish;          // [M] simulated time at which the pending iteration ends
+  std::vector<double> ema;             // [M][M] EMA of measured iteration times (Algorithm 2)
+  std::vector<int64_t> ema_count;      // [M][M] samples folded into the EMA
+  double now = 0.0;
+  std::vector<int32_t> ev_worker, ev_peer;
+  std::vector<int64_t> ev_n;
+  std::vector<double> ev_time;
 };
 
 void sim_set_policy(Sim* s, const double* P, const uint8_t* adj, double rho) {
@@ -262,6 +280,64 @@ void sim_round(Sim* s, int threads) {
   }
   s->x.swap(s->xn);
   s->round += 1;
+}
+
+// ---------------------------------------------------------------- asynchronous timeline
+// Worker i's iteration n: peer m drawn from P[i,:] with the PEER stream at counter (0, i, n),
+// duration t_im (Section II-B: t_im = max{C_i, N_im}); the next iteration starts when this
+// one ends.  A policy or time-matrix change affects iterations that START afterwards.
+void async_start_iteration(Sim* s, int i, double start) {
+  uint32_t ctr[4], r[4];
+  make_ctr(0, (uint32_t)i, (uint64_t)s->local_n[i], TAG_PEER, ctr);
+  philox4x32_10(ctr, s->key, r);
+  const int m = sample_row(s->T.data() + (size_t)i * s->M, s->M, s->last_nz[i], r[0]);
+  s->pending_peer[i] = m;
+  s->finish[i] = start + s->t_iter[(size_t)i * s->M + m];
+}
+
+// One global step (Eq. 17): the worker whose iteration finishes first (ties: lowest index)
+// applies  x_i <- (1 - w_im)(x_i - alpha g_i) + w_im x_m  with the peer's current replica;
+// every other replica is unchanged.  Then it records the iteration time (Algorithm 2,
+// UpdateTimeVector: T_i[m] <- beta T_i[m] + (1 - beta) t_im) and starts its next iteration.
+void async_step(Sim* s) {
+  const int M = s->M;
+  int i = 0;
+  for (int j = 1; j < M; ++j)
+    if (s->finish[j] < s->finish[i]) i = j;
+  const int m = s->pending_peer[i];
+  const int64_t nloc = s->local_n[i];
+  const double w = (double)s->w[(size_t)i * M + m];
+  const int64_t n = s->ncols;
+  float* xi = s->x.data() + (size_t)i * n;
+  const float* xm = s->x.data() + (size_t)m * n;
+  const float* ci = s->c.data() + (size_t)i * n;
+  for (int64_t k = 0; k < n; ++k) {
+    const int64_t e = s->cols[k];
+    const double xv = (double)xi[k];
+    double g = 0.0;
+    if (s->objective == 1) {
+      uint32_t ctr[4], r[4];
+      double z[4];
+      make_ctr((uint32_t)(e >> 2), (uint32_t)i, (uint64_t)nloc, TAG_NOISE, ctr);
+      philox4x32_10(ctr, s->key, r);
+      normals4(r, z);
+      g = (xv - (double)ci[k]) + s->sigma * z[e & 3];
+    }
+    const double h = xv - s->alpha * g;
+    double xnew = h;
+    if (m != i) xnew = h - w * (h - (double)xm[k]);
+    xi[k] = (float)xnew;
+  }
+  s->now = s->finish[i];
+  s->ev_worker.push_back(i);
+  s->ev_peer.push_back(m);
+  s->ev_n.push_back(nloc);
+  s->ev_time.push_back(s->now);
+  const size_t at = (size_t)i * M + m;
+  s->ema[at] = s->beta * s->ema[at] + (1.0 - s->beta) * s->t_iter[at];
+  s->ema_count[at] += 1;
+  s->local_n[i] = nloc + 1;
+  async_start_iteration(s, i, s->now);
 }
 
 }  // namespace
@@ -381,5 +457,49 @@ void nmo_sim_get_telemetry(void* h, int64_t first, int64_t n, double* consensus,
 }
 
 void nmo_sim_telemetry_now(void* h, double* consensus, double* loss) { telemetry((Sim*)h, consensus, loss); }
+
+// ---- asynchronous timeline
+void nmo_async_begin(void* h, const double* t_iter, double beta) {
+  Sim* s = (Sim*)h;
+  const int M = s->M;
+  s->async_on = true;
+  s->beta = beta;
+  s->t_iter.assign(t_iter, t_iter + (size_t)M * M);
+  s->local_n.assign(M, 0);
+  s->pending_peer.assign(M, 0);
+  s->finish.assign(M, 0.0);
+  s->ema.assign((size_t)M * M, 0.0);
+  s->ema_count.assign((size_t)M * M, 0);
+  s->now = 0.0;
+  for (int i = 0; i < M; ++i) async_start_iteration(s, i, 0.0);
+}
+
+void nmo_async_set_times(void* h, const double* t_iter) {
+  Sim* s = (Sim*)h;
+  s->t_iter.assign(t_iter, t_iter + (size_t)s->M * s->M);
+}
+
+void nmo_async_steps(void* h, int64_t n) {
+  for (int64_t k = 0; k < n; ++k) async_step((Sim*)h);
+}
+
+int64_t nmo_async_steps_done(void* h) { return (int64_t)((Sim*)h)->ev_worker.size(); }
+double nmo_async_now(void* h) { return ((Sim*)h)->now; }
+
+void nmo_async_trace(void* h, int64_t first, int64_t n, int32_t* worker, int32_t* peer, int64_t* local_iter, double* time) {
+  Sim* s = (Sim*)h;
+  for (int64_t k = 0; k < n; ++k) {
+    worker[k] = s->ev_worker[first + k];
+    peer[k] = s->ev_peer[first + k];
+    local_iter[k] = s->ev_n[first + k];
+    time[k] = s->ev_time[first + k];
+  }
+}
+
+void nmo_async_ema(void* h, double* ema, int64_t* count) {
+  Sim* s = (Sim*)h;
+  std::memcpy(ema, s->ema.data(), s->ema.size() * sizeof(double));
+  std::memcpy(count, s->ema_count.data(), s->ema_count.size() * sizeof(int64_t));
+}
 
 }  // extern "C"

@@ -63,6 +63,15 @@ def lib():
         L.nmo_sim_get_trace.argtypes = [vp, i64, i64, vp]
         L.nmo_sim_get_telemetry.argtypes = [vp, i64, i64, vp, vp]
         L.nmo_sim_telemetry_now.argtypes = [vp, vp, vp]
+        L.nmo_async_begin.argtypes = [vp, vp, dbl]
+        L.nmo_async_set_times.argtypes = [vp, vp]
+        L.nmo_async_steps.argtypes = [vp, i64]
+        L.nmo_async_steps_done.argtypes = [vp]
+        L.nmo_async_steps_done.restype = i64
+        L.nmo_async_now.argtypes = [vp]
+        L.nmo_async_now.restype = dbl
+        L.nmo_async_trace.argtypes = [vp, i64, i64, vp, vp, vp, vp]
+        L.nmo_async_ema.argtypes = [vp, vp, vp]
         _lib = L
     return _lib
 
@@ -199,6 +208,42 @@ class Sim:
         loss = np.empty(n, dtype=np.float64)
         lib().nmo_sim_get_telemetry(self._h, first, n, _p(cons), _p(loss))
         return cons, loss
+
+    # ---- asynchronous timeline (the paper's one-worker-per-global-step process)
+    def async_begin(self, t_iter, beta):
+        t = np.ascontiguousarray(t_iter, dtype=np.float64)
+        assert t.shape == (self.M, self.M)
+        lib().nmo_async_begin(self._h, _p(t), float(beta))
+
+    def async_set_times(self, t_iter):
+        t = np.ascontiguousarray(t_iter, dtype=np.float64)
+        lib().nmo_async_set_times(self._h, _p(t))
+
+    def async_steps(self, n):
+        lib().nmo_async_steps(self._h, int(n))
+
+    @property
+    def async_steps_done(self) -> int:
+        return int(lib().nmo_async_steps_done(self._h))
+
+    @property
+    def async_now(self) -> float:
+        return float(lib().nmo_async_now(self._h))
+
+    def async_trace(self, first=0, n=None):
+        n = self.async_steps_done - first if n is None else n
+        worker = np.empty(n, dtype=np.int32)
+        peer = np.empty(n, dtype=np.int32)
+        local_iter = np.empty(n, dtype=np.int64)
+        time = np.empty(n, dtype=np.float64)
+        lib().nmo_async_trace(self._h, first, n, _p(worker), _p(peer), _p(local_iter), _p(time))
+        return worker, peer, local_iter, time
+
+    def async_ema(self):
+        ema = np.empty((self.M, self.M), dtype=np.float64)
+        count = np.empty((self.M, self.M), dtype=np.int64)
+        lib().nmo_async_ema(self._h, _p(ema), _p(count))
+        return ema, count
 
     def telemetry_now(self):
         a, b = C.c_double(), C.c_double()
