@@ -188,6 +188,50 @@ int netmax_peer_trace(netmax_ctx* ctx, int64_t first_round, int64_t n, int32_t* 
 int netmax_telemetry(netmax_ctx* ctx, int64_t first_round, int64_t n, double* host_consensus, double* host_loss);
 
 /*
+ * Telemetry of the CURRENT replicas, on demand: the same two quantities as netmax_telemetry
+ * (consensus distance and mean loss, the observable parts of Eq. 1), computed by one
+ * read-only kernel.  Either output may be NULL.  Synchronises.
+ */
+int netmax_measure(netmax_ctx* ctx, double* consensus, double* loss);
+
+/*
+ * Asynchronous timeline: the paper's own process (Section II-B and Eq. 17), in which workers
+ * run on their own clocks and exactly ONE worker updates at every global step.
+ *
+ * Worker i's local iteration n draws its peer m from P[i,:] (Algorithm 2; the peer stream at
+ * counter (worker i, iteration n)), lasts t_im = max{C_i, N_im} (t_ii for a self-draw) and is
+ * followed at once by iteration n + 1.  Global step k belongs to the worker whose iteration
+ * finishes next (ties: the lowest index); it applies Eq. 15 and Eq. 16 to x_i IN PLACE with the
+ * peer's replica as it is at that moment (x_m^k in Eq. 17), then folds the iteration time into
+ * its moving average T_i[m] <- beta T_i[m] + (1 - beta) t_im (Algorithm 2, UpdateTimeVector;
+ * T starts at 0).  A policy set with netmax_set_policy, and the iteration times that come
+ * with new link speeds, apply to iterations that START afterwards (Algorithm 2: "if received
+ * new policy").  The clocks and draws are host control plane; the replica updates run on the
+ * GPU, consecutive steps on disjoint replicas sharing a launch.
+ *
+ * netmax_async_begin switches a context that has run no round to this timeline for good
+ * (netmax_round is refused afterwards).  t_iter (host, M*M, t_ii on the diagonal) overrides
+ * the iteration times derived from the context's link speeds; NULL keeps those.
+ */
+int netmax_async_begin(netmax_ctx* ctx, const double* t_iter, double beta);
+/* Replaces the iteration-time matrix (host, M*M) for iterations that start afterwards. */
+int netmax_async_set_times(netmax_ctx* ctx, const double* t_iter);
+/* Runs the next n_steps global steps, asynchronously on the context's stream. */
+int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps);
+/* Simulated time of the last global step and the number of global steps so far. */
+int netmax_async_time(netmax_ctx* ctx, double* sim_time, int64_t* steps_done);
+/*
+ * The global steps [first_step, first_step + n): which worker acted, the peer it pulled from,
+ * its local iteration number and the simulated finish time.  Host arrays of n entries, any of
+ * which may be NULL.  The last max(trace_rounds * M, 1024) steps are kept.
+ */
+int netmax_async_trace(netmax_ctx* ctx, int64_t first_step, int64_t n, int32_t* worker, int32_t* peer,
+                       int64_t* local_iter, double* finish_time);
+/* The moving averages T_i[m] (host, M*M) and how many samples each has seen (may be NULL):
+ * what the Network Monitor of Algorithm 1 collects. */
+int netmax_async_ema(netmax_ctx* ctx, double* ema_out, int64_t* samples_out);
+
+/*
  * Device access for callers that keep working on the GPU (for example through PyTorch):
  * *x is the buffer holding the current replicas, row i at x + i * ld, ld >= d floats,
  * valid until the next netmax_round / netmax_set_* call; nothing is synchronised.

@@ -24,6 +24,8 @@ EXPORTS = [
     "netmax_rounds_done", "netmax_read_replicas", "netmax_read_centres", "netmax_read_columns",
     "netmax_read_columns_static",
     "netmax_peer_trace", "netmax_telemetry", "netmax_replicas_device", "netmax_sample_peers",
+    "netmax_measure", "netmax_async_begin", "netmax_async_set_times", "netmax_async_steps", "netmax_async_time",
+    "netmax_async_trace", "netmax_async_ema",
     "netmax_iteration_times", "netmax_policy_generate", "netmax_kernel_launches", "netmax_last_error",
 ]
 
@@ -80,6 +82,13 @@ def lib():
             "netmax_telemetry": ([vp, i64, i64, vp, vp], C.c_int),
             "netmax_replicas_device": ([vp, vp, vp], C.c_int),
             "netmax_sample_peers": ([vp, i64, i64, vp], C.c_int),
+            "netmax_measure": ([vp, vp, vp], C.c_int),
+            "netmax_async_begin": ([vp, vp, dbl], C.c_int),
+            "netmax_async_set_times": ([vp, vp], C.c_int),
+            "netmax_async_steps": ([vp, i64], C.c_int),
+            "netmax_async_time": ([vp, vp, vp], C.c_int),
+            "netmax_async_trace": ([vp, i64, i64, vp, vp, vp, vp], C.c_int),
+            "netmax_async_ema": ([vp, vp, vp], C.c_int),
             "netmax_iteration_times": ([i32, i64, vp, vp, vp], C.c_int),
             "netmax_policy_generate": ([i32, vp, vp, dbl, i32, i32, vp, vp, vp], C.c_int),
             "netmax_kernel_launches": ([vp], i64),
@@ -265,6 +274,44 @@ class Netmax:
 
     def sample_peers(self, first_round: int, n_rounds: int, device_out: int):
         _check(lib().netmax_sample_peers(self._h, int(first_round), int(n_rounds), C.c_void_p(device_out)), self._h)
+
+    def measure(self):
+        cons, loss = C.c_double(), C.c_double()
+        _check(lib().netmax_measure(self._h, C.byref(cons), C.byref(loss)), self._h)
+        return cons.value, loss.value
+
+    # ---- asynchronous timeline (one worker per global step)
+    def async_begin(self, t_iter=None, beta: float = 0.9):
+        t = _f64(t_iter, (self.M, self.M)) if t_iter is not None else None
+        _check(lib().netmax_async_begin(self._h, _p(t), float(beta)), self._h)
+
+    def async_set_times(self, t_iter):
+        t = _f64(t_iter, (self.M, self.M))
+        _check(lib().netmax_async_set_times(self._h, _p(t)), self._h)
+
+    def async_steps(self, n_steps: int):
+        _check(lib().netmax_async_steps(self._h, int(n_steps)), self._h)
+
+    def async_time(self):
+        t, k = C.c_double(), C.c_int64()
+        _check(lib().netmax_async_time(self._h, C.byref(t), C.byref(k)), self._h)
+        return t.value, k.value
+
+    def async_trace(self, first_step: int = 0, n: Optional[int] = None):
+        n = self.async_time()[1] - first_step if n is None else n
+        worker = np.empty(n, dtype=np.int32)
+        peer = np.empty(n, dtype=np.int32)
+        local_iter = np.empty(n, dtype=np.int64)
+        time = np.empty(n, dtype=np.float64)
+        _check(lib().netmax_async_trace(self._h, int(first_step), int(n), _p(worker), _p(peer), _p(local_iter),
+                                        _p(time)), self._h)
+        return worker, peer, local_iter, time
+
+    def async_ema(self):
+        ema = np.empty((self.M, self.M), dtype=np.float64)
+        count = np.empty((self.M, self.M), dtype=np.int64)
+        _check(lib().netmax_async_ema(self._h, _p(ema), _p(count)), self._h)
+        return ema, count
 
     @property
     def kernel_launches(self) -> int:

@@ -105,6 +105,26 @@ struct netmax_ctx {
   unsigned int* grid_barrier = nullptr;  // arrival counter of multi-round launches
   unsigned int* dev_error = nullptr;     // raised by a kernel whose bounded wait gave up
   bool cooperative = false;              // device supports cooperative launches
+  double* measure_out = nullptr;         // device: (consensus, loss) of netmax_measure
+  // host copies of the tables in force (the asynchronous timeline draws peers on the host)
+  std::vector<uint32_t> h_thr;
+  std::vector<int32_t> h_last;
+  std::vector<float> h_w;
+  std::vector<double> t_iter;  // iteration times derived from the link speeds in force
+  // asynchronous timeline (one worker per global step)
+  bool async_on = false;
+  double beta = 0.0;
+  double now = 0.0;
+  int64_t steps = 0;
+  std::vector<int64_t> local_n;
+  std::vector<int32_t> pending_peer;
+  std::vector<double> finish;
+  std::vector<double> ema;
+  std::vector<int64_t> ema_count;
+  int64_t ev_cap = 0;
+  std::vector<int32_t> ev_worker, ev_peer;
+  std::vector<int64_t> ev_n;
+  std::vector<double> ev_time;
   unsigned int* coltick = nullptr;
   int cur = 0;  // index of the buffer holding the current replicas
   int64_t rounds = 0;
@@ -227,9 +247,9 @@ void build_tables(int32_t M, const double* P, const std::vector<uint8_t>& adj, d
 }
 
 int upload_policy(netmax_ctx* ctx) {
-  std::vector<uint32_t> thr;
-  std::vector<int32_t> last;
-  std::vector<float> w;
+  std::vector<uint32_t>& thr = ctx->h_thr;
+  std::vector<int32_t>& last = ctx->h_last;
+  std::vector<float>& w = ctx->h_w;
   build_tables(ctx->M, ctx->P.data(), ctx->adj, (double)(float)ctx->alpha, ctx->rho, thr, last, w);
   // pageable sources: the copies are complete (staged) when these calls return
   NM_CUDA(ctx, cudaMemcpyAsync(ctx->thr, thr.data(), thr.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));
@@ -239,9 +259,29 @@ int upload_policy(netmax_ctx* ctx) {
   return NETMAX_OK;
 }
 
-// Chooses P and rho: the caller's, or Algorithm 3's.
+// Iteration times of the link speeds in force (equal speeds when none were given).
+int refresh_iteration_times(netmax_ctx* ctx, const double* speed) {
+  const int32_t M = ctx->M;
+  std::vector<double> flat;
+  if (!speed) {
+    flat.assign((size_t)M * M, 1.0);
+    speed = flat.data();
+  }
+  std::vector<uint8_t> adj2((size_t)M * M);
+  ctx->t_iter.assign((size_t)M * M, 0.0);
+  int rc = netmax_iteration_times(M, ctx->d, speed, ctx->t_iter.data(), adj2.data());
+  if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
+  return NETMAX_OK;
+}
+
+// Chooses P and rho: the caller's, or Algorithm 3's.  speed == NULL keeps the iteration times
+// in force (or, at creation, takes equal speeds).
 int resolve_policy(netmax_ctx* ctx, const double* speed, const double* prob, double rho) {
   const int32_t M = ctx->M;
+  if (speed || ctx->t_iter.empty()) {
+    int rc = refresh_iteration_times(ctx, speed);
+    if (rc) return rc;
+  }
   if (prob) {
     int rc = validate_policy(ctx, M, prob, ctx->adj);
     if (rc) return rc;
@@ -249,17 +289,10 @@ int resolve_policy(netmax_ctx* ctx, const double* speed, const double* prob, dou
     ctx->rho = rho > 0.0 ? rho : default_rho(M, prob, ctx->adj, ctx->alpha);
     return NETMAX_OK;
   }
-  std::vector<double> t((size_t)M * M), flat;
-  std::vector<uint8_t> adj2((size_t)M * M);
-  if (!speed) {
-    flat.assign((size_t)M * M, 1.0);
-    speed = flat.data();
-  }
-  int rc = netmax_iteration_times(M, ctx->d, speed, t.data(), adj2.data());
-  if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
   ctx->P.assign((size_t)M * M, 0.0);
   double rho_sel = 0.0;
-  rc = netmax_policy_generate(M, t.data(), adj2.data(), ctx->alpha, ctx->policy_K, ctx->policy_R, ctx->P.data(), &rho_sel, nullptr);
+  int rc = netmax_policy_generate(M, ctx->t_iter.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K, ctx->policy_R,
+                                  ctx->P.data(), &rho_sel, nullptr);
   if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
   ctx->rho = rho > 0.0 ? rho : rho_sel;
   return NETMAX_OK;
@@ -316,7 +349,12 @@ struct RoundPlan {
 
 using RoundKernel = void (*)(const RoundParams);
 
+using StepKernel = void (*)(const StepParams);
+
+StepKernel pick_step_kernel(int objective) { return objective == 1 ? step_kernel<1, true> : step_kernel<0, true>; }
+
 RoundKernel pick_kernel(int objective, bool short_vectors) {
+  if (objective == 2) return short_vectors ? round_kernel<2, true, 4> : round_kernel<2, true, 1>;
   if (short_vectors) return objective == 1 ? round_kernel<1, true, 4> : round_kernel<0, true, 4>;
   return objective == 1 ? round_kernel<1, true, 1> : round_kernel<0, true, 1>;
 }
@@ -512,6 +550,7 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   ctx->colpart = (float4*)(ctx->base + L.off_colpart);
   ctx->grid_barrier = ctx->ticket + 16;
   ctx->dev_error = ctx->ticket + 32;
+  ctx->measure_out = (double*)(ctx->ticket + 48);
   ctx->coltick = (unsigned int*)(ctx->base + L.off_coltick);
 
   auto step = [&](cudaError_t e, const char* what) {
@@ -567,7 +606,7 @@ int netmax_set_policy(netmax_ctx* ctx, const double* link_speed_gbps, const doub
   if (!std::isfinite(rho)) return fail(ctx, NETMAX_INVALID_ARG, "rho is not finite");
   DeviceGuard guard(ctx->device);
   std::vector<uint8_t> old_adj = ctx->adj;
-  std::vector<double> old_P = ctx->P;
+  std::vector<double> old_P = ctx->P, old_t = ctx->t_iter;
   const double old_rho = ctx->rho;
   int rc = NETMAX_OK;
   if (link_speed_gbps) rc = build_adjacency(ctx, ctx->M, link_speed_gbps, ctx->adj);
@@ -575,6 +614,7 @@ int netmax_set_policy(netmax_ctx* ctx, const double* link_speed_gbps, const doub
   if (rc) {  // leave the policy in force untouched
     ctx->adj.swap(old_adj);
     ctx->P.swap(old_P);
+    ctx->t_iter.swap(old_t);
     ctx->rho = old_rho;
     return rc;
   }
@@ -626,6 +666,7 @@ int netmax_read_centres(netmax_ctx* ctx, float* host_out) { return copy_out(ctx,
 int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
   if (n_rounds < 0) return fail(ctx, NETMAX_INVALID_ARG, "n_rounds = %lld < 0", (long long)n_rounds);
+  if (ctx->async_on) return fail(ctx, NETMAX_INVALID_ARG, "the context runs the asynchronous timeline; use netmax_async_steps");
   if (n_rounds == 0) return NETMAX_OK;
   if ((uint64_t)(ctx->rounds + n_rounds) >= ((uint64_t)1 << 56)) return fail(ctx, NETMAX_INVALID_ARG, "round counter would exceed 2^56");
   DeviceGuard guard(ctx->device);
@@ -864,6 +905,226 @@ int netmax_sample_peers(netmax_ctx* ctx, int64_t first_round, int64_t n_rounds, 
   if (first_round < 0 || n_rounds < 0 || (n_rounds > 0 && !device_out)) return fail(ctx, NETMAX_INVALID_ARG, "bad range or NULL output");
   DeviceGuard guard(ctx->device);
   return launch_sampler(ctx, (uint64_t)first_round, n_rounds, device_out, 0, INT64_MAX);
+}
+
+// ---- telemetry on demand --------------------------------------------------------------------
+int netmax_measure(netmax_ctx* ctx, double* consensus, double* loss) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  DeviceGuard guard(ctx->device);
+  const int saved = ctx->objective;
+  ctx->objective = 2;  // plan and pick the measuring instantiation
+  RoundPlan plan;
+  int rc = plan_round(ctx, plan);
+  RoundKernel kernel = pick_kernel(2, plan.short_vectors);
+  ctx->objective = saved;
+  if (rc) return rc;
+  RoundParams p;
+  std::memset(&p, 0, sizeof p);
+  p.x_cur = reinterpret_cast<const float4*>(ctx->x[ctx->cur]);
+  p.x_nxt = nullptr;
+  p.c = reinterpret_cast<const float4*>(ctx->c);
+  p.peers = nullptr;
+  p.wtab = ctx->wtab;
+  p.partials = ctx->partials;
+  p.ticket = ctx->ticket;
+  p.tel_out = ctx->measure_out;
+  p.ldq = ctx->L.ldq;
+  p.row_bytes = (uint32_t)(ctx->L.ld * sizeof(float));
+  p.nq = ctx->L.nq;
+  p.n_tiles = plan.n_tiles;
+  p.M = ctx->M;
+  p.tail = (int32_t)(ctx->d % 4);
+  p.cg = plan.cg;
+  p.rl = plan.rl;
+  p.rg = plan.rg;
+  p.rows_per_group = plan.rows_per_group;
+  p.colpart = ctx->colpart;
+  p.coltick = ctx->coltick;
+  p.inv_M = 1.0f / (float)ctx->M;
+  p.keys = ctx->keys;
+  kernel<<<plan.grid, kThreads, plan.smem, ctx->stream>>>(p);
+  ctx->launches += 1;
+  NM_CUDA(ctx, cudaGetLastError());
+  double out[2] = {0.0, 0.0};
+  NM_CUDA(ctx, cudaMemcpyAsync(out, ctx->measure_out, sizeof out, cudaMemcpyDeviceToHost, ctx->stream));
+  NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  if (consensus) *consensus = out[0];
+  if (loss) *loss = out[1];
+  return check_device_error(ctx);
+}
+
+// ---- asynchronous timeline --------------------------------------------------------------------
+// First word of the Philox block of the peer stream at counter (0, worker, iteration): the host
+// twin of the device sampler (same published algorithm, 32x32->64 products and xors).
+static uint32_t host_peer_word(const PhiloxKeys& keys, uint32_t worker, uint64_t iter) {
+  uint32_t c0 = 0, c1 = worker, c2 = (uint32_t)iter, c3 = philox_ctr3(kTagPeer, iter);
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = (uint64_t)kPhiloxMul0 * c0, p1 = (uint64_t)kPhiloxMul1 * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ keys.k0[r];
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ keys.k1[r];
+    c0 = n0;
+    c1 = (uint32_t)p1;
+    c2 = n2;
+    c3 = (uint32_t)p0;
+  }
+  return c0;
+}
+
+// Draws the peer of worker i's next local iteration (Algorithm 2) and sets when it will finish.
+static void async_start_iteration(netmax_ctx* ctx, int i, double start) {
+  const int32_t M = ctx->M;
+  const uint32_t u = host_peer_word(ctx->keys, (uint32_t)i, (uint64_t)ctx->local_n[i]);
+  const uint32_t* row = ctx->h_thr.data() + (size_t)i * M;
+  const int32_t count = (int32_t)(std::upper_bound(row, row + M, u) - row);  // #{j : T[j] <= u}
+  const int32_t m = std::min(count, ctx->h_last[i]);
+  ctx->pending_peer[i] = m;
+  ctx->finish[i] = start + ctx->t_iter[(size_t)i * M + m];
+}
+
+int netmax_async_begin(netmax_ctx* ctx, const double* t_iter, double beta) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (ctx->rounds != 0) return fail(ctx, NETMAX_INVALID_ARG, "netmax_async_begin must precede any netmax_round");
+  if (!(beta >= 0.0 && beta < 1.0)) return fail(ctx, NETMAX_INVALID_ARG, "beta = %g outside [0, 1)", beta);
+  const int32_t M = ctx->M;
+  if (t_iter) {
+    for (size_t k = 0; k < (size_t)M * M; ++k) {
+      const int i = (int)(k / M), m = (int)(k % M);
+      const bool used = (i == m) || ctx->adj[k];
+      if (used && !(t_iter[k] > 0.0 && std::isfinite(t_iter[k])))
+        return fail(ctx, NETMAX_INVALID_ARG, "t_iter[%d,%d] = %g must be positive and finite", i, m, t_iter[k]);
+    }
+    ctx->t_iter.assign(t_iter, t_iter + (size_t)M * M);
+  }
+  ctx->async_on = true;
+  ctx->beta = beta;
+  ctx->now = 0.0;
+  ctx->steps = 0;
+  ctx->local_n.assign(M, 0);
+  ctx->pending_peer.assign(M, 0);
+  ctx->finish.assign(M, 0.0);
+  ctx->ema.assign((size_t)M * M, 0.0);
+  ctx->ema_count.assign((size_t)M * M, 0);
+  ctx->ev_cap = std::max<int64_t>(ctx->trace_rounds * (int64_t)M, 1024);
+  ctx->ev_worker.assign(ctx->ev_cap, 0);
+  ctx->ev_peer.assign(ctx->ev_cap, 0);
+  ctx->ev_n.assign(ctx->ev_cap, 0);
+  ctx->ev_time.assign(ctx->ev_cap, 0.0);
+  for (int i = 0; i < M; ++i) async_start_iteration(ctx, i, 0.0);
+  return NETMAX_OK;
+}
+
+int netmax_async_set_times(netmax_ctx* ctx, const double* t_iter) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (!t_iter) return fail(ctx, NETMAX_INVALID_ARG, "t_iter is NULL");
+  ctx->t_iter.assign(t_iter, t_iter + (size_t)ctx->M * ctx->M);
+  return NETMAX_OK;
+}
+
+int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (!ctx->async_on) return fail(ctx, NETMAX_INVALID_ARG, "call netmax_async_begin first");
+  if (n_steps < 0) return fail(ctx, NETMAX_INVALID_ARG, "n_steps = %lld < 0", (long long)n_steps);
+  DeviceGuard guard(ctx->device);
+  const int32_t M = ctx->M;
+  StepKernel kernel = pick_step_kernel(ctx->objective);
+  StepParams p;
+  p.x = reinterpret_cast<float4*>(ctx->x[ctx->cur]);
+  p.c = reinterpret_cast<const float4*>(ctx->c);
+  p.nq = ctx->L.nq;
+  p.row_bytes = (uint32_t)(ctx->L.ld * sizeof(float));
+  p.tail = (int32_t)(ctx->d % 4);
+  p.alpha = (float)ctx->alpha;
+  p.sigma = (float)ctx->sigma;
+  p.q_offset = ctx->q_offset;
+  p.n_events = 0;
+  p.keys = ctx->keys;
+  std::vector<uint8_t> writes(M, 0), reads(M, 0);
+  auto flush = [&]() -> int {
+    if (p.n_events == 0) return NETMAX_OK;
+    const int64_t want = (ctx->L.nq + kThreads - 1) / kThreads;
+    const int64_t cap = std::max<int64_t>(1, (int64_t)8 * ctx->sm_count / p.n_events);
+    dim3 grid((unsigned)std::min<int64_t>(want, cap), (unsigned)p.n_events);
+    kernel<<<grid, kThreads, 0, ctx->stream>>>(p);
+    ctx->launches += 1;
+    NM_CUDA(ctx, cudaGetLastError());
+    for (int e = 0; e < p.n_events; ++e) {
+      writes[p.ev[e].worker] = 0;
+      reads[p.ev[e].worker] = 0;
+      reads[p.ev[e].peer] = 0;
+    }
+    p.n_events = 0;
+    return NETMAX_OK;
+  };
+  for (int64_t k = 0; k < n_steps; ++k) {
+    // the next global step: the worker whose iteration finishes first (ties: lowest index)
+    int i = 0;
+    for (int j = 1; j < M; ++j)
+      if (ctx->finish[j] < ctx->finish[i]) i = j;
+    const int m = ctx->pending_peer[i];
+    // a launch holds steps on disjoint replicas only: this one must not write a row that an
+    // earlier step of the launch reads or writes, nor read a row that one writes
+    if (p.n_events == kMaxStepEvents || writes[i] || reads[i] || writes[m]) {
+      int rc = flush();
+      if (rc) return rc;
+    }
+    const uint64_t n = (uint64_t)ctx->local_n[i];
+    StepEvent& e = p.ev[p.n_events++];
+    e.worker = i;
+    e.peer = m;
+    e.iter_lo = (uint32_t)n;
+    e.ctr3 = philox_ctr3(kTagNoise, n);
+    e.w = (m == i) ? 0.0f : ctx->h_w[(size_t)i * M + m];
+    writes[i] = 1;
+    reads[i] = 1;
+    reads[m] = 1;
+    // bookkeeping of Algorithm 2: the clock, the EMA of the iteration time, the next iteration
+    ctx->now = ctx->finish[i];
+    const int64_t slot = ctx->steps % ctx->ev_cap;
+    ctx->ev_worker[slot] = i;
+    ctx->ev_peer[slot] = m;
+    ctx->ev_n[slot] = (int64_t)n;
+    ctx->ev_time[slot] = ctx->now;
+    const size_t at = (size_t)i * M + m;
+    ctx->ema[at] = ctx->beta * ctx->ema[at] + (1.0 - ctx->beta) * ctx->t_iter[at];
+    ctx->ema_count[at] += 1;
+    ctx->local_n[i] += 1;
+    ctx->steps += 1;
+    async_start_iteration(ctx, i, ctx->now);
+  }
+  return flush();
+}
+
+int netmax_async_time(netmax_ctx* ctx, double* sim_time, int64_t* steps_done) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (!ctx->async_on) return fail(ctx, NETMAX_INVALID_ARG, "call netmax_async_begin first");
+  if (sim_time) *sim_time = ctx->now;
+  if (steps_done) *steps_done = ctx->steps;
+  return NETMAX_OK;
+}
+
+int netmax_async_trace(netmax_ctx* ctx, int64_t first_step, int64_t n, int32_t* worker, int32_t* peer, int64_t* local_iter,
+                       double* finish_time) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (!ctx->async_on) return fail(ctx, NETMAX_INVALID_ARG, "call netmax_async_begin first");
+  if (first_step < 0 || n < 0 || first_step + n > ctx->steps || first_step < ctx->steps - ctx->ev_cap)
+    return fail(ctx, NETMAX_TRACE_RANGE, "steps [%lld, %lld) are not in the ring (steps done %lld, capacity %lld)",
+                (long long)first_step, (long long)(first_step + n), (long long)ctx->steps, (long long)ctx->ev_cap);
+  for (int64_t k = 0; k < n; ++k) {
+    const int64_t slot = (first_step + k) % ctx->ev_cap;
+    if (worker) worker[k] = ctx->ev_worker[slot];
+    if (peer) peer[k] = ctx->ev_peer[slot];
+    if (local_iter) local_iter[k] = ctx->ev_n[slot];
+    if (finish_time) finish_time[k] = ctx->ev_time[slot];
+  }
+  return NETMAX_OK;
+}
+
+int netmax_async_ema(netmax_ctx* ctx, double* ema_out, int64_t* samples_out) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (!ctx->async_on) return fail(ctx, NETMAX_INVALID_ARG, "call netmax_async_begin first");
+  if (ema_out) std::memcpy(ema_out, ctx->ema.data(), ctx->ema.size() * sizeof(double));
+  if (samples_out) std::memcpy(samples_out, ctx->ema_count.data(), ctx->ema_count.size() * sizeof(int64_t));
+  return NETMAX_OK;
 }
 
 int64_t netmax_kernel_launches(const netmax_ctx* ctx) { return ctx ? ctx->launches : -1; }

@@ -85,20 +85,24 @@ struct RowAcc {
 // Eq. 15 and Eq. 16 on one column group of one worker, on packed fp32 pairs:
 //   g = (x - c) + sigma z,  h = x - alpha g                                       (Eq. 15)
 //   x' = h - w (h - x_m),   w = alpha rho gamma_im  (w = 0 on a self-draw)          (Eq. 16)
-// q32 is the global column-group index (first Philox counter word), tail > 0 marks the ragged
-// last group of a row whose padding lanes must stay zero.
+// q32 is the global column-group index (first Philox counter word), iter_lo / ctr3 carry the
+// round (or, on the asynchronous timeline, the worker's local iteration); `ragged` marks the
+// last group of a row whose padding lanes (beyond `tail` live ones) must stay zero.  ta, tb
+// return x - c for the caller's loss statistic.
 template <int kObjective, bool kFastNoise>
-__device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t round_lo, uint32_t ctr3, uint32_t q32,
-                                                 uint32_t worker, ulonglong2 xv, ulonglong2 cv, ulonglong2 xm,
-                                                 ulonglong2 pivot, float w, bool ragged, RowAcc& acc) {
+__device__ __forceinline__ ulonglong2 update_core(float alpha, float sigma, int32_t tail, const PhiloxKeys& keys,
+                                                  uint32_t iter_lo, uint32_t ctr3, uint32_t q32, uint32_t worker,
+                                                  ulonglong2 xv, ulonglong2 cv, ulonglong2 xm, float w, bool ragged,
+                                                  pair_t& ta, pair_t& tb) {
   const pair_t neg1 = pack2(-1.0f, -1.0f);
   const pair_t nw2 = pack2(-w, -w);
-  const pair_t ta = fma2(cv.x, neg1, xv.x), tb = fma2(cv.y, neg1, xv.y);  // x - c
+  ta = fma2(cv.x, neg1, xv.x);  // x - c
+  tb = fma2(cv.y, neg1, xv.y);
   pair_t ha = xv.x, hb = xv.y;
   if (kObjective == 1) {
-    const pair_t sig2 = pack2(p.sigma, p.sigma);
-    const pair_t nalpha2 = pack2(-p.alpha, -p.alpha);
-    const uint4 rnd = philox4x32_10(q32, worker, round_lo, ctr3, p.keys);
+    const pair_t sig2 = pack2(sigma, sigma);
+    const pair_t nalpha2 = pack2(-alpha, -alpha);
+    const uint4 rnd = philox4x32_10(q32, worker, iter_lo, ctr3, keys);
     pair_t za, zb;
     if (kFastNoise) {
       za = normal_pair_fast_packed(rnd.x, rnd.y);
@@ -117,10 +121,28 @@ __device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t 
     float o0, o1, o2, o3;
     unpack2(oa, o0, o1);
     unpack2(ob, o2, o3);
-    if (p.tail < 2) o1 = 0.f;
-    if (p.tail < 3) o2 = 0.f;
+    if (tail < 2) o1 = 0.f;
+    if (tail < 3) o2 = 0.f;
     oa = pack2(o0, o1);
     ob = pack2(o2, 0.f);
+  }
+  return make_ulonglong2(oa, ob);
+}
+
+// update_core plus the telemetry sums of the round-start values.  kObjective == 2 measures only.
+template <int kObjective, bool kFastNoise>
+__device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t round_lo, uint32_t ctr3, uint32_t q32,
+                                                 uint32_t worker, ulonglong2 xv, ulonglong2 cv, ulonglong2 xm,
+                                                 ulonglong2 pivot, float w, bool ragged, RowAcc& acc) {
+  const pair_t neg1 = pack2(-1.0f, -1.0f);
+  pair_t ta, tb;
+  ulonglong2 o = xv;
+  if (kObjective == 2) {
+    ta = fma2(cv.x, neg1, xv.x);
+    tb = fma2(cv.y, neg1, xv.y);
+  } else {
+    o = update_core<kObjective, kFastNoise>(p.alpha, p.sigma, p.tail, p.keys, round_lo, ctr3, q32, worker, xv, cv, xm, w,
+                                            ragged, ta, tb);
   }
   const pair_t da = fma2(pivot.x, neg1, xv.x), db = fma2(pivot.y, neg1, xv.y);  // x - pivot
   acc.s1a = add2(acc.s1a, da);
@@ -129,7 +151,7 @@ __device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t 
   acc.s2b = fma2(db, db, acc.s2b);
   acc.la = fma2(ta, ta, acc.la);
   acc.lb = fma2(tb, tb, acc.lb);
-  return make_ulonglong2(oa, ob);
+  return o;
 }
 
 // Block reduction of a CTA's two telemetry sums into partials[2 * blockIdx.x ..].
@@ -251,7 +273,7 @@ __device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* 
   const int rli = tid / p.cg;
   const int M = p.M;
   const int step = p.rl;
-  if (G == 1) {
+  if (G == 1 && kObjective != 2) {
     __syncthreads();  // readers of the previous round's draws are done
     load_draws(p, peers, s_pw, 0, M);
     __syncthreads();
@@ -261,7 +283,7 @@ __device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* 
     const int64_t ct = G == 1 ? tile : tile / G;      // column tile
     const int grp = G == 1 ? 0 : (int)(tile - ct * G);  // row group
     const int r0 = grp * p.rows_per_group, r1 = min(M, r0 + p.rows_per_group);
-    if (G > 1) {
+    if (G > 1 && kObjective != 2) {
       __syncthreads();  // the previous tile's readers of s_pw are done
       load_draws(p, peers, s_pw, r0, r1);
       __syncthreads();
@@ -286,10 +308,15 @@ __device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* 
         for (int u = 0; u < kRowsInFlight; ++u) {  // issue the loads of kRowsInFlight rows
           const int i = i0 + u * step;
           if (kRowsInFlight == 1 || i < r1) {
-            pw[u] = s_pw[i];
             const uint64_t row = (uint64_t)(uint32_t)i * p.row_bytes;
             xv[u] = ld_x<kCoherent>(xq + row);
-            xm[u] = ld_x<kCoherent>(xq + (uint64_t)(uint32_t)pw[u].x * p.row_bytes);
+            if (kObjective == 2) {  // measuring: no peers involved
+              pw[u] = make_int2(i, 0);
+              xm[u] = xv[u];
+            } else {
+              pw[u] = s_pw[i];
+              xm[u] = ld_x<kCoherent>(xq + (uint64_t)(uint32_t)pw[u].x * p.row_bytes);
+            }
             cv[u] = __ldg(reinterpret_cast<const ulonglong2*>(cq + row));
           }
         }
@@ -299,7 +326,7 @@ __device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* 
           if (kRowsInFlight == 1 || i < r1) {
             const ulonglong2 o = row_update<kObjective, kFastNoise>(p, round_lo, ctr3, q32, (uint32_t)i, xv[u], cv[u],
                                                                     xm[u], pivot, __int_as_float(pw[u].y), ragged, acc);
-            *reinterpret_cast<ulonglong2*>(oq + (uint64_t)(uint32_t)i * p.row_bytes) = o;
+            if (kObjective != 2) *reinterpret_cast<ulonglong2*>(oq + (uint64_t)(uint32_t)i * p.row_bytes) = o;
           }
         }
       }
@@ -455,6 +482,54 @@ __global__ void __launch_bounds__(256, 2) multi_round_kernel(const MultiRoundPar
     const float4* t = x_cur;
     x_cur = x_nxt;
     x_nxt = const_cast<float4*>(t);
+  }
+}
+
+// ------------------------------------------------------------------------- asynchronous steps
+// The paper's own process (Eq. 17): at a global step ONE worker i applies Eq. 15-16 to its
+// replica, in place, with the peer's current replica; every other replica is unchanged.  A
+// launch carries up to kMaxStepEvents consecutive global steps that touch disjoint replicas
+// (no step writes a row another step of the launch reads or writes), so their order inside
+// the launch does not matter.  16 bytes of HBM traffic per element: nothing is shared.
+constexpr int kMaxStepEvents = 32;
+
+struct StepEvent {
+  int32_t worker, peer;
+  uint32_t iter_lo, ctr3;  // the worker's local iteration, as Philox counter words of the noise stream
+  float w;                 // pull weight w_im (0 on a self-draw)
+};
+
+struct StepParams {
+  float4* x;        // [M][ldq] replicas, updated in place
+  const float4* c;  // [M][ldq]
+  int64_t nq;
+  uint32_t row_bytes;
+  int32_t tail;
+  float alpha, sigma;
+  uint32_t q_offset;
+  int32_t n_events;
+  StepEvent ev[kMaxStepEvents];
+  PhiloxKeys keys;
+};
+
+template <int kObjective, bool kFastNoise>
+__global__ void __launch_bounds__(256) step_kernel(const StepParams p) {
+  const StepEvent& e = p.ev[blockIdx.y];
+  const uint64_t row_i = (uint64_t)(uint32_t)e.worker * p.row_bytes;
+  const uint64_t row_m = (uint64_t)(uint32_t)e.peer * p.row_bytes;
+  char* xb = reinterpret_cast<char*>(p.x);
+  const char* cb = reinterpret_cast<const char*>(p.c);
+  for (int64_t q = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; q < p.nq; q += (int64_t)gridDim.x * blockDim.x) {
+    const uint64_t off = (uint64_t)q * 16;
+    const ulonglong2 xv = *reinterpret_cast<const ulonglong2*>(xb + row_i + off);
+    const ulonglong2 xm = *reinterpret_cast<const ulonglong2*>(xb + row_m + off);
+    ulonglong2 cv = make_ulonglong2(0ull, 0ull);
+    if (kObjective == 1) cv = __ldg(reinterpret_cast<const ulonglong2*>(cb + row_i + off));
+    pair_t ta, tb;
+    const ulonglong2 o = update_core<kObjective, kFastNoise>(p.alpha, p.sigma, p.tail, p.keys, e.iter_lo, e.ctr3,
+                                                             (uint32_t)q + p.q_offset, (uint32_t)e.worker, xv, cv, xm, e.w,
+                                                             (p.tail != 0) && (q == p.nq - 1), ta, tb);
+    *reinterpret_cast<ulonglong2*>(xb + row_i + off) = o;
   }
 }
 

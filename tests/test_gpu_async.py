@@ -1,0 +1,163 @@
+"""GPU parity of the asynchronous timeline (one worker per global step, Eq. 17) and of the
+on-demand telemetry, against the CPU oracle: event traces (worker, peer, local iteration,
+finish time) bit-exact, replicas within 1e-5 (1 + |x|)."""
+import numpy as np
+import pytest
+
+from oracle import oracle
+from oracle import policy as opolicy
+from paper_2009_05766_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def nm():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    from paper_2009_05766_b200 import binding
+    binding.lib()
+    return binding
+
+
+def full_adj(M):
+    return (1 - np.eye(M)).astype(np.uint8)
+
+
+def close(got, want, tol=TOL):
+    got64, want64 = got.astype(np.float64), want.astype(np.float64)
+    excess = np.abs(got64 - want64) - tol * (1.0 + np.abs(want64))
+    assert excess.max() <= 0.0, f"max excess {excess.max():.3e}"
+
+
+def random_policy(M, rng, self_prob=True):
+    P = rng.random((M, M)) + 0.05
+    if not self_prob:
+        np.fill_diagonal(P, 0.0)
+    return P / P.sum(axis=1, keepdims=True)
+
+
+def random_times(M, rng):
+    t = rng.uniform(1.0, 4.0, (M, M))
+    t = 0.5 * (t + t.T)
+    t[np.diag_indices(M)] = 0.2
+    return t
+
+
+@pytest.mark.parametrize("objective", [0, 1])
+@pytest.mark.parametrize("M,d", [(2, 5), (3, 1), (5, 67), (8, 4099), (16, 3001), (64, 515), (300, 37)])
+def test_async_steps_match_oracle(nm, M, d, objective):
+    rng = np.random.default_rng(M * 13 + d)
+    P, t = random_policy(M, rng), random_times(M, rng)
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=objective, seed=d + 3)
+    rho = g.get_policy()[1]
+    o = oracle.Sim(M, d, P, full_adj(M), alpha=0.05, rho=rho, sigma=0.1, objective=objective, seed=d + 3)
+    o.init(1.0, 1.0)
+    g.async_begin(t, beta=0.7)
+    o.async_begin(t, beta=0.7)
+    steps = 12 * M
+    for n in (1, 0, steps // 3, steps - 1 - steps // 3):
+        g.async_steps(n)
+        o.async_steps(n)
+    gw, gp, gn, gt = g.async_trace()
+    ow, op, on, ot = o.async_trace()
+    assert (gw == ow).all() and (gp == op).all() and (gn == on).all() and (gt == ot).all()
+    close(g.read_replicas(), o.x(), tol=2e-5 if objective == 0 else TOL)
+    assert g.async_time() == (o.async_now, steps)
+    ge, gc = g.async_ema()
+    oe, oc = o.async_ema()
+    assert (gc == oc).all() and (ge == oe).all()
+    # on-demand telemetry against the oracle's definition on its own state
+    cons, loss = g.measure()
+    ocons, oloss = o.telemetry_now()
+    assert cons == pytest.approx(ocons, rel=1e-4) and loss == pytest.approx(oloss, rel=1e-4)
+    with pytest.raises(nm.NetmaxError):
+        g.round(1)
+    g.close()
+
+
+def test_async_policy_and_time_changes_apply_to_later_iterations(nm):
+    rng = np.random.default_rng(5)
+    M, d = 6, 500
+    P1, P2 = random_policy(M, rng, self_prob=False), random_policy(M, rng)
+    t1, t2 = random_times(M, rng), random_times(M, rng)
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=P1, sigma=0.05, x0_std=1.0, c_std=1.0, seed=8)
+    o = oracle.Sim(M, d, P1, full_adj(M), alpha=0.05, rho=g.get_policy()[1], sigma=0.05, objective=1, seed=8)
+    o.init(1.0, 1.0)
+    g.async_begin(t1, 0.5)
+    o.async_begin(t1, 0.5)
+    g.async_steps(40)
+    o.async_steps(40)
+    g.set_policy(prob=P2)
+    o.set_policy(P2, full_adj(M), g.get_policy()[1])
+    g.async_set_times(t2)
+    o.async_set_times(t2)
+    g.async_steps(60)
+    o.async_steps(60)
+    for a, b in zip(g.async_trace(), o.async_trace()):
+        assert (a == b).all()
+    close(g.read_replicas(), o.x())
+    g.close()
+
+
+def test_async_needs_begin_and_a_fresh_context(nm):
+    M, d = 3, 10
+    P = random_policy(M, np.random.default_rng(1))
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, x0_std=1.0, c_std=1.0, seed=1)
+    with pytest.raises(nm.NetmaxError):
+        g.async_steps(1)
+    g.round(1)
+    with pytest.raises(nm.NetmaxError):
+        g.async_begin(None, 0.5)
+    h = nm.Netmax(M=M, d=d, lr=0.05, prob=P, x0_std=1.0, c_std=1.0, seed=1, trace_rounds=4)
+    with pytest.raises(nm.NetmaxError):
+        h.async_begin(None, 1.0)
+    h.async_begin(None, 0.5)                      # iteration times from (equal) link speeds
+    h.async_steps(2000)
+    assert h.async_time()[1] == 2000
+    w, p, n, t = h.async_trace(2000 - 1024, 1024)
+    assert (np.diff(t) >= 0).all()
+    with pytest.raises(nm.NetmaxError) as e:
+        h.async_trace(0, 10)
+    assert e.value.code == -5
+    g.close()
+    h.close()
+
+
+def test_measure_matches_round_telemetry(nm):
+    M, d = 7, 12345
+    P = random_policy(M, np.random.default_rng(2))
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, seed=2)
+    g.round(5)
+    cons, loss = g.measure()
+    before = g.read_replicas()
+    g.round(1)
+    tc, tl = g.telemetry(5, 1)                   # the round's telemetry is taken on its start state
+    assert cons == pytest.approx(tc[0], rel=1e-6) and loss == pytest.approx(tl[0], rel=1e-6)
+    h = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, seed=2)
+    h.round(5)
+    assert (h.read_replicas() == before).all()   # measuring changed nothing
+    g.close()
+    h.close()
+
+
+def test_async_full_size_resnet18_vectors_on_sampled_columns(nm):
+    w = workloads.config(2)
+    t, adj = opolicy.iteration_times(w.link_speeds(0), w.d)
+    P, rho, _ = opolicy.generate_policy(t, adj, w.lr, 6, 6)
+    cols = workloads.sample_columns(w.d, 2000, w.seed)
+    g = nm.Netmax(M=w.M, d=w.d, lr=w.lr, link_speed_gbps=w.link_speeds(0), prob=P, rho=rho, sigma=w.sigma,
+                  x0_std=w.x0_std, c_std=w.c_std, seed=w.seed)
+    o = oracle.Sim(w.M, w.d, P, adj, alpha=w.lr, rho=rho, sigma=w.sigma, objective=1, seed=w.seed, cols=cols)
+    o.init(w.x0_std, w.c_std)
+    g.async_begin(None, 0.9)                      # the library's own iteration times from the link speeds
+    o.async_begin(t, 0.9)
+    steps = 40 * w.M
+    g.async_steps(steps)
+    o.async_steps(steps)
+    for a, b in zip(g.async_trace(), o.async_trace()):
+        assert (a == b).all()
+    close(g.read_columns(cols), o.x())
+    g.close()
