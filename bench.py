@@ -356,6 +356,58 @@ def run_ours(args, w):
         print(json.dumps(line), flush=True)
 
 
+def run_async(args, w):
+    """The asynchronous timeline (one worker per global step, Eq. 17): a step is one global step,
+    i.e. one replica of d elements updated in place from its peer (16 bytes of HBM per element)."""
+    import torch
+    from paper_2009_05766_b200 import binding
+    if int(os.environ.get("WORLD_SIZE", "1")) != 1 or args.gpus != 1:
+        raise SystemExit("--mode async runs on one GPU")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    binding.lib()
+    speeds = w.link_speeds(0)
+    t_iter, adj = binding.netmax_iteration_times(speeds, w.d)
+    P, rho, _ = binding.netmax_policy_generate(t_iter, adj, w.lr, w.K, w.R)
+    stream = torch.cuda.Stream()
+    g = binding.Netmax(M=w.M, d=w.d, lr=w.lr, link_speed_gbps=speeds, prob=P, rho=rho, sigma=w.sigma,
+                       x0_std=w.x0_std, c_std=w.c_std, objective=1, seed=w.seed, stream=stream.cuda_stream)
+    g.async_begin(None, 0.9)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g.async_steps(max(args.warmup, 3) * w.M)
+    torch.cuda.synchronize()
+    launches0 = g.kernel_launches
+    with ClockSampler(0) as clocks:
+        with torch.cuda.stream(stream):
+            start.record()
+        g.async_steps(args.steps)
+        with torch.cuda.stream(stream):
+            stop.record()
+        stop.synchronize()
+    ms = start.elapsed_time(stop)
+    launches = g.kernel_launches - launches0
+    sim_time, steps_done = g.async_time()
+    cons, loss = g.measure()
+    peak, peak_kind = measured_peak()
+    achieved = BYTES_PER_ELEMENT * w.d * args.steps / (ms / 1e3) / 1e9
+    line = {
+        "metric": "replica GB/s", "value": achieved, "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3) * w.M, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name + ", asynchronous timeline (one worker per global step)", "M": w.M, "d": w.d,
+                   "l2": "each replica is %.0f MB; a step touches three of them" % (w.d * 4 / 1e6)},
+        "global_steps_per_s": args.steps / (ms / 1e3), "steps_per_launch": args.steps / max(launches, 1),
+        "simulated_seconds": sim_time,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "step_kernel",
+                     "bytes_per_launch": BYTES_PER_ELEMENT * w.d * args.steps / max(launches, 1)},
+        "gpu_launches": int(launches), "clocks": clocks.summary(),
+        "telemetry_now": {"consensus": cons, "loss": loss},
+    }
+    g.close()
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -366,6 +418,8 @@ def main():
     ap.add_argument("--d", type=int, default=0, help="override the workload's vector length (profiling on a smaller case)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", choices=["rounds", "async"], default="rounds",
+                    help="rounds: synchronous rounds (default); async: the paper's one-worker-per-step timeline")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -374,6 +428,8 @@ def main():
         w = w.scaled(d=args.d)
     if args.impl == "reference":
         run_reference(args, w)
+    elif args.mode == "async":
+        run_async(args, w)
     else:
         run_ours(args, w)
 
