@@ -68,6 +68,11 @@ typedef struct netmax_config {
   double rho;                    /* rho; <= 0: with prob given, the largest rho meeting Eq. 11 with a
                                     1e-6 margin, min_{p_im>0} p_im / (alpha (d_im+d_mi)); with prob
                                     NULL, the rho Algorithm 3 selects                                  */
+  double pull_weight;            /* 0 (default): Eq. 16's weight alpha rho (d_im+d_mi)/(2 p_im).  In (0, 1):
+                                    every pull uses this constant instead -- the update rule of gossip /
+                                    AD-PSGD style averaging (1/2), which the paper's section on extending
+                                    existing decentralised PSGD approaches writes in the same form
+                                    x <- D (x - alpha g); rho is then unused                             */
   double sigma;                  /* std of the gradient noise; the update uses its fp32 rounding       */
   double x0_std, c_std;          /* x_i(0) ~ N(0, x0_std^2), c_i ~ N(0, c_std^2), drawn from the seed  */
   int32_t objective;             /* 0: zero gradients (sigma ignored); 1: f_i = 1/2 ||x - c_i||^2      */

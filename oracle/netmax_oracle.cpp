@@ -132,11 +132,19 @@ inline int32_t sample_row(const uint32_t* T, int M, int32_t last_nz, uint32_t u)
 // Pull weight  w_im = alpha * rho * gamma_im = alpha*rho*(d_im + d_mi) / (2 p_im),
 // computed in double and rounded to fp32 (the precision the replicas are updated in).
 // Entries with p_im = 0 or m = i are 0 (never used: a self-draw skips the pull).
-void build_weight_row(int M, int i, const double* P, const uint8_t* adj, double alpha, double rho, float* w) {
+// fixed_w > 0 replaces it by one constant for every pull: the update rule of gossip / AD-PSGD
+// style averaging (fixed_w = 1/2), which the paper's Section "Extension to existing
+// decentralized PSGD approaches" puts in the same form x <- D(x - alpha g).
+void build_weight_row(int M, int i, const double* P, const uint8_t* adj, double alpha, double rho, float* w,
+                      double fixed_w = 0.0) {
   for (int m = 0; m < M; ++m) {
     const double p = P[(size_t)i * M + m];
     if (m == i || !(p > 0.0)) {
       w[m] = 0.0f;
+      continue;
+    }
+    if (fixed_w > 0.0) {
+      w[m] = (float)fixed_w;
       continue;
     }
     const double dsum = (double)adj[(size_t)i * M + m] + (double)adj[(size_t)m * M + i];
@@ -151,6 +159,7 @@ struct Sim {
   int64_t ncols = 0;       // number of simulated columns (== d, or a sample of them)
   std::vector<int64_t> cols;  // logical element index of each simulated column
   double alpha = 0, rho = 0, sigma = 0;  // alpha, sigma already rounded to fp32 values
+  double fixed_w = 0.0;                  // > 0: every pull uses this weight instead of Eq. 16's
   int objective = 1;
   uint32_t key[2] = {0, 0};
   uint64_t round = 0;
@@ -183,7 +192,7 @@ void sim_set_policy(Sim* s, const double* P, const uint8_t* adj, double rho) {
   s->w.assign((size_t)M * M, 0.0f);
   for (int i = 0; i < M; ++i) {
     build_threshold_row(M, P + (size_t)i * M, s->T.data() + (size_t)i * M, &s->last_nz[i]);
-    build_weight_row(M, i, P, adj, s->alpha, rho, s->w.data() + (size_t)i * M);
+    build_weight_row(M, i, P, adj, s->alpha, rho, s->w.data() + (size_t)i * M, s->fixed_w);
   }
 }
 
@@ -423,6 +432,8 @@ void* nmo_sim_create(int32_t M, int64_t d, const int64_t* cols, int64_t ncols, c
 }
 
 void nmo_sim_destroy(void* h) { delete (Sim*)h; }
+// Takes effect at the next nmo_sim_set_policy.
+void nmo_sim_set_fixed_weight(void* h, double fixed_w) { ((Sim*)h)->fixed_w = fixed_w; }
 void nmo_sim_set_policy(void* h, const double* P, const uint8_t* adj, double rho) { sim_set_policy((Sim*)h, P, adj, rho); }
 
 // x_i(0) = x0_std * z, c_i = c_std * z from the X0 / C streams (round word 0).

@@ -53,6 +53,7 @@ def lib():
         L.nmo_sim_create.argtypes = [i32, i64, vp, i64, vp, vp, dbl, dbl, dbl, i32, u64]
         L.nmo_sim_create.restype = vp
         L.nmo_sim_destroy.argtypes = [vp]
+        L.nmo_sim_set_fixed_weight.argtypes = [vp, dbl]
         L.nmo_sim_set_policy.argtypes = [vp, vp, vp, dbl]
         L.nmo_sim_init.argtypes = [vp, dbl, dbl]
         for name in ("nmo_sim_set_x", "nmo_sim_set_c", "nmo_sim_get_x", "nmo_sim_get_c"):
@@ -141,7 +142,7 @@ def peer_draws(P: np.ndarray, seed: int, first_round: int, n_rounds: int) -> np.
 class Sim:
     """The round simulator: all M replicas (or a sample of their columns) on the CPU."""
 
-    def __init__(self, M, d, P, adj, alpha, rho, sigma, objective, seed, cols=None):
+    def __init__(self, M, d, P, adj, alpha, rho, sigma, objective, seed, cols=None, pull_weight=0.0):
         self.M, self.d = int(M), int(d)
         self._P = np.ascontiguousarray(P, dtype=np.float64)
         self._adj = np.ascontiguousarray(adj, dtype=np.uint8)
@@ -153,6 +154,9 @@ class Sim:
             self.ncols, cptr = int(self._cols.shape[0]), _p(self._cols)
         self._h = lib().nmo_sim_create(self.M, self.d, cptr, self.ncols, _p(self._P), _p(self._adj), float(alpha),
                                        float(rho), float(sigma), int(objective), int(seed))
+        if pull_weight > 0.0:      # fixed pull weight (gossip / AD-PSGD style averaging)
+            lib().nmo_sim_set_fixed_weight(self._h, float(pull_weight))
+            lib().nmo_sim_set_policy(self._h, _p(self._P), _p(self._adj), float(rho))
 
     def close(self):
         if self._h:

@@ -39,7 +39,7 @@ class NetmaxError(RuntimeError):
 class Config(C.Structure):
     _fields_ = [
         ("M", C.c_int32), ("d", C.c_int64), ("element_offset", C.c_int64), ("link_speed_gbps", C.c_void_p), ("prob", C.c_void_p),
-        ("lr", C.c_double), ("rho", C.c_double), ("sigma", C.c_double), ("x0_std", C.c_double),
+        ("lr", C.c_double), ("rho", C.c_double), ("pull_weight", C.c_double), ("sigma", C.c_double), ("x0_std", C.c_double),
         ("c_std", C.c_double), ("objective", C.c_int32), ("seed", C.c_uint64), ("device", C.c_int32),
         ("stream", C.c_void_p), ("trace_rounds", C.c_int64), ("policy_K", C.c_int32), ("policy_R", C.c_int32),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
@@ -147,7 +147,7 @@ class Netmax:
                  sigma: float = 0.0, x0_std: float = 0.0, c_std: float = 0.0, objective: int = 1, seed: int = 0,
                  device: int = 0, stream: Optional[int] = None, trace_rounds: int = 1024, policy_K: int = 20,
                  policy_R: int = 20, workspace: Optional[int] = None, workspace_bytes: int = 0,
-                 element_offset: int = 0):
+                 element_offset: int = 0, pull_weight: float = 0.0):
         L = lib()
         cfg = Config()
         _check(L.netmax_config_init(C.byref(cfg)))
@@ -157,6 +157,7 @@ class Netmax:
         cfg.link_speed_gbps = self._speed.ctypes.data if self._speed is not None else None
         cfg.prob = self._prob.ctypes.data if self._prob is not None else None
         cfg.lr, cfg.rho, cfg.sigma = float(lr), float(rho), float(sigma)
+        cfg.pull_weight = float(pull_weight)
         cfg.x0_std, cfg.c_std = float(x0_std), float(c_std)
         cfg.objective, cfg.seed, cfg.device = int(objective), int(seed), int(device)
         cfg.stream = stream

@@ -130,6 +130,7 @@ struct netmax_ctx {
   int64_t rounds = 0;
   int64_t trace_rounds = 0;
   double alpha = 0, rho = 0, sigma = 0;
+  double pull_weight = 0;  // > 0: fixed weight of every pull
   int objective = 1;
   uint64_t seed = 0;
   int policy_K = 20, policy_R = 20;
@@ -218,7 +219,7 @@ double default_rho(int32_t M, const double* P, const std::vector<uint8_t>& adj, 
 // T_j = floor(cum_j 2^32 + 1/2) over the left-to-right double prefix sums of the row,
 // non-decreasing, saturated, and pinned to the top from the last positive entry on.
 void build_tables(int32_t M, const double* P, const std::vector<uint8_t>& adj, double alpha32, double rho,
-                  std::vector<uint32_t>& thr, std::vector<int32_t>& last_nz, std::vector<float>& w) {
+                  double pull_weight, std::vector<uint32_t>& thr, std::vector<int32_t>& last_nz, std::vector<float>& w) {
   thr.resize((size_t)M * M);
   last_nz.resize(M);
   w.resize((size_t)M * M);
@@ -239,7 +240,8 @@ void build_tables(int32_t M, const double* P, const std::vector<uint8_t>& adj, d
       float wv = 0.0f;
       if (j != i && p[j] > 0.0) {
         const double dsum = (double)adj[(size_t)i * M + j] + (double)adj[(size_t)j * M + i];
-        wv = (float)(alpha32 * rho * dsum / (2.0 * p[j]));   // alpha rho gamma_im   (Eq. 16)
+        wv = pull_weight > 0.0 ? (float)pull_weight                         // fixed-weight averaging
+                               : (float)(alpha32 * rho * dsum / (2.0 * p[j]));  // alpha rho gamma_im (Eq. 16)
       }
       w[(size_t)i * M + j] = wv;
     }
@@ -250,7 +252,7 @@ int upload_policy(netmax_ctx* ctx) {
   std::vector<uint32_t>& thr = ctx->h_thr;
   std::vector<int32_t>& last = ctx->h_last;
   std::vector<float>& w = ctx->h_w;
-  build_tables(ctx->M, ctx->P.data(), ctx->adj, (double)(float)ctx->alpha, ctx->rho, thr, last, w);
+  build_tables(ctx->M, ctx->P.data(), ctx->adj, (double)(float)ctx->alpha, ctx->rho, ctx->pull_weight, thr, last, w);
   // pageable sources: the copies are complete (staged) when these calls return
   NM_CUDA(ctx, cudaMemcpyAsync(ctx->thr, thr.data(), thr.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));
   NM_CUDA(ctx, cudaMemcpyAsync(ctx->last_nz, last.data(), last.size() * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
@@ -470,6 +472,8 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   if (!(cfg->x0_std >= 0.0) || !std::isfinite(cfg->x0_std) || !(cfg->c_std >= 0.0) || !std::isfinite(cfg->c_std))
     return fail(nullptr, NETMAX_INVALID_ARG, "x0_std and c_std must be >= 0 and finite");
   if (!std::isfinite(cfg->rho)) return fail(nullptr, NETMAX_INVALID_ARG, "rho is not finite");
+  if (!(cfg->pull_weight >= 0.0 && cfg->pull_weight < 1.0))
+    return fail(nullptr, NETMAX_INVALID_ARG, "pull_weight = %g outside [0, 1)", cfg->pull_weight);
   if (cfg->objective != 0 && cfg->objective != 1) return fail(nullptr, NETMAX_INVALID_ARG, "objective = %d is not 0 or 1", cfg->objective);
   if (cfg->device < 0) return fail(nullptr, NETMAX_INVALID_ARG, "device = %d", cfg->device);
 
@@ -488,6 +492,7 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   ctx->trace_rounds = cfg->trace_rounds;
   ctx->alpha = cfg->lr;
   ctx->sigma = cfg->sigma;
+  ctx->pull_weight = cfg->pull_weight;
   ctx->objective = cfg->objective;
   ctx->seed = cfg->seed;
   ctx->policy_K = cfg->policy_K > 0 ? cfg->policy_K : 20;

@@ -326,3 +326,21 @@ def test_column_shards_match_the_unsharded_problem(nm):
         nm.Netmax(M=M, d=d, lr=0.05, prob=P, element_offset=2)
     for g in parts:
         g.close()
+
+
+@pytest.mark.parametrize("M,d", [(2, 9), (6, 4099), (64, 515)])
+def test_fixed_pull_weight_matches_oracle(nm, M, d):
+    """The gossip / AD-PSGD style rule: every pull averages with a constant weight."""
+    rng = np.random.default_rng(M + 7 * d)
+    P = random_policy(M, rng)
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=1, seed=17, pull_weight=0.5)
+    o = oracle.Sim(M, d, P, full_adj(M), alpha=0.05, rho=g.get_policy()[1], sigma=0.1, objective=1, seed=17,
+                   pull_weight=0.5)
+    o.init(1.0, 1.0)
+    g.round(25)
+    o.round(25)
+    assert (g.peer_trace() == o.trace()).all()
+    assert_replicas_close(g.read_replicas(), o.x())
+    with pytest.raises(nm.NetmaxError):
+        nm.Netmax(M=M, d=d, lr=0.05, prob=P, pull_weight=1.0)
+    g.close()

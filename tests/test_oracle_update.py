@@ -296,3 +296,42 @@ def test_telemetry_matches_its_definition():
     x64, c64 = x0.astype(np.float64), c.astype(np.float64)
     assert cons[0] == pytest.approx(((x64 - x64.mean(axis=0)) ** 2).sum() / M, rel=1e-12)
     assert loss[0] == pytest.approx(0.5 * ((x64 - c64) ** 2).sum() / M, rel=1e-12)
+
+
+# ---------------------------------------------------------------- fixed pull weight (gossip / AD-PSGD style)
+def test_fixed_weight_half_averages_two_workers_in_one_round():
+    """w = 1/2, M = 2, both pull each other from the round-start snapshot: x1' = x2' = (x1+x2)/2."""
+    d = 9
+    P = np.array([[0.0, 1.0], [1.0, 0.0]])
+    x0 = np.random.default_rng(30).standard_normal((2, d)).astype(np.float32)
+    sim = oracle.Sim(2, d, P, full_adj(2), alpha=0.1, rho=123.0, sigma=0.0, objective=0, seed=1, pull_weight=0.5)
+    sim.set_x(x0)
+    sim.round(1)
+    want = ((x0[0].astype(np.float64) + x0[1]) / 2).astype(np.float32)
+    assert (sim.x()[0] == want).all() and (sim.x()[1] == want).all()
+    assert (oracle.Sim(2, d, P, full_adj(2), 0.1, 123.0, 0.0, 0, 1, pull_weight=0.5).x() == 0).all()
+
+
+def test_fixed_weight_ignores_rho_and_probabilities():
+    rng = np.random.default_rng(31)
+    M, d = 5, 16
+    P = random_policy(M, rng)
+    x0 = rng.standard_normal((M, d)).astype(np.float32)
+    sims = []
+    for rho in (0.01, 7.0):
+        s = oracle.Sim(M, d, P, full_adj(M), alpha=0.1, rho=rho, sigma=0.0, objective=0, seed=2, pull_weight=0.25)
+        s.set_x(x0)
+        s.round(6)
+        sims.append(s)
+    assert (sims[0].x() == sims[1].x()).all()
+    trace = sims[0].trace()
+    x = x0.astype(np.float64)
+    for r in range(6):                                   # D^r with the constant weight on every pull
+        D = np.eye(M)
+        for i in range(M):
+            m = trace[r, i]
+            if m != i:
+                D[i, i] -= 0.25
+                D[i, m] += 0.25
+        x = (D @ x).astype(np.float32).astype(np.float64)
+    np.testing.assert_allclose(sims[0].x(), x, atol=1e-6)
