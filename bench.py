@@ -228,7 +228,8 @@ def run_ours(args, w):
     # control plane (host, untimed): Algorithm 3 on the workload's link speeds
     speeds = w.link_speeds(0)
     t_iter, adj = binding.netmax_iteration_times(speeds, w.d)
-    P, rho, pinfo = binding.netmax_policy_generate(t_iter, adj, w.lr, w.K, w.R)
+    generate = binding.netmax_policy_generate_device if w.M >= 512 else binding.netmax_policy_generate
+    P, rho, pinfo = generate(t_iter, adj, w.lr, w.K, w.R)
 
     plan = shard_plan(w.d, world, rank)
     stream = torch.cuda.Stream()

@@ -267,6 +267,18 @@ int netmax_iteration_times(int32_t M, int64_t d, const double* link_speed_gbps, 
 int netmax_policy_generate(int32_t M, const double* t_iter, const uint8_t* adj, double lr, int32_t K, int32_t R,
                            double* prob_out, double* rho_out, double* info_out /* 5 doubles */);
 
+/*
+ * Algorithm 3 on the GPU, for large M (thousands of workers, links redrawn often): the same
+ * grids, the same row-wise LP optimum and the same selection as netmax_policy_generate, with
+ * one CTA per row of P, Y_P (Eq. 22) kept in device memory and lambda_2 by Lanczos on the
+ * device.  Host arrays in and out as for netmax_policy_generate; allocates its own device
+ * buffers (about 4 M*M doubles) on `device` and works on `stream` (a cudaStream_t, may be
+ * NULL); synchronises before returning.  Results agree with the host generator to rounding.
+ */
+int netmax_policy_generate_device(int32_t M, const double* t_iter, const uint8_t* adj, double lr, int32_t K, int32_t R,
+                                  int32_t device, void* stream, double* prob_out, double* rho_out,
+                                  double* info_out /* 5 doubles or NULL */);
+
 /* Counters for benchmarks: kernels launched by this context so far. */
 int64_t netmax_kernel_launches(const netmax_ctx* ctx);
 

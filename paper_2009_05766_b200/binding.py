@@ -26,7 +26,7 @@ EXPORTS = [
     "netmax_peer_trace", "netmax_telemetry", "netmax_replicas_device", "netmax_sample_peers",
     "netmax_measure", "netmax_async_begin", "netmax_async_set_times", "netmax_async_steps", "netmax_async_time",
     "netmax_async_trace", "netmax_async_ema",
-    "netmax_iteration_times", "netmax_policy_generate", "netmax_kernel_launches", "netmax_last_error",
+    "netmax_iteration_times", "netmax_policy_generate", "netmax_policy_generate_device", "netmax_kernel_launches", "netmax_last_error",
 ]
 
 
@@ -91,6 +91,7 @@ def lib():
             "netmax_async_ema": ([vp, vp, vp], C.c_int),
             "netmax_iteration_times": ([i32, i64, vp, vp, vp], C.c_int),
             "netmax_policy_generate": ([i32, vp, vp, dbl, i32, i32, vp, vp, vp], C.c_int),
+            "netmax_policy_generate_device": ([i32, vp, vp, dbl, i32, i32, i32, vp, vp, vp, vp], C.c_int),
             "netmax_kernel_launches": ([vp], i64),
             "netmax_last_error": ([vp], C.c_char_p),
         }
@@ -137,6 +138,18 @@ def netmax_policy_generate(t_iter, adj, lr: float, K: int, R: int):
     rho = C.c_double()
     info = np.empty(5, dtype=np.float64)
     _check(lib().netmax_policy_generate(M, _p(t), _p(adj), float(lr), int(K), int(R), _p(P), C.byref(rho), _p(info)))
+    return P, rho.value, dict(lam2=info[0], tbar=info[1], t_conv=info[2], k=int(info[3]), r=int(info[4]))
+
+
+def netmax_policy_generate_device(t_iter, adj, lr: float, K: int, R: int, device: int = 0, stream=None):
+    t = _f64(t_iter)
+    M = t.shape[0]
+    adj = np.ascontiguousarray(adj, dtype=np.uint8)
+    P = np.empty((M, M), dtype=np.float64)
+    rho = C.c_double()
+    info = np.empty(5, dtype=np.float64)
+    _check(lib().netmax_policy_generate_device(M, _p(t), _p(adj), float(lr), int(K), int(R), int(device), stream,
+                                               _p(P), C.byref(rho), _p(info)))
     return P, rho.value, dict(lam2=info[0], tbar=info[1], t_conv=info[2], k=int(info[3]), r=int(info[4]))
 
 

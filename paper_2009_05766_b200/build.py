@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnetmax.so")
-SOURCES = ["netmax.cu", "netmax_policy.cpp"]
-DEPS = SOURCES + ["netmax_kernels.cuh", "netmax_rng.cuh", "netmax_policy.h", os.path.join("..", "..", "include", "netmax.h")]
+SOURCES = ["netmax.cu", "netmax_policy.cpp", "netmax_policy_gpu.cu"]
+DEPS = SOURCES + ["netmax_policy_gpu_host.inc", "netmax_kernels.cuh", "netmax_rng.cuh", "netmax_policy.h", os.path.join("..", "..", "include", "netmax.h")]
 
 
 def _nvcc() -> str:

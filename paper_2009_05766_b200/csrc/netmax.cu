@@ -293,8 +293,14 @@ int resolve_policy(netmax_ctx* ctx, const double* speed, const double* prob, dou
   }
   ctx->P.assign((size_t)M * M, 0.0);
   double rho_sel = 0.0;
-  int rc = netmax_policy_generate(M, ctx->t_iter.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K, ctx->policy_R,
-                                  ctx->P.data(), &rho_sel, nullptr);
+  // Algorithm 3: on the device from 512 workers up (where the host generator takes seconds)
+  int ndev = 0;
+  const bool on_device = M >= 512 && cudaGetDeviceCount(&ndev) == cudaSuccess && ctx->device < ndev;
+  if (!on_device) cudaGetLastError();
+  int rc = on_device ? netmax_policy_generate_device(M, ctx->t_iter.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K,
+                                                     ctx->policy_R, ctx->device, ctx->stream, ctx->P.data(), &rho_sel, nullptr)
+                     : netmax_policy_generate(M, ctx->t_iter.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K,
+                                              ctx->policy_R, ctx->P.data(), &rho_sel, nullptr);
   if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
   ctx->rho = rho > 0.0 ? rho : rho_sel;
   return NETMAX_OK;

@@ -245,6 +245,21 @@ double second_eigenvalue(const std::vector<double>& Y, int M) {
 
 }  // namespace
 
+namespace netmax {
+// Largest eigenvalue of the symmetric tridiagonal matrix with diagonal alpha[0..m) and
+// off-diagonal beta[0..m-1) (the Ritz values of a Lanczos run).
+double tridiagonal_top_eigenvalue(const std::vector<double>& alpha, const std::vector<double>& beta) {
+  const int m = (int)alpha.size();
+  std::vector<double> Tm((size_t)m * m, 0.0), eig;
+  for (int k = 0; k < m; ++k) {
+    Tm[(size_t)k * m + k] = alpha[k];
+    if (k + 1 < m) Tm[(size_t)k * m + k + 1] = Tm[(size_t)(k + 1) * m + k] = beta[k];
+  }
+  jacobi_eigenvalues(Tm, m, eig);
+  return eig[m - 1];
+}
+}  // namespace netmax
+
 extern "C" {
 
 int netmax_iteration_times(int32_t M, int64_t d, const double* speed, double* t_out, uint8_t* adj_out) {
