@@ -223,6 +223,18 @@ int netmax_async_begin(netmax_ctx* ctx, const double* t_iter, double beta);
 int netmax_async_set_times(netmax_ctx* ctx, const double* t_iter);
 /* Runs the next n_steps global steps, asynchronously on the context's stream. */
 int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps);
+/*
+ * Network Monitor (Algorithm 1) on the simulated clock: every period_s simulated seconds,
+ * before the first global step at or after the boundary, the moving averages T_i[m] are
+ * collected, Algorithm 3 runs on them (policy_K x policy_R grid) and the resulting P and rho are
+ * installed for iterations that start afterwards.  An average with n samples is read as
+ * T / (1 - beta^n) (Algorithm 2 starts T at 0); a link never sampled so far is taken at its
+ * current iteration time; a grid with no feasible point leaves the policy unchanged.
+ * period_s = 0 switches the monitor off.  netmax_async_monitor_refreshes counts the policies
+ * installed so far.
+ */
+int netmax_async_monitor(netmax_ctx* ctx, double period_s);
+int64_t netmax_async_monitor_refreshes(const netmax_ctx* ctx);
 /* Simulated time of the last global step and the number of global steps so far. */
 int netmax_async_time(netmax_ctx* ctx, double* sim_time, int64_t* steps_done);
 /*

@@ -496,6 +496,11 @@ void nmo_async_steps(void* h, int64_t n) {
 
 int64_t nmo_async_steps_done(void* h) { return (int64_t)((Sim*)h)->ev_worker.size(); }
 double nmo_async_now(void* h) { return ((Sim*)h)->now; }
+// Simulated time of the next global step (the earliest pending finish time).
+double nmo_async_next_time(void* h) {
+  Sim* s = (Sim*)h;
+  return *std::min_element(s->finish.begin(), s->finish.end());
+}
 
 void nmo_async_trace(void* h, int64_t first, int64_t n, int32_t* worker, int32_t* peer, int64_t* local_iter, double* time) {
   Sim* s = (Sim*)h;

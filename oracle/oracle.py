@@ -71,6 +71,8 @@ def lib():
         L.nmo_async_steps_done.restype = i64
         L.nmo_async_now.argtypes = [vp]
         L.nmo_async_now.restype = dbl
+        L.nmo_async_next_time.argtypes = [vp]
+        L.nmo_async_next_time.restype = dbl
         L.nmo_async_trace.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.nmo_async_ema.argtypes = [vp, vp, vp]
         _lib = L
@@ -233,6 +235,10 @@ class Sim:
     @property
     def async_now(self) -> float:
         return float(lib().nmo_async_now(self._h))
+
+    @property
+    def async_next_time(self) -> float:
+        return float(lib().nmo_async_next_time(self._h))
 
     def async_trace(self, first=0, n=None):
         n = self.async_steps_done - first if n is None else n

@@ -25,7 +25,7 @@ EXPORTS = [
     "netmax_read_columns_static",
     "netmax_peer_trace", "netmax_telemetry", "netmax_replicas_device", "netmax_sample_peers",
     "netmax_measure", "netmax_async_begin", "netmax_async_set_times", "netmax_async_steps", "netmax_async_time",
-    "netmax_async_trace", "netmax_async_ema",
+    "netmax_async_trace", "netmax_async_ema", "netmax_async_monitor", "netmax_async_monitor_refreshes",
     "netmax_iteration_times", "netmax_policy_generate", "netmax_policy_generate_device", "netmax_kernel_launches", "netmax_last_error",
 ]
 
@@ -89,6 +89,8 @@ def lib():
             "netmax_async_time": ([vp, vp, vp], C.c_int),
             "netmax_async_trace": ([vp, i64, i64, vp, vp, vp, vp], C.c_int),
             "netmax_async_ema": ([vp, vp, vp], C.c_int),
+            "netmax_async_monitor": ([vp, dbl], C.c_int),
+            "netmax_async_monitor_refreshes": ([vp], i64),
             "netmax_iteration_times": ([i32, i64, vp, vp, vp], C.c_int),
             "netmax_policy_generate": ([i32, vp, vp, dbl, i32, i32, vp, vp, vp], C.c_int),
             "netmax_policy_generate_device": ([i32, vp, vp, dbl, i32, i32, i32, vp, vp, vp, vp], C.c_int),
@@ -305,6 +307,13 @@ class Netmax:
 
     def async_steps(self, n_steps: int):
         _check(lib().netmax_async_steps(self._h, int(n_steps)), self._h)
+
+    def async_monitor(self, period_s: float):
+        _check(lib().netmax_async_monitor(self._h, float(period_s)), self._h)
+
+    @property
+    def async_monitor_refreshes(self) -> int:
+        return int(lib().netmax_async_monitor_refreshes(self._h))
 
     def async_time(self):
         t, k = C.c_double(), C.c_int64()

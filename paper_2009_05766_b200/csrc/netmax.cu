@@ -121,6 +121,8 @@ struct netmax_ctx {
   std::vector<double> finish;
   std::vector<double> ema;
   std::vector<int64_t> ema_count;
+  double monitor_period = 0.0, monitor_next = 0.0;  // Network Monitor on the simulated clock (0: off)
+  int64_t monitor_refreshes = 0;
   int64_t ev_cap = 0;
   std::vector<int32_t> ev_worker, ev_peer;
   std::vector<int64_t> ev_n;
@@ -1031,6 +1033,47 @@ int netmax_async_set_times(netmax_ctx* ctx, const double* t_iter) {
   return NETMAX_OK;
 }
 
+// Network Monitor (Algorithm 1): collect the workers' moving averages of iteration times, run
+// Algorithm 3 on them and send P and rho back.  An average that has seen n samples is read as
+// T / (1 - beta^n) (Algorithm 2 starts T at 0); a link that was never sampled is taken at its
+// current iteration time.  An infeasible grid leaves the policy in force.
+static int monitor_refresh(netmax_ctx* ctx) {
+  const int32_t M = ctx->M;
+  std::vector<double> t((size_t)M * M, 0.0);
+  for (size_t at = 0; at < (size_t)M * M; ++at) {
+    const int i = (int)(at / M), m = (int)(at % M);
+    if (i != m && !ctx->adj[at]) continue;
+    const int64_t n = ctx->ema_count[at];
+    t[at] = n > 0 ? ctx->ema[at] / (1.0 - std::pow(ctx->beta, (double)n)) : ctx->t_iter[at];
+  }
+  std::vector<double> P((size_t)M * M);
+  double rho = 0.0;
+  int ndev = 0;
+  const bool on_device = M >= 512 && cudaGetDeviceCount(&ndev) == cudaSuccess && ctx->device < ndev;
+  int rc = on_device ? netmax_policy_generate_device(M, t.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K, ctx->policy_R,
+                                                     ctx->device, ctx->stream, P.data(), &rho, nullptr)
+                     : netmax_policy_generate(M, t.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K, ctx->policy_R,
+                                              P.data(), &rho, nullptr);
+  if (rc == NETMAX_INFEASIBLE) return NETMAX_OK;
+  if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
+  ctx->P.swap(P);
+  ctx->rho = rho;
+  ctx->monitor_refreshes += 1;
+  NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  return upload_policy(ctx);
+}
+
+int netmax_async_monitor(netmax_ctx* ctx, double period_s) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (!ctx->async_on) return fail(ctx, NETMAX_INVALID_ARG, "call netmax_async_begin first");
+  if (!(period_s >= 0.0) || !std::isfinite(period_s)) return fail(ctx, NETMAX_INVALID_ARG, "period_s = %g", period_s);
+  ctx->monitor_period = period_s;
+  ctx->monitor_next = ctx->now + period_s;
+  return NETMAX_OK;
+}
+
+int64_t netmax_async_monitor_refreshes(const netmax_ctx* ctx) { return ctx ? ctx->monitor_refreshes : -1; }
+
 int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps) {
   if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
   if (!ctx->async_on) return fail(ctx, NETMAX_INVALID_ARG, "call netmax_async_begin first");
@@ -1071,6 +1114,13 @@ int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps) {
     int i = 0;
     for (int j = 1; j < M; ++j)
       if (ctx->finish[j] < ctx->finish[i]) i = j;
+    // the Network Monitor wakes up before any step at or after its next period boundary
+    while (ctx->monitor_period > 0.0 && ctx->finish[i] >= ctx->monitor_next) {
+      int rc = flush();
+      if (!rc) rc = monitor_refresh(ctx);
+      if (rc) return rc;
+      ctx->monitor_next += ctx->monitor_period;
+    }
     const int m = ctx->pending_peer[i];
     // a launch holds steps on disjoint replicas only: this one must not write a row that an
     // earlier step of the launch reads or writes, nor read a row that one writes

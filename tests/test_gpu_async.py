@@ -161,3 +161,60 @@ def test_async_full_size_resnet18_vectors_on_sampled_columns(nm):
         assert (a == b).all()
     close(g.read_columns(cols), o.x())
     g.close()
+
+
+def test_network_monitor_loop_matches_an_oracle_driven_replay(nm):
+    """Algorithm 1 on the simulated clock: workers start with uniform probabilities, the monitor
+    installs Algorithm 3's policy from the measured (EMA) iteration times every period, and
+    adapts one period after the link speeds change.  The replay drives the oracle step by step
+    and computes each policy with the oracle's numpy Algorithm 3."""
+    rng = np.random.default_rng(21)
+    M, d, lr, beta, K, R = 6, 400, 0.05, 0.8, 6, 6
+
+    def times(seed):
+        r = np.random.default_rng(seed)
+        s = np.triu(np.exp(r.uniform(np.log(1.0), np.log(40.0), (M, M))), 1)
+        return opolicy.iteration_times(s + s.T, 1_000_000)
+
+    t1, adj = times(1)
+    t2, _ = times(2)
+    P0 = np.full((M, M), 1.0 / M)                       # Algorithm 2: initial probabilities 1/M
+    rho0 = 0.5 / (2 * lr * M)
+    period = 12 * t1[adj == 1].mean()
+    g = nm.Netmax(M=M, d=d, lr=lr, prob=P0, rho=rho0, sigma=0.05, x0_std=1.0, c_std=1.0, seed=4, policy_K=K, policy_R=R)
+    o = oracle.Sim(M, d, P0, adj, alpha=lr, rho=rho0, sigma=0.05, objective=1, seed=4)
+    o.init(1.0, 1.0)
+    g.async_begin(t1, beta)
+    o.async_begin(t1, beta)
+    g.async_monitor(period)
+    state = dict(next=period, t=t1, refreshes=0)
+
+    def replay(n):
+        for _ in range(n):
+            while o.async_next_time >= state["next"]:
+                ema, count = o.async_ema()
+                est = np.where(count > 0, ema / (1.0 - beta ** np.maximum(count, 1)), state["t"])
+                est = np.where((adj == 1) | np.eye(M, dtype=bool), est, 0.0)
+                try:
+                    P, rho, _ = opolicy.generate_policy(est, adj, lr, K, R)
+                    o.set_policy(P, adj, rho)
+                    state["refreshes"] += 1
+                except ValueError:
+                    pass
+                state["next"] += period
+            o.async_steps(1)
+
+    g.async_steps(150)
+    replay(150)
+    g.async_set_times(t2)                                # the network changes
+    o.async_set_times(t2)
+    state["t"] = t2
+    g.async_steps(250)
+    replay(250)
+    for a, b in zip(g.async_trace(), o.async_trace()):
+        assert (a == b).all()
+    close(g.read_replicas(), o.x())
+    assert g.async_monitor_refreshes == state["refreshes"] >= 3
+    Pg, rhog = g.get_policy()
+    assert np.abs(Pg - P0).max() > 0.05                  # the monitor moved the policy away from uniform
+    g.close()
