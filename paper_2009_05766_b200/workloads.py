@@ -106,3 +106,27 @@ def sample_columns(d: int, n: int, seed: int) -> np.ndarray:
     edge = np.concatenate([np.arange(0, min(d, 9)), np.arange(max(0, d - 9), d)])
     body = rng.integers(0, d, size=max(0, n - edge.shape[0]))
     return np.unique(np.concatenate([edge, body])).astype(np.int64)
+
+
+def clustered_centres(M: int, d: int, group_size: int, spread: float, within: float, seed: int) -> np.ndarray:
+    """Non-IID-like objectives: the workers of one machine share a cluster centre (drawn with
+    standard deviation `spread`), their own centres scatter around it with `within`."""
+    rng = np.random.default_rng([seed, 11])
+    groups = (M + group_size - 1) // group_size
+    base = spread * rng.standard_normal((groups, d))
+    c = base[np.arange(M) // group_size] + within * rng.standard_normal((M, d))
+    return c.astype(np.float32)
+
+
+def sparse_ring_of_groups(M: int, group_size: int, intra_gbps: float, inter_gbps: float) -> np.ndarray:
+    """A sparse link graph: all-to-all inside a machine, and only the first worker of each
+    machine linked to the first worker of the next machine (a ring of machines)."""
+    s = np.zeros((M, M), dtype=np.float64)
+    group = np.arange(M) // group_size
+    s[group[:, None] == group[None, :]] = intra_gbps
+    heads = np.arange(0, M, group_size)
+    for a, b in zip(heads, np.roll(heads, -1)):
+        if a != b:
+            s[a, b] = s[b, a] = inter_gbps
+    np.fill_diagonal(s, 0.0)
+    return s

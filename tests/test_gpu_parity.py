@@ -344,3 +344,36 @@ def test_fixed_pull_weight_matches_oracle(nm, M, d):
     with pytest.raises(nm.NetmaxError):
         nm.Netmax(M=M, d=d, lr=0.05, prob=P, pull_weight=1.0)
     g.close()
+
+
+def test_sparse_graph_with_clustered_centres(nm):
+    """A ring of machines (most d_im = 0) and non-IID-like objectives: centres clustered by machine."""
+    M, d, gsz = 12, 6007, 4
+    s = workloads.sparse_ring_of_groups(M, gsz, 100.0, 5.0)
+    t, adj = opolicy.iteration_times(s, 5_000_000)
+    assert adj.sum() < M * (M - 1) / 2
+    P, rho, _ = opolicy.generate_policy(t, adj, 0.05, 20, 20)   # slow ring links leave only small rho feasible
+    assert (P[(adj == 0) & ~np.eye(M, dtype=bool)] == 0).all()
+    c = workloads.clustered_centres(M, d, gsz, spread=1.0, within=0.05, seed=3)
+    g = nm.Netmax(M=M, d=d, lr=0.05, link_speed_gbps=s, prob=P, rho=rho, sigma=0.05, x0_std=1.0, objective=1, seed=29)
+    o = oracle.Sim(M, d, P, adj, alpha=0.05, rho=rho, sigma=0.05, objective=1, seed=29)
+    o.init(1.0, 0.0)
+    g.set_centres(c)
+    o.set_c(c)
+    g.round(200)
+    o.round(200)
+    assert (g.peer_trace(0, 200) == o.trace()).all()
+    assert_replicas_close(g.read_replicas(), o.x())
+    cons, loss = g.telemetry(0, 200)
+    assert cons[-1] < 0.8 * cons[0]          # clustered optima and a weak coupling keep machines apart
+    # the library's own Algorithm 3 on the same sparse graph gives the same policy
+    h = nm.Netmax(M=M, d=5_000_000, lr=0.05, link_speed_gbps=s, policy_K=20, policy_R=20)
+    np.testing.assert_allclose(h.get_policy()[0], P, atol=1e-9)
+    with pytest.raises(nm.NetmaxError) as e:
+        bad = P.copy()
+        bad[0, 5] = 0.01
+        bad[0] /= bad[0].sum()
+        nm.Netmax(M=M, d=d, lr=0.05, link_speed_gbps=s, prob=bad)
+    assert e.value.code == -2                              # Eq. 12: no probability on a missing link
+    g.close()
+    h.close()
