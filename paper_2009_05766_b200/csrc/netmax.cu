@@ -11,6 +11,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <queue>
 #include <string>
 #include <vector>
 
@@ -119,6 +120,8 @@ struct netmax_ctx {
   std::vector<int64_t> local_n;
   std::vector<int32_t> pending_peer;
   std::vector<double> finish;
+  // pending iterations ordered by (finish time, worker): exactly one entry per worker
+  std::priority_queue<std::pair<double, int>, std::vector<std::pair<double, int>>, std::greater<std::pair<double, int>>> queue;
   std::vector<double> ema;
   std::vector<int64_t> ema_count;
   double monitor_period = 0.0, monitor_next = 0.0;  // Network Monitor on the simulated clock (0: off)
@@ -1022,7 +1025,11 @@ int netmax_async_begin(netmax_ctx* ctx, const double* t_iter, double beta) {
   ctx->ev_peer.assign(ctx->ev_cap, 0);
   ctx->ev_n.assign(ctx->ev_cap, 0);
   ctx->ev_time.assign(ctx->ev_cap, 0.0);
-  for (int i = 0; i < M; ++i) async_start_iteration(ctx, i, 0.0);
+  ctx->queue = decltype(ctx->queue)();
+  for (int i = 0; i < M; ++i) {
+    async_start_iteration(ctx, i, 0.0);
+    ctx->queue.emplace(ctx->finish[i], i);
+  }
   return NETMAX_OK;
 }
 
@@ -1111,9 +1118,7 @@ int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps) {
   };
   for (int64_t k = 0; k < n_steps; ++k) {
     // the next global step: the worker whose iteration finishes first (ties: lowest index)
-    int i = 0;
-    for (int j = 1; j < M; ++j)
-      if (ctx->finish[j] < ctx->finish[i]) i = j;
+    const int i = ctx->queue.top().second;
     // the Network Monitor wakes up before any step at or after its next period boundary
     while (ctx->monitor_period > 0.0 && ctx->finish[i] >= ctx->monitor_next) {
       int rc = flush();
@@ -1151,6 +1156,8 @@ int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps) {
     ctx->local_n[i] += 1;
     ctx->steps += 1;
     async_start_iteration(ctx, i, ctx->now);
+    ctx->queue.pop();
+    ctx->queue.emplace(ctx->finish[i], i);
   }
   return flush();
 }
