@@ -291,6 +291,15 @@ int netmax_policy_generate_device(int32_t M, const double* t_iter, const uint8_t
                                   int32_t device, void* stream, double* prob_out, double* rho_out,
                                   double* info_out /* 5 doubles or NULL */);
 
+/*
+ * Test hook for the bounded waits of multi-round launches (short vectors, netmax_round(n >= 2)):
+ * the NEXT such launch also waits, at its grid-wide barrier, for n CTAs that do not exist, so
+ * every wait runs out (about two seconds), the kernel returns after its first round and the
+ * next synchronising call reports NETMAX_CUDA_ERROR; the replicas are then not valid and should
+ * be set again.  Nothing faults or hangs, and the context stays usable.  n = 0 cancels.
+ */
+int netmax_debug_absent_ctas(netmax_ctx* ctx, int32_t n);
+
 /* Counters for benchmarks: kernels launched by this context so far. */
 int64_t netmax_kernel_launches(const netmax_ctx* ctx);
 

@@ -26,7 +26,7 @@ EXPORTS = [
     "netmax_peer_trace", "netmax_telemetry", "netmax_replicas_device", "netmax_sample_peers",
     "netmax_measure", "netmax_async_begin", "netmax_async_set_times", "netmax_async_steps", "netmax_async_time",
     "netmax_async_trace", "netmax_async_ema", "netmax_async_monitor", "netmax_async_monitor_refreshes",
-    "netmax_iteration_times", "netmax_policy_generate", "netmax_policy_generate_device", "netmax_kernel_launches", "netmax_last_error",
+    "netmax_iteration_times", "netmax_policy_generate", "netmax_policy_generate_device", "netmax_debug_absent_ctas", "netmax_kernel_launches", "netmax_last_error",
 ]
 
 
@@ -94,6 +94,7 @@ def lib():
             "netmax_iteration_times": ([i32, i64, vp, vp, vp], C.c_int),
             "netmax_policy_generate": ([i32, vp, vp, dbl, i32, i32, vp, vp, vp], C.c_int),
             "netmax_policy_generate_device": ([i32, vp, vp, dbl, i32, i32, i32, vp, vp, vp, vp], C.c_int),
+            "netmax_debug_absent_ctas": ([vp, i32], C.c_int),
             "netmax_kernel_launches": ([vp], i64),
             "netmax_last_error": ([vp], C.c_char_p),
         }
@@ -335,6 +336,9 @@ class Netmax:
         count = np.empty((self.M, self.M), dtype=np.int64)
         _check(lib().netmax_async_ema(self._h, _p(ema), _p(count)), self._h)
         return ema, count
+
+    def debug_absent_ctas(self, n: int):
+        _check(lib().netmax_debug_absent_ctas(self._h, int(n)), self._h)
 
     @property
     def kernel_launches(self) -> int:

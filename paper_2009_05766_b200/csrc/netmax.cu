@@ -106,6 +106,7 @@ struct netmax_ctx {
   unsigned int* grid_barrier = nullptr;  // arrival counter of multi-round launches
   unsigned int* dev_error = nullptr;     // raised by a kernel whose bounded wait gave up
   bool cooperative = false;              // device supports cooperative launches
+  uint32_t inject_absent_ctas = 0;       // test hook: applied to the next multi-round launch, then cleared
   double* measure_out = nullptr;         // device: (consensus, loss) of netmax_measure
   // host copies of the tables in force (the asynchronous timeline draws peers on the host)
   std::vector<uint32_t> h_thr;
@@ -741,6 +742,8 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
         mp.ring = ctx->trace_rounds;
         mp.first_round = (uint64_t)ctx->rounds;
         mp.n_rounds = (int32_t)chunk;
+        mp.absent_ctas = ctx->inject_absent_ctas;
+        ctx->inject_absent_ctas = 0;
         NM_CUDA(ctx, cudaMemsetAsync(ctx->grid_barrier, 0, sizeof(unsigned int), ctx->stream));
         void* args[] = {&mp};
         NM_CUDA(ctx, cudaLaunchCooperativeKernel((const void*)pick_multi_kernel(ctx->objective), dim3(plan.grid), dim3(kThreads),
@@ -1192,6 +1195,13 @@ int netmax_async_ema(netmax_ctx* ctx, double* ema_out, int64_t* samples_out) {
   if (!ctx->async_on) return fail(ctx, NETMAX_INVALID_ARG, "call netmax_async_begin first");
   if (ema_out) std::memcpy(ema_out, ctx->ema.data(), ctx->ema.size() * sizeof(double));
   if (samples_out) std::memcpy(samples_out, ctx->ema_count.data(), ctx->ema_count.size() * sizeof(int64_t));
+  return NETMAX_OK;
+}
+
+int netmax_debug_absent_ctas(netmax_ctx* ctx, int32_t n) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (n < 0 || n > 1024) return fail(ctx, NETMAX_INVALID_ARG, "n = %d outside [0, 1024]", n);
+  ctx->inject_absent_ctas = (uint32_t)n;
   return NETMAX_OK;
 }
 

@@ -429,18 +429,20 @@ struct MultiRoundParams {
   int64_t slot0, ring;    // ring slot of the first round
   uint64_t first_round;
   int32_t n_rounds;
+  uint32_t absent_ctas;   // test hook: the barrier also waits for this many CTAs that do not exist
 };
 
 constexpr uint32_t kBarrierSpinLimit = 1u << 21;
 
 // Grid-wide barrier number `epoch` (1, 2, ...).  Returns false if the wait gave up.
-__device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int epoch, unsigned int* error) {
+__device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int epoch, unsigned int* error,
+                                             unsigned int absent_ctas) {
   __shared__ int s_ok;
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();  // this CTA's writes of the round are visible before it is counted
     atomicAdd(counter, 1u);
-    const unsigned int target = epoch * gridDim.x;
+    const unsigned int target = epoch * (gridDim.x + absent_ctas);
     int ok = 0;
     for (uint32_t it = 0; it < kBarrierSpinLimit; ++it) {
       if (*reinterpret_cast<volatile unsigned int*>(counter) >= target) {
@@ -475,7 +477,7 @@ __global__ void __launch_bounds__(256, 2) multi_round_kernel(const MultiRoundPar
     round_tiles<kObjective, kFastNoise, 4, true>(p, x_cur, x_nxt, mp.trace + slot * p.M, (uint32_t)round,
                                                  philox_ctr3(kTagNoise, round), s_pw, s_col, acc_cons, acc_loss);
     block_partials(partials, acc_cons, acc_loss, s_red);
-    if (!grid_barrier(mp.barrier, (unsigned int)(k + 1), mp.error)) return;
+    if (!grid_barrier(mp.barrier, (unsigned int)(k + 1), mp.error, mp.absent_ctas)) return;
     // round k is complete everywhere: one CTA publishes its telemetry while the rest move on
     // (partials alternate, so round k+1 cannot overwrite what is being summed here)
     if (blockIdx.x == 0) sum_partials(partials, (double)p.inv_M, mp.tel + 2 * slot, s_red);

@@ -377,3 +377,35 @@ def test_sparse_graph_with_clustered_centres(nm):
     assert e.value.code == -2                              # Eq. 12: no probability on a missing link
     g.close()
     h.close()
+
+
+def test_a_barrier_wait_that_runs_out_is_reported_and_the_context_survives(nm):
+    """The multi-round launch polls its grid barrier a bounded number of times.  Made to wait for
+    CTAs that do not exist, it gives up, the next synchronising call reports the error, and the
+    same context then runs correctly again (no fault, no hang)."""
+    import time
+    M, d = 4, 4096
+    rng = np.random.default_rng(33)
+    P = random_policy(M, rng)
+    x0 = rng.standard_normal((M, d)).astype(np.float32)
+    kw = dict(M=M, d=d, lr=0.05, prob=P, sigma=0.1, c_std=1.0, seed=3)
+    g, ref = nm.Netmax(**kw), nm.Netmax(**kw)
+    g.set_replicas(x0)
+    g.debug_absent_ctas(1)
+    t0 = time.perf_counter()
+    g.round(5)
+    with pytest.raises(nm.NetmaxError) as e:
+        g.read_replicas()
+    assert e.value.code == -4 and "barrier" in str(e.value)
+    assert time.perf_counter() - t0 < 60.0
+    # the context is still usable: rounds 5.. from a fresh state equal an undisturbed context's
+    g.set_replicas(x0)
+    ref.set_replicas(x0)
+    ref.round(5)
+    ref.set_replicas(x0)
+    g.round(6)
+    ref.round(6)
+    assert (g.read_replicas() == ref.read_replicas()).all()
+    assert (g.peer_trace(5, 6) == ref.peer_trace(5, 6)).all()
+    g.close()
+    ref.close()
