@@ -409,3 +409,19 @@ def test_a_barrier_wait_that_runs_out_is_reported_and_the_context_survives(nm):
     assert (g.peer_trace(5, 6) == ref.peer_trace(5, 6)).all()
     g.close()
     ref.close()
+
+
+def test_fast_gaussian_noise_stays_within_its_error_bound(nm):
+    """The kernel's normals (hardware lg2 / sqrt / sin / cos approximations) against the oracle's
+    fp64 Box-Muller on the same Philox words: with x = c = 0 and self-draws only, one round leaves
+    x' = -alpha sigma z.  Typical error ~2e-7; the bound for radii below 1e-3 is 6e-4."""
+    M, d, lr, sigma = 2, 2_000_003, 0.5, 0.5
+    g = nm.Netmax(M=M, d=d, lr=lr, prob=np.eye(M), rho=0.1, sigma=sigma, objective=1, seed=123)
+    g.round(1)
+    z_gpu = -g.read_replicas().astype(np.float64) / (lr * sigma)
+    err = np.concatenate([np.abs(z_gpu[i] - oracle.noise(123, i, 0, 0, d)) for i in range(M)])
+    assert err.max() < 6e-4
+    assert np.quantile(err, 0.9999) < 3e-6
+    assert np.median(err) < 2e-7
+    assert abs(z_gpu.mean()) < 4.0 / np.sqrt(z_gpu.size) and abs(z_gpu.var() - 1.0) < 4.0 * np.sqrt(2.0 / z_gpu.size)
+    g.close()
