@@ -127,7 +127,12 @@ int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
  * Runs n_rounds rounds (n_rounds >= 0), asynchronously on the context's stream.  Per round:
  * the peer of every worker is drawn (Algorithm 2), then ONE fused kernel applies Eq. 15 and
  * Eq. 16 to every element of every replica, reading the round-start buffer and writing the
- * other one, and reduces that round's telemetry.
+ * other one, and reduces that round's telemetry.  The peers of up to trace_rounds rounds are
+ * drawn ahead in one sampler launch (the draws are counter-based and do not depend on x).
+ * Short vectors (a round of a few microseconds) run all rounds of a call in one cooperative
+ * launch with a grid-wide barrier per round; its waits are bounded, and one that runs out is
+ * reported by the next synchronising call as NETMAX_CUDA_ERROR (the replicas are then not
+ * valid).  Either way the results are the same, bit for bit, however a run is split into calls.
  */
 int netmax_round(netmax_ctx* ctx, int64_t n_rounds);
 

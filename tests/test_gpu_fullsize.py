@@ -113,3 +113,67 @@ def test_full_size_sampling_stress_config(nm):
     g.round(1)
     assert g.telemetry(rounds, 1)[0][0] == pytest.approx(want_cons, rel=1e-4)
     g.close()
+
+
+def test_maximum_vector_length(nm):
+    """d just below the limit (a padded row of 2^32 - 128 bytes), odd so that the tail is ragged:
+    every 64-bit offset, the ragged last group and the last elements of the rows are exercised.
+    26 GB of device memory; the oracle follows a sample of columns."""
+    import torch
+    d, M = (1 << 30) - 33, 2
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * (1 << 30):
+        pytest.skip("needs 40 GB of free device memory")
+    P = np.array([[0.1, 0.9], [0.7, 0.3]])
+    adj = (1 - np.eye(M)).astype(np.uint8)
+    cols = workloads.sample_columns(d, 3000, 77)
+    assert cols[-1] == d - 1
+    g = nm.Netmax(M=M, d=d, lr=0.1, prob=P, sigma=0.05, x0_std=1.0, c_std=1.0, objective=1, seed=77, trace_rounds=8)
+    _, rho = g.get_policy()
+    o = oracle.Sim(M, d, P, adj, alpha=0.1, rho=rho, sigma=0.05, objective=1, seed=77, cols=cols)
+    o.init(1.0, 1.0)
+    g.round(3)
+    o.round(3)
+    assert (g.peer_trace() == o.trace()).all()
+    assert_replicas_close(g.read_columns(cols), o.x())
+    ptr, ld = g.replicas_device()
+    assert ld * 4 == (1 << 32) - 128
+    pad = _as_tensor(ptr, M, ld)[:, d:]
+    assert pad.numel() == M * (ld - d) and float(pad.abs().max().item()) == 0.0      # padding stays zero
+    want_cons = telemetry_from_device(g)
+    g.round(1)
+    assert g.telemetry(3, 1)[0][0] == pytest.approx(want_cons, rel=1e-4)
+    g.close()
+    torch.cuda.empty_cache()
+    with pytest.raises(nm.NetmaxError) as e:
+        nm.Netmax(M=M, d=(1 << 30) - 32, lr=0.1, prob=P)
+    assert e.value.code == -1
+
+
+def test_maximum_worker_count(nm):
+    """M at its limit (16384 workers, 1 GB threshold table, 1 GB weight table), short vectors."""
+    M, d, rounds = 16384, 8, 3
+    rng = np.random.default_rng(5)
+    P = rng.random((M, M), dtype=np.float32).astype(np.float64)
+    P[rng.random((M, M), dtype=np.float32) < 0.5] = 0.0
+    P[np.arange(M), (np.arange(M) + 1) % M] = 1.0
+    np.fill_diagonal(P, 0.0)
+    P /= P.sum(axis=1, keepdims=True)
+    adj = np.ones((M, M), dtype=np.uint8)
+    np.fill_diagonal(adj, 0)
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=1, seed=9, trace_rounds=4)
+    _, rho = g.get_policy()
+    o = oracle.Sim(M, d, P, adj, alpha=0.05, rho=rho, sigma=0.1, objective=1, seed=9)
+    o.init(1.0, 1.0)
+    g.round(rounds)
+    o.round(rounds)
+    assert (g.peer_trace() == o.trace()).all()
+    assert_replicas_close(g.read_replicas(), o.x())
+    gc, gl = g.telemetry()
+    oc, ol = o.telemetry()
+    np.testing.assert_allclose(gc, oc, rtol=1e-4)
+    np.testing.assert_allclose(gl, ol, rtol=1e-4)
+    g.close()
+    with pytest.raises(nm.NetmaxError) as e:
+        nm.Netmax(M=M + 1, d=d, lr=0.05)
+    assert e.value.code == -1
