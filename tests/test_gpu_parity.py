@@ -425,3 +425,29 @@ def test_fast_gaussian_noise_stays_within_its_error_bound(nm):
     assert np.median(err) < 2e-7
     assert abs(z_gpu.mean()) < 4.0 / np.sqrt(z_gpu.size) and abs(z_gpu.var() - 1.0) < 4.0 * np.sqrt(2.0 / z_gpu.size)
     g.close()
+
+
+def test_short_form_create(nm):
+    """netmax_create(M, d, link_speed, prob, lr, seed): objective 1, sigma 0, unit-variance start."""
+    import ctypes as C
+    M, d = 4, 777
+    P = random_policy(M, np.random.default_rng(44))
+    L = nm.lib()
+    h = C.c_void_p()
+    assert L.netmax_create(M, d, None, P.ctypes.data_as(C.c_void_p), 0.05, 1234, C.byref(h)) == 0
+    assert L.netmax_round(h, 9) == 0 and L.netmax_rounds_done(h) == 9
+    out = np.empty((M, d), dtype=np.float32)
+    assert L.netmax_read_replicas(h, out.ctypes.data_as(C.c_void_p)) == 0
+    L.netmax_destroy(h)
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.0, x0_std=1.0, c_std=1.0, objective=1, seed=1234)
+    g.round(9)
+    assert (g.read_replicas() == out).all()
+    g.close()
+    # prob = NULL: Algorithm 3 on equal link speeds gives uniform neighbour choice
+    assert L.netmax_create(M, d, None, None, 0.05, 1, C.byref(h)) == 0
+    Pu = np.empty((M, M))
+    rho = C.c_double()
+    assert L.netmax_get_policy(h, Pu.ctypes.data_as(C.c_void_p), C.byref(rho)) == 0
+    off = ~np.eye(M, dtype=bool)
+    assert np.ptp(Pu[off]) < 1e-12 and rho.value > 0
+    L.netmax_destroy(h)
