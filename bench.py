@@ -163,10 +163,13 @@ def cpu_baseline(w, budget_s: float = 15.0):
     n_cols = int(min(w.d, max(probe_cols, rate * budget_s / (rounds * w.M))))
     per_round = time_oracle(w, n_cols, rounds, 1, threads)
     gbs = BYTES_PER_ELEMENT * w.M * n_cols / per_round / 1e9
+    one_cols = int(min(w.d, max(4096, rate / threads * 4.0 / (2 * w.M))))       # about 4 s on one thread
+    one = time_oracle(w, one_cols, 2, 1, 1)
     return {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",
             "sample": f"first {n_cols} of {w.d} columns of all {w.M} replicas, {rounds} rounds, "
                       f"{threads} threads over column blocks",
-            "rounds_per_s_extrapolated": n_cols / per_round / w.d}
+            "rounds_per_s_extrapolated": n_cols / per_round / w.d,
+            "value_1_thread": BYTES_PER_ELEMENT * w.M * one_cols / one / 1e9}
 
 
 def run_reference(args, w):
@@ -271,6 +274,19 @@ def run_ours(args, w):
     sec = ms / 1e3
     value = BYTES_PER_ELEMENT * elements * world * args.steps / sec / 1e9
 
+    # five more untimed-by-the-contract repeats of a shorter run: best and median per round
+    rep_rounds = max(1, min(args.steps, 200))
+    rep_ms = []
+    for _ in range(5):
+        barrier()
+        with torch.cuda.stream(stream):
+            start.record()
+        g.round(rep_rounds)
+        with torch.cuda.stream(stream):
+            stop.record()
+        stop.synchronize()
+        rep_ms.append(start.elapsed_time(stop) / rep_rounds)
+
     # end to end through the C ABI with host buffers: upload x and c, one round, download x'
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     hx = torch.empty((w.M, w.d), dtype=torch.float32, pin_memory=True)
@@ -333,6 +349,9 @@ def run_ours(args, w):
                    "sigma": w.sigma, "policy": f"Algorithm 3, K={w.K}, R={w.R}, rho={rho:.6g}",
                    "sharding": "columns, no exchange" if world > 1 else "none",
                    "l2": "inputs larger than L2: each of x, x', c is %.0f MB" % (elements * 4 / 1e6)},
+        "repeats": {"rounds_each": rep_rounds, "ms_per_step_best": min(rep_ms),
+                    "ms_per_step_median": statistics.median(rep_ms)},
+        "hbm_footprint_bytes": int(size),
         "rounds_per_s": args.steps / sec, "peer_draws_per_s": w.M * world * args.steps / sec,
         "sampler_only_draws_per_s": sampler_draws_per_s,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
