@@ -392,7 +392,7 @@ int floor_pow2(int64_t v) {
 // Short vectors (fewer than two such tiles per SM; everything is L2-resident then): 128-byte
 // column segments where M allows, no idle row lanes, and the rows split into rg groups so that
 // about two CTAs per SM have work.
-int plan_round(netmax_ctx* ctx, RoundPlan& plan) {
+int plan_round(netmax_ctx* ctx, RoundPlan& plan, int objective) {
   const int64_t M = ctx->M, nq = ctx->L.nq;
   const int64_t target = 2 * (int64_t)ctx->sm_count;  // the short-vector kernel runs 2 CTAs per SM
   int cg = kThreads;
@@ -423,14 +423,14 @@ int plan_round(netmax_ctx* ctx, RoundPlan& plan) {
   plan.rows_per_group = (int)((M + rg - 1) / rg);
   plan.n_tiles = (nq + cg - 1) / cg * rg;
   plan.smem = align_up((size_t)M * 8, 16) + (plan.rl > 1 ? (size_t)kThreads * 32 : 0) + 64 * sizeof(double);
-  RoundKernel k = pick_kernel(ctx->objective, plan.short_vectors);
+  RoundKernel k = pick_kernel(objective, plan.short_vectors);
   if (plan.smem > 48 * 1024)
     NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
   int per_sm = 0;
   NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, plan.smem));
   if (per_sm < 1) return fail(ctx, NETMAX_CUDA_ERROR, "round kernel does not fit on an SM (smem %zu)", plan.smem);
   if (plan.short_vectors && ctx->cooperative) {  // the multi-round kernel needs all of its CTAs resident
-    MultiRoundKernel mk = pick_multi_kernel(ctx->objective);
+    MultiRoundKernel mk = pick_multi_kernel(objective == 2 ? 0 : objective);
     if (plan.smem > 48 * 1024)
       NM_CUDA(ctx, cudaFuncSetAttribute(mk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
     int per_sm_multi = 0;
@@ -688,7 +688,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   if ((uint64_t)(ctx->rounds + n_rounds) >= ((uint64_t)1 << 56)) return fail(ctx, NETMAX_INVALID_ARG, "round counter would exceed 2^56");
   DeviceGuard guard(ctx->device);
   RoundPlan plan;
-  int rc = plan_round(ctx, plan);
+  int rc = plan_round(ctx, plan, ctx->objective);
   if (rc) return rc;
   RoundKernel kernel = pick_kernel(ctx->objective, plan.short_vectors);
 
@@ -930,13 +930,10 @@ int netmax_sample_peers(netmax_ctx* ctx, int64_t first_round, int64_t n_rounds, 
 int netmax_measure(netmax_ctx* ctx, double* consensus, double* loss) {
   if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
   DeviceGuard guard(ctx->device);
-  const int saved = ctx->objective;
-  ctx->objective = 2;  // plan and pick the measuring instantiation
   RoundPlan plan;
-  int rc = plan_round(ctx, plan);
-  RoundKernel kernel = pick_kernel(2, plan.short_vectors);
-  ctx->objective = saved;
+  int rc = plan_round(ctx, plan, 2);  // 2: the measuring instantiation of the round kernel
   if (rc) return rc;
+  RoundKernel kernel = pick_kernel(2, plan.short_vectors);
   RoundParams p;
   std::memset(&p, 0, sizeof p);
   p.x_cur = reinterpret_cast<const float4*>(ctx->x[ctx->cur]);
