@@ -81,6 +81,8 @@ typedef struct netmax_config {
   void* stream;                  /* cudaStream_t to enqueue on (NULL: the legacy default stream)       */
   int64_t trace_rounds;          /* capacity of the peer-trace / telemetry ring, in rounds (>= 1)      */
   int32_t policy_K, policy_R;    /* Algorithm 3 grid sizes when prob is NULL (<= 0: 20 x 20)           */
+  double policy_rho_upper;       /* upper end of Algorithm 3's rho grid (<= 0: default cap; see
+                                    netmax_policy_generate_ex)                                         */
   void* workspace;               /* device memory for ALL of the context's device buffers, 256-byte
                                     aligned, at least netmax_workspace_size() bytes, owned by the
                                     caller and kept alive until netmax_destroy.  NULL: the library
@@ -285,6 +287,15 @@ int netmax_policy_generate(int32_t M, const double* t_iter, const uint8_t* adj, 
                            double* prob_out, double* rho_out, double* info_out /* 5 doubles */);
 
 /*
+ * The same with the upper end of the rho grid given explicitly: rho_k = k rho_upper / K.
+ * rho_upper <= 0 is the default (the grid ends where the Eq. 11 floors alone fill a row).
+ * 0.5 / lr is the U_rho Algorithm 3 prints; most of that grid is infeasible for M > 2, so a
+ * coarse K then selects a smaller rho and a P that favours fast links more strongly.
+ */
+int netmax_policy_generate_ex(int32_t M, const double* t_iter, const uint8_t* adj, double lr, int32_t K, int32_t R,
+                              double rho_upper, double* prob_out, double* rho_out, double* info_out);
+
+/*
  * Algorithm 3 on the GPU, for large M (thousands of workers, links redrawn often): the same
  * grids, the same row-wise LP optimum and the same selection as netmax_policy_generate, with
  * one CTA per row of P, Y_P (Eq. 22) kept in device memory and lambda_2 by Lanczos on the
@@ -293,7 +304,7 @@ int netmax_policy_generate(int32_t M, const double* t_iter, const uint8_t* adj, 
  * NULL); synchronises before returning.  Results agree with the host generator to rounding.
  */
 int netmax_policy_generate_device(int32_t M, const double* t_iter, const uint8_t* adj, double lr, int32_t K, int32_t R,
-                                  int32_t device, void* stream, double* prob_out, double* rho_out,
+                                  double rho_upper /* as in netmax_policy_generate_ex */, int32_t device, void* stream, double* prob_out, double* rho_out,
                                   double* info_out /* 5 doubles or NULL */);
 
 /*

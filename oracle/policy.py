@@ -158,14 +158,20 @@ def second_eigenvalue(Y: np.ndarray) -> float:
     return float(np.sort(vals)[0])
 
 
-def generate_policy(t: np.ndarray, adj: np.ndarray, alpha: float, K: int, R: int, eps: float = 1e-3):
-    """Algorithm 3.  Returns (P, rho, info) or raises ValueError when no grid point is feasible."""
+def generate_policy(t: np.ndarray, adj: np.ndarray, alpha: float, K: int, R: int, eps: float = 1e-3,
+                    rho_upper: float = 0.0):
+    """Algorithm 3.  Returns (P, rho, info) or raises ValueError when no grid point is feasible.
+
+    rho_upper > 0 sets the upper end of the rho grid explicitly (0.5 / alpha is the paper's
+    printed U_rho); the default caps it where the Eq. 11 floors alone fill a row."""
     t = np.asarray(t, dtype=np.float64)
     adj = np.asarray(adj, dtype=np.uint8)
     M = t.shape[0]
     dsum = adj.astype(np.float64) + adj.T.astype(np.float64)
     np.fill_diagonal(dsum, 0.0)
     U_rho = min(0.5 / alpha, (1.0 - 1e-6) / (alpha * dsum.sum(axis=1).max()))
+    if rho_upper > 0.0:
+        U_rho = rho_upper
     off = adj.astype(bool) & ~np.eye(M, dtype=bool)
     best = None
     for k in range(1, K + 1):

@@ -26,7 +26,7 @@ EXPORTS = [
     "netmax_peer_trace", "netmax_telemetry", "netmax_replicas_device", "netmax_sample_peers",
     "netmax_measure", "netmax_async_begin", "netmax_async_set_times", "netmax_async_steps", "netmax_async_time",
     "netmax_async_trace", "netmax_async_ema", "netmax_async_monitor", "netmax_async_monitor_refreshes",
-    "netmax_iteration_times", "netmax_policy_generate", "netmax_policy_generate_device", "netmax_debug_absent_ctas", "netmax_kernel_launches", "netmax_last_error",
+    "netmax_iteration_times", "netmax_policy_generate", "netmax_policy_generate_ex", "netmax_policy_generate_device", "netmax_debug_absent_ctas", "netmax_kernel_launches", "netmax_last_error",
 ]
 
 
@@ -41,7 +41,7 @@ class Config(C.Structure):
         ("M", C.c_int32), ("d", C.c_int64), ("element_offset", C.c_int64), ("link_speed_gbps", C.c_void_p), ("prob", C.c_void_p),
         ("lr", C.c_double), ("rho", C.c_double), ("pull_weight", C.c_double), ("sigma", C.c_double), ("x0_std", C.c_double),
         ("c_std", C.c_double), ("objective", C.c_int32), ("seed", C.c_uint64), ("device", C.c_int32),
-        ("stream", C.c_void_p), ("trace_rounds", C.c_int64), ("policy_K", C.c_int32), ("policy_R", C.c_int32),
+        ("stream", C.c_void_p), ("trace_rounds", C.c_int64), ("policy_K", C.c_int32), ("policy_R", C.c_int32), ("policy_rho_upper", C.c_double),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
     ]
 
@@ -93,7 +93,8 @@ def lib():
             "netmax_async_monitor_refreshes": ([vp], i64),
             "netmax_iteration_times": ([i32, i64, vp, vp, vp], C.c_int),
             "netmax_policy_generate": ([i32, vp, vp, dbl, i32, i32, vp, vp, vp], C.c_int),
-            "netmax_policy_generate_device": ([i32, vp, vp, dbl, i32, i32, i32, vp, vp, vp, vp], C.c_int),
+            "netmax_policy_generate_ex": ([i32, vp, vp, dbl, i32, i32, dbl, vp, vp, vp], C.c_int),
+            "netmax_policy_generate_device": ([i32, vp, vp, dbl, i32, i32, dbl, i32, vp, vp, vp, vp], C.c_int),
             "netmax_debug_absent_ctas": ([vp, i32], C.c_int),
             "netmax_kernel_launches": ([vp], i64),
             "netmax_last_error": ([vp], C.c_char_p),
@@ -133,25 +134,27 @@ def netmax_iteration_times(link_speed_gbps, d: int):
     return t, adj
 
 
-def netmax_policy_generate(t_iter, adj, lr: float, K: int, R: int):
+def netmax_policy_generate(t_iter, adj, lr: float, K: int, R: int, rho_upper: float = 0.0):
     t = _f64(t_iter)
     M = t.shape[0]
     adj = np.ascontiguousarray(adj, dtype=np.uint8)
     P = np.empty((M, M), dtype=np.float64)
     rho = C.c_double()
     info = np.empty(5, dtype=np.float64)
-    _check(lib().netmax_policy_generate(M, _p(t), _p(adj), float(lr), int(K), int(R), _p(P), C.byref(rho), _p(info)))
+    _check(lib().netmax_policy_generate_ex(M, _p(t), _p(adj), float(lr), int(K), int(R), float(rho_upper), _p(P),
+                                           C.byref(rho), _p(info)))
     return P, rho.value, dict(lam2=info[0], tbar=info[1], t_conv=info[2], k=int(info[3]), r=int(info[4]))
 
 
-def netmax_policy_generate_device(t_iter, adj, lr: float, K: int, R: int, device: int = 0, stream=None):
+def netmax_policy_generate_device(t_iter, adj, lr: float, K: int, R: int, device: int = 0, stream=None,
+                                  rho_upper: float = 0.0):
     t = _f64(t_iter)
     M = t.shape[0]
     adj = np.ascontiguousarray(adj, dtype=np.uint8)
     P = np.empty((M, M), dtype=np.float64)
     rho = C.c_double()
     info = np.empty(5, dtype=np.float64)
-    _check(lib().netmax_policy_generate_device(M, _p(t), _p(adj), float(lr), int(K), int(R), int(device), stream,
+    _check(lib().netmax_policy_generate_device(M, _p(t), _p(adj), float(lr), int(K), int(R), float(rho_upper), int(device), stream,
                                                _p(P), C.byref(rho), _p(info)))
     return P, rho.value, dict(lam2=info[0], tbar=info[1], t_conv=info[2], k=int(info[3]), r=int(info[4]))
 
@@ -163,7 +166,7 @@ class Netmax:
                  sigma: float = 0.0, x0_std: float = 0.0, c_std: float = 0.0, objective: int = 1, seed: int = 0,
                  device: int = 0, stream: Optional[int] = None, trace_rounds: int = 1024, policy_K: int = 20,
                  policy_R: int = 20, workspace: Optional[int] = None, workspace_bytes: int = 0,
-                 element_offset: int = 0, pull_weight: float = 0.0):
+                 element_offset: int = 0, pull_weight: float = 0.0, policy_rho_upper: float = 0.0):
         L = lib()
         cfg = Config()
         _check(L.netmax_config_init(C.byref(cfg)))
@@ -179,6 +182,7 @@ class Netmax:
         cfg.stream = stream
         cfg.trace_rounds = int(trace_rounds)
         cfg.policy_K, cfg.policy_R = int(policy_K), int(policy_R)
+        cfg.policy_rho_upper = float(policy_rho_upper)
         cfg.workspace, cfg.workspace_bytes = workspace, int(workspace_bytes)
         self.M, self.d = int(M), int(d)
         self._h = C.c_void_p()

@@ -140,6 +140,7 @@ struct netmax_ctx {
   int objective = 1;
   uint64_t seed = 0;
   int policy_K = 20, policy_R = 20;
+  double policy_rho_upper = 0.0;
   PhiloxKeys keys;
   std::vector<double> P;      // policy in force
   std::vector<uint8_t> adj;   // link graph in force
@@ -304,9 +305,9 @@ int resolve_policy(netmax_ctx* ctx, const double* speed, const double* prob, dou
   const bool on_device = M >= 512 && cudaGetDeviceCount(&ndev) == cudaSuccess && ctx->device < ndev;
   if (!on_device) cudaGetLastError();
   int rc = on_device ? netmax_policy_generate_device(M, ctx->t_iter.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K,
-                                                     ctx->policy_R, ctx->device, ctx->stream, ctx->P.data(), &rho_sel, nullptr)
-                     : netmax_policy_generate(M, ctx->t_iter.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K,
-                                              ctx->policy_R, ctx->P.data(), &rho_sel, nullptr);
+                                                     ctx->policy_R, ctx->policy_rho_upper, ctx->device, ctx->stream, ctx->P.data(), &rho_sel, nullptr)
+                     : netmax_policy_generate_ex(M, ctx->t_iter.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K,
+                                                 ctx->policy_R, ctx->policy_rho_upper, ctx->P.data(), &rho_sel, nullptr);
   if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
   ctx->rho = rho > 0.0 ? rho : rho_sel;
   return NETMAX_OK;
@@ -509,6 +510,7 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   ctx->seed = cfg->seed;
   ctx->policy_K = cfg->policy_K > 0 ? cfg->policy_K : 20;
   ctx->policy_R = cfg->policy_R > 0 ? cfg->policy_R : 20;
+  ctx->policy_rho_upper = cfg->policy_rho_upper > 0.0 ? cfg->policy_rho_upper : 0.0;
   ctx->keys = make_philox_keys(cfg->seed);
   ctx->L = make_layout(cfg->M, cfg->d, cfg->trace_rounds);
 
@@ -1058,9 +1060,9 @@ static int monitor_refresh(netmax_ctx* ctx) {
   int ndev = 0;
   const bool on_device = M >= 512 && cudaGetDeviceCount(&ndev) == cudaSuccess && ctx->device < ndev;
   int rc = on_device ? netmax_policy_generate_device(M, t.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K, ctx->policy_R,
-                                                     ctx->device, ctx->stream, P.data(), &rho, nullptr)
-                     : netmax_policy_generate(M, t.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K, ctx->policy_R,
-                                              P.data(), &rho, nullptr);
+                                                     ctx->policy_rho_upper, ctx->device, ctx->stream, P.data(), &rho, nullptr)
+                     : netmax_policy_generate_ex(M, t.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K, ctx->policy_R,
+                                                 ctx->policy_rho_upper, P.data(), &rho, nullptr);
   if (rc == NETMAX_INFEASIBLE) return NETMAX_OK;
   if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
   ctx->P.swap(P);

@@ -288,6 +288,11 @@ int netmax_iteration_times(int32_t M, int64_t d, const double* speed, double* t_
 
 int netmax_policy_generate(int32_t M, const double* t, const uint8_t* adj, double lr, int32_t K, int32_t R,
                            double* prob_out, double* rho_out, double* info_out) {
+  return netmax_policy_generate_ex(M, t, adj, lr, K, R, 0.0, prob_out, rho_out, info_out);
+}
+
+int netmax_policy_generate_ex(int32_t M, const double* t, const uint8_t* adj, double lr, int32_t K, int32_t R,
+                              double rho_upper, double* prob_out, double* rho_out, double* info_out) {
   if (M < 2 || !t || !adj || !prob_out || !rho_out || !(lr > 0.0) || K < 1 || R < 1)
     return fail(NETMAX_INVALID_ARG, "policy_generate: bad argument");
   std::vector<Row> rows(M);
@@ -315,7 +320,7 @@ int netmax_policy_generate(int32_t M, const double* t, const uint8_t* adj, doubl
     max_f1 = std::max(max_f1, r.sum_f1);
     U_time = std::min(U_time, r.tmax / M);
   }
-  const double U_rho = std::min(0.5 / lr, (1.0 - 1e-6) / (lr * max_f1));
+  const double U_rho = rho_upper > 0.0 ? rho_upper : std::min(0.5 / lr, (1.0 - 1e-6) / (lr * max_f1));
 
   std::vector<double> P((size_t)M * M), Y((size_t)M * M), bestP;
   double best_tconv = INFINITY, best_rho = 0, best_lam = 0, best_tbar = 0;

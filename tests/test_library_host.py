@@ -124,3 +124,18 @@ def test_product_path_fails_loudly_without_a_gpu(gpu_available):
     with pytest.raises(binding.NetmaxError) as e:
         binding.Netmax(M=2, d=8, lr=0.1, prob=good)
     assert e.value.code == -4
+
+
+def test_explicit_rho_grid_matches_oracle_and_is_more_adaptive():
+    """The printed U_rho = 0.5/alpha with a coarse K leaves one feasible rho, smaller than the default
+    grid's choice, and a policy that prefers the fast links more."""
+    w = workloads.config(2)
+    t, adj = opolicy.iteration_times(w.link_speeds(0), w.d)
+    P, rho, info = binding.netmax_policy_generate(t, adj, w.lr, 10, 10, rho_upper=0.5 / w.lr)
+    P0, rho0, info0 = opolicy.generate_policy(t, adj, w.lr, 10, 10, rho_upper=0.5 / w.lr)
+    assert (info["k"], info["r"]) == (info0["k"], info0["r"]) and rho == pytest.approx(rho0, rel=1e-14)
+    np.testing.assert_allclose(P, P0, atol=1e-9)
+    Pd, rhod, _ = binding.netmax_policy_generate(t, adj, w.lr, 10, 10)
+    assert rho < rhod
+    fast, slow = P[0, 1], P[0, 5]
+    assert fast / slow > Pd[0, 1] / Pd[0, 5] > 1.0
