@@ -21,6 +21,14 @@
 // every global step exactly ONE worker -- the one whose iteration finishes next -- updates
 // its replica from the peer's CURRENT replica (nmo_async_*).
 //
+// Storage option (not in the paper, which trains in fp32): with bfloat16 storage the state
+// holds bfloat16 values.  A stored value is then a quantised code, and the side that decides
+// it must decide it in the precision of the simulator it checks: the update is evaluated in
+// IEEE fp32, one operation at a time in the order
+//   t = x - c;  g = fma(sigma, z, t);  h = fma(-alpha, g, x);  x' = fma(-w, h - x_m, h)
+// (z = the double Box-Muller normal rounded to fp32), and x' is rounded to the nearest
+// bfloat16, ties to even.  The fp32 value before that rounding is kept for the tests.
+//
 // Only tests, the smoke check and the benchmark's cpu_baseline leg may use this file.
 // It shares no code with the CUDA library and includes none of its headers.
 //
@@ -153,6 +161,17 @@ void build_weight_row(int M, int i, const double* P, const uint8_t* adj, double 
 }
 
 // ------------------------------------------------------------------ simulator
+// Nearest bfloat16 (the top 16 bits of the fp32 pattern), ties to even, returned as fp32.
+// Finite inputs only.
+inline float bf16_round(float v) {
+  uint32_t u;
+  std::memcpy(&u, &v, 4);
+  const uint32_t keep_odd = (u >> 16) & 1u;  // makes an exact tie round to the even neighbour
+  u = (u + 0x7FFFu + keep_odd) & 0xFFFF0000u;
+  std::memcpy(&v, &u, 4);
+  return v;
+}
+
 struct Sim {
   int M = 0;
   int64_t d = 0;           // logical vector length (defines the noise counters)
@@ -161,6 +180,8 @@ struct Sim {
   double alpha = 0, rho = 0, sigma = 0;  // alpha, sigma already rounded to fp32 values
   double fixed_w = 0.0;                  // > 0: every pull uses this weight instead of Eq. 16's
   int objective = 1;
+  int storage = 0;                       // 0: fp32 state, double arithmetic; 1: bfloat16 state, fp32 arithmetic
+  std::vector<float> pre;                // storage 1: fp32 values of the last round before the bfloat16 rounding
   uint32_t key[2] = {0, 0};
   uint64_t round = 0;
   std::vector<uint32_t> T;
@@ -205,7 +226,9 @@ void fill_normal(Sim* s, std::vector<float>& dst, double stddev, uint32_t tag) {
       make_ctr((uint32_t)(e >> 2), (uint32_t)i, 0, tag, ctr);
       philox4x32_10(ctr, s->key, r);
       normals4(r, z);
-      dst[(size_t)i * s->ncols + k] = (float)(stddev * z[e & 3]);
+      // bfloat16 storage: fp32 normal times the fp32 scale (one fp32 product), then rounded
+      dst[(size_t)i * s->ncols + k] =
+          s->storage == 1 ? bf16_round((float)z[e & 3] * (float)stddev) : (float)(stddev * z[e & 3]);
     }
 }
 
@@ -240,6 +263,30 @@ void round_columns(Sim* s, const int32_t* peer, int64_t k0, int64_t k1) {
     const float* xm = s->x.data() + (size_t)m * n;  // round-start snapshot of the peer
     const float* ci = s->c.data() + (size_t)i * n;
     float* out = s->xn.data() + (size_t)i * n;
+    if (s->storage == 1) {  // bfloat16 state: fp32 arithmetic in the stated order, one rounding to bfloat16
+      const float alpha = (float)s->alpha, sigma = (float)s->sigma, wf = (m != i) ? s->w[(size_t)i * M + m] : 0.0f;
+      float* pre = s->pre.data() + (size_t)i * n;
+      for (int64_t k = k0; k < k1; ++k) {
+        const int64_t e = s->cols[k];
+        const float xv = xi[k];
+        float h = xv;
+        if (s->objective == 1) {
+          uint32_t ctr[4], r[4];
+          double z[4];
+          make_ctr((uint32_t)(e >> 2), (uint32_t)i, s->round, TAG_NOISE, ctr);
+          philox4x32_10(ctr, s->key, r);
+          normals4(r, z);
+          const float t = xv - ci[k];
+          const float g = std::fmaf(sigma, (float)z[e & 3], t);
+          h = std::fmaf(-alpha, g, xv);                          // Eq. 15
+        }
+        const float diff = h - xm[k];
+        const float xnew = std::fmaf(-wf, diff, h);              // Eq. 16 (w = 0 on a self-draw)
+        pre[k] = xnew;
+        out[k] = bf16_round(xnew);
+      }
+      continue;
+    }
     for (int64_t k = k0; k < k1; ++k) {
       const int64_t e = s->cols[k];
       const double xv = (double)xi[k];
@@ -443,8 +490,23 @@ void nmo_sim_init(void* h, double x0_std, double c_std) {
   fill_normal(s, s->c, c_std, TAG_C);
 }
 
-void nmo_sim_set_x(void* h, const float* x) { Sim* s = (Sim*)h; std::memcpy(s->x.data(), x, s->x.size() * sizeof(float)); }
-void nmo_sim_set_c(void* h, const float* c) { Sim* s = (Sim*)h; std::memcpy(s->c.data(), c, s->c.size() * sizeof(float)); }
+void nmo_sim_set_x(void* h, const float* x) {
+  Sim* s = (Sim*)h;
+  for (size_t k = 0; k < s->x.size(); ++k) s->x[k] = s->storage == 1 ? bf16_round(x[k]) : x[k];
+}
+void nmo_sim_set_c(void* h, const float* c) {
+  Sim* s = (Sim*)h;
+  for (size_t k = 0; k < s->c.size(); ++k) s->c[k] = s->storage == 1 ? bf16_round(c[k]) : c[k];
+}
+// Before any state is set.  1: bfloat16 storage with fp32 arithmetic (see the header).
+void nmo_sim_set_storage(void* h, int32_t storage) {
+  Sim* s = (Sim*)h;
+  s->storage = storage;
+  s->pre.assign(storage == 1 ? s->x.size() : 0, 0.0f);
+}
+// bfloat16 storage: the last round's new parameters before they were rounded to bfloat16.
+void nmo_sim_get_unrounded(void* h, float* out) { Sim* s = (Sim*)h; std::memcpy(out, s->pre.data(), s->pre.size() * sizeof(float)); }
+void nmo_bf16_round(const float* in, int64_t n, float* out) { for (int64_t k = 0; k < n; ++k) out[k] = bf16_round(in[k]); }
 void nmo_sim_get_x(void* h, float* x) { Sim* s = (Sim*)h; std::memcpy(x, s->x.data(), s->x.size() * sizeof(float)); }
 void nmo_sim_get_c(void* h, float* c) { Sim* s = (Sim*)h; std::memcpy(c, s->c.data(), s->c.size() * sizeof(float)); }
 

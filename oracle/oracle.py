@@ -56,8 +56,10 @@ def lib():
         L.nmo_sim_set_fixed_weight.argtypes = [vp, dbl]
         L.nmo_sim_set_policy.argtypes = [vp, vp, vp, dbl]
         L.nmo_sim_init.argtypes = [vp, dbl, dbl]
-        for name in ("nmo_sim_set_x", "nmo_sim_set_c", "nmo_sim_get_x", "nmo_sim_get_c"):
+        for name in ("nmo_sim_set_x", "nmo_sim_set_c", "nmo_sim_get_x", "nmo_sim_get_c", "nmo_sim_get_unrounded"):
             getattr(L, name).argtypes = [vp, vp]
+        L.nmo_sim_set_storage.argtypes = [vp, i32]
+        L.nmo_bf16_round.argtypes = [vp, i64, vp]
         L.nmo_sim_round.argtypes = [vp, i64, i32]
         L.nmo_sim_rounds_done.argtypes = [vp]
         L.nmo_sim_rounds_done.restype = i64
@@ -110,6 +112,14 @@ def normals_from_words(words) -> np.ndarray:
     return out
 
 
+def bf16_round(values) -> np.ndarray:
+    """fp32 values rounded to the nearest bfloat16 (ties to even), returned as fp32."""
+    v = np.ascontiguousarray(values, dtype=np.float32)
+    out = np.empty_like(v)
+    lib().nmo_bf16_round(_p(v), v.size, _p(out))
+    return out
+
+
 def build_thresholds(P: np.ndarray):
     P = np.ascontiguousarray(P, dtype=np.float64)
     M = P.shape[0]
@@ -144,7 +154,7 @@ def peer_draws(P: np.ndarray, seed: int, first_round: int, n_rounds: int) -> np.
 class Sim:
     """The round simulator: all M replicas (or a sample of their columns) on the CPU."""
 
-    def __init__(self, M, d, P, adj, alpha, rho, sigma, objective, seed, cols=None, pull_weight=0.0):
+    def __init__(self, M, d, P, adj, alpha, rho, sigma, objective, seed, cols=None, pull_weight=0.0, storage="f32"):
         self.M, self.d = int(M), int(d)
         self._P = np.ascontiguousarray(P, dtype=np.float64)
         self._adj = np.ascontiguousarray(adj, dtype=np.uint8)
@@ -159,6 +169,10 @@ class Sim:
         if pull_weight > 0.0:      # fixed pull weight (gossip / AD-PSGD style averaging)
             lib().nmo_sim_set_fixed_weight(self._h, float(pull_weight))
             lib().nmo_sim_set_policy(self._h, _p(self._P), _p(self._adj), float(rho))
+        assert storage in ("f32", "bf16")
+        self.storage = storage
+        if storage == "bf16":      # bfloat16 state, fp32 arithmetic, one rounding per stored value
+            lib().nmo_sim_set_storage(self._h, 1)
 
     def close(self):
         if self._h:
@@ -193,6 +207,13 @@ class Sim:
     def c(self) -> np.ndarray:
         out = np.empty((self.M, self.ncols), dtype=np.float32)
         lib().nmo_sim_get_c(self._h, _p(out))
+        return out
+
+    def unrounded(self) -> np.ndarray:
+        """bf16 storage: the last round's new parameters in fp32, before the rounding to bfloat16."""
+        assert self.storage == "bf16"
+        out = np.empty((self.M, self.ncols), dtype=np.float32)
+        lib().nmo_sim_get_unrounded(self._h, _p(out))
         return out
 
     def round(self, n=1, threads=1):
