@@ -36,6 +36,7 @@ import numpy as np  # noqa: E402
 from paper_2009_05766_b200 import workloads  # noqa: E402
 
 BYTES_PER_ELEMENT = 16          # x_i, x_peer, c_i read + x_i' written, fp32
+BYTES_PER_ELEMENT_BF16 = 8      # the same four accesses with bfloat16 storage
 FALLBACK_HBM_GBS = 6650.0
 KERNEL_SOURCES = ("netmax_kernels.cuh", "netmax_rng.cuh")
 # dram__bytes_read.sum + dram__bytes_write.sum of one round-kernel launch, from an ncu capture
@@ -139,12 +140,13 @@ def oracle_policy_inputs(w):
     return P, rho, adj
 
 
-def time_oracle(w, n_cols: int, rounds: int, warm: int, threads: int):
+def time_oracle(w, n_cols: int, rounds: int, warm: int, threads: int, storage: str = "f32"):
     """Seconds per round of the oracle on the first n_cols columns of all M replicas."""
     from oracle import oracle
     P, rho, adj = oracle_policy_inputs(w)
     cols = np.arange(n_cols, dtype=np.int64)
-    sim = oracle.Sim(w.M, w.d, P, adj, alpha=w.lr, rho=rho, sigma=w.sigma, objective=1, seed=w.seed, cols=cols)
+    sim = oracle.Sim(w.M, w.d, P, adj, alpha=w.lr, rho=rho, sigma=w.sigma, objective=1, seed=w.seed, cols=cols,
+                     storage=storage)
     sim.init(w.x0_std, w.c_std)
     sim.round(warm, threads=threads)
     t0 = time.perf_counter()
@@ -154,22 +156,23 @@ def time_oracle(w, n_cols: int, rounds: int, warm: int, threads: int):
     return dt
 
 
-def cpu_baseline(w, budget_s: float = 15.0):
+def cpu_baseline(w, budget_s: float = 15.0, storage: str = "f32"):
     threads = max(1, min(os.cpu_count() or 1, 64))
+    bpe = BYTES_PER_ELEMENT_BF16 if storage == "bf16" else BYTES_PER_ELEMENT
     probe_cols = int(min(w.d, max(4096, 200_000 // w.M)))
-    per_round = time_oracle(w, probe_cols, 2, 1, threads)
+    per_round = time_oracle(w, probe_cols, 2, 1, threads, storage)
     rate = w.M * probe_cols / per_round                       # elements per second
     rounds = 5
     n_cols = int(min(w.d, max(probe_cols, rate * budget_s / (rounds * w.M))))
-    per_round = time_oracle(w, n_cols, rounds, 1, threads)
-    gbs = BYTES_PER_ELEMENT * w.M * n_cols / per_round / 1e9
+    per_round = time_oracle(w, n_cols, rounds, 1, threads, storage)
+    gbs = bpe * w.M * n_cols / per_round / 1e9
     one_cols = int(min(w.d, max(4096, rate / threads * 4.0 / (2 * w.M))))       # about 4 s on one thread
-    one = time_oracle(w, one_cols, 2, 1, 1)
+    one = time_oracle(w, one_cols, 2, 1, 1, storage)
     return {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",
             "sample": f"first {n_cols} of {w.d} columns of all {w.M} replicas, {rounds} rounds, "
                       f"{threads} threads over column blocks",
             "rounds_per_s_extrapolated": n_cols / per_round / w.d,
-            "value_1_thread": BYTES_PER_ELEMENT * w.M * one_cols / one / 1e9}
+            "value_1_thread": bpe * w.M * one_cols / one / 1e9}
 
 
 def run_reference(args, w):
@@ -179,18 +182,19 @@ def run_reference(args, w):
         return
     threads = max(1, min(os.cpu_count() or 1, 64))
     probe_cols = int(min(w.d, max(4096, 200_000 // w.M)))
-    per_round = time_oracle(w, probe_cols, 2, 1, threads)
+    bpe = BYTES_PER_ELEMENT_BF16 if args.storage == "bf16" else BYTES_PER_ELEMENT
+    per_round = time_oracle(w, probe_cols, 2, 1, threads, args.storage)
     rate = w.M * probe_cols / per_round
     budget = 90.0
     n_cols = int(min(w.d, max(1024, rate * budget / ((args.steps + args.warmup) * w.M))))
-    per_round = time_oracle(w, n_cols, args.steps, args.warmup, threads)
-    gbs = BYTES_PER_ELEMENT * w.M * n_cols / per_round / 1e9
+    per_round = time_oracle(w, n_cols, args.steps, args.warmup, threads, args.storage)
+    gbs = bpe * w.M * n_cols / per_round / 1e9
     sample = (f"first {n_cols} of {w.d} columns of all {w.M} replicas per step, {threads} threads")
     line = {
         "impl": "reference", "metric": "replica GB/s", "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_round * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "M": w.M, "d": w.d, "sample": sample},
+        "config": {"workload": w.name, "M": w.M, "d": w.d, "storage": args.storage, "sample": sample},
         "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -199,10 +203,11 @@ def run_reference(args, w):
 
 
 # ---------------------------------------------------------------------------- GPU arm
-def shard_plan(d: int, world: int, rank: int):
+def shard_plan(d: int, world: int, rank: int, align: int = 4):
     """Weak scaling by columns: rank g holds logical elements [g*d4, g*d4 + d) of a world*d4-long
-    vector, d4 = d rounded up to a multiple of 4 (counter alignment)."""
-    d4 = (d + 3) // 4 * 4
+    vector, d4 = d rounded up to a multiple of `align` (counter alignment: 4 elements per Philox
+    block; 8 with bfloat16 storage, whose 16-byte column groups hold two blocks)."""
+    d4 = (d + align - 1) // align * align
     return {"element_offset": rank * d4, "d": d, "global_d": world * d4}
 
 
@@ -219,7 +224,7 @@ def run_ours(args, w):
 
     base = None
     if rank == 0 and not args.no_cpu_baseline:
-        base = cpu_baseline(w)          # before the first CUDA call
+        base = cpu_baseline(w, storage=args.storage)          # before the first CUDA call
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
@@ -234,16 +239,18 @@ def run_ours(args, w):
     generate = binding.netmax_policy_generate_device if w.M >= 512 else binding.netmax_policy_generate
     P, rho, pinfo = generate(t_iter, adj, w.lr, w.K, w.R)
 
-    plan = shard_plan(w.d, world, rank)
+    bf16 = args.storage == "bf16"
+    bytes_per_element = BYTES_PER_ELEMENT_BF16 if bf16 else BYTES_PER_ELEMENT
+    plan = shard_plan(w.d, world, rank, 8 if bf16 else 4)
     stream = torch.cuda.Stream()
     ring = 1024
-    size = binding.Netmax.workspace_size(w.M, w.d, ring)
+    size = binding.Netmax.workspace_size(w.M, w.d, ring, storage=args.storage)
     ws = torch.empty(size + 256, dtype=torch.uint8, device="cuda")       # device memory from PyTorch
     ws_ptr = (ws.data_ptr() + 255) // 256 * 256
     g = binding.Netmax(M=w.M, d=w.d, lr=w.lr, link_speed_gbps=speeds, prob=P, rho=rho, sigma=w.sigma,
                        x0_std=w.x0_std, c_std=w.c_std, objective=1, seed=w.seed, device=local,
                        stream=stream.cuda_stream, trace_rounds=ring, workspace=ws_ptr, workspace_bytes=size,
-                       element_offset=plan["element_offset"])
+                       element_offset=plan["element_offset"], storage=args.storage)
 
     def barrier():
         torch.cuda.synchronize()
@@ -272,7 +279,7 @@ def run_ours(args, w):
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         ms = float(tmax.item())
     sec = ms / 1e3
-    value = BYTES_PER_ELEMENT * elements * world * args.steps / sec / 1e9
+    value = bytes_per_element * elements * world * args.steps / sec / 1e9
 
     # five more untimed-by-the-contract repeats of a shorter run: best and median per round
     rep_rounds = max(1, min(args.steps, 200))
@@ -319,7 +326,7 @@ def run_ours(args, w):
         tmax = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         e2e_ms = float(tmax.item())
-    e2e_value = BYTES_PER_ELEMENT * elements * world * e2e_steps / (e2e_ms / 1e3) / 1e9
+    e2e_value = bytes_per_element * elements * world * e2e_steps / (e2e_ms / 1e3) / 1e9
 
     # the sampler alone: one batched launch of 1024 rounds x M draws (Algorithm 2's peer selection)
     batch = 1024
@@ -339,16 +346,16 @@ def run_ours(args, w):
     cons, loss = g.telemetry(g.rounds_done - 1, 1)
     peak, peak_kind = measured_peak()
     per_launch_ms = ms / args.steps
-    achieved = BYTES_PER_ELEMENT * elements / (per_launch_ms / 1e3) / 1e9
-    traffic = NCU_TRAFFIC.get((kernel_source_hash(), w.name))
+    achieved = bytes_per_element * elements / (per_launch_ms / 1e3) / 1e9
+    traffic = NCU_TRAFFIC.get((kernel_source_hash(), w.name + ("/bf16" if bf16 else "")))
     line = {
         "metric": "replica GB/s", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": per_launch_ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "M": w.M, "d_per_gpu": w.d, "global_d": plan["global_d"], "lr": w.lr,
                    "sigma": w.sigma, "policy": f"Algorithm 3, K={w.K}, R={w.R}, rho={rho:.6g}",
-                   "sharding": "columns, no exchange" if world > 1 else "none",
-                   "l2": "inputs larger than L2: each of x, x', c is %.0f MB" % (elements * 4 / 1e6)},
+                   "sharding": "columns, no exchange" if world > 1 else "none", "storage": args.storage,
+                   "l2": "inputs larger than L2: each of x, x', c is %.0f MB" % (elements * bytes_per_element / 4 / 1e6)},
         "repeats": {"rounds_each": rep_rounds, "ms_per_step_best": min(rep_ms),
                     "ms_per_step_median": statistics.median(rep_ms)},
         "hbm_footprint_bytes": int(size),
@@ -356,7 +363,7 @@ def run_ours(args, w):
         "sampler_only_draws_per_s": sampler_draws_per_s,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "round_kernel",
-                     "bytes_per_launch": BYTES_PER_ELEMENT * elements,
+                     "bytes_per_launch": bytes_per_element * elements,
                      "frac_of_nominal_8TBs": achieved / 8000.0},
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": 2 * elements * 4,
                 "d2h_bytes_per_step": elements * 4, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
@@ -391,7 +398,9 @@ def run_async(args, w):
     P, rho, _ = binding.netmax_policy_generate(t_iter, adj, w.lr, w.K, w.R)
     stream = torch.cuda.Stream()
     g = binding.Netmax(M=w.M, d=w.d, lr=w.lr, link_speed_gbps=speeds, prob=P, rho=rho, sigma=w.sigma,
-                       x0_std=w.x0_std, c_std=w.c_std, objective=1, seed=w.seed, stream=stream.cuda_stream)
+                       x0_std=w.x0_std, c_std=w.c_std, objective=1, seed=w.seed, stream=stream.cuda_stream,
+                       storage=args.storage)
+    bytes_per_element = BYTES_PER_ELEMENT_BF16 if args.storage == "bf16" else BYTES_PER_ELEMENT
     g.async_begin(None, 0.9)
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     g.async_steps(max(args.warmup, 3) * w.M)
@@ -409,18 +418,19 @@ def run_async(args, w):
     sim_time, steps_done = g.async_time()
     cons, loss = g.measure()
     peak, peak_kind = measured_peak()
-    achieved = BYTES_PER_ELEMENT * w.d * args.steps / (ms / 1e3) / 1e9
+    achieved = bytes_per_element * w.d * args.steps / (ms / 1e3) / 1e9
     line = {
         "metric": "replica GB/s", "value": achieved, "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
         "warmup": max(args.warmup, 3) * w.M, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name + ", asynchronous timeline (one worker per global step)", "M": w.M, "d": w.d,
-                   "l2": "each replica is %.0f MB; a step touches three of them" % (w.d * 4 / 1e6)},
+                   "storage": args.storage,
+                   "l2": "each replica is %.0f MB; a step touches three of them" % (w.d * bytes_per_element / 4 / 1e6)},
         "global_steps_per_s": args.steps / (ms / 1e3), "steps_per_launch": args.steps / max(launches, 1),
         "simulated_seconds": sim_time,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "step_kernel",
-                     "bytes_per_launch": BYTES_PER_ELEMENT * w.d * args.steps / max(launches, 1)},
+                     "bytes_per_launch": bytes_per_element * w.d * args.steps / max(launches, 1)},
         "gpu_launches": int(launches), "clocks": clocks.summary(),
         "telemetry_now": {"consensus": cons, "loss": loss},
     }
@@ -438,6 +448,8 @@ def main():
     ap.add_argument("--d", type=int, default=0, help="override the workload's vector length (profiling on a smaller case)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--storage", choices=["f32", "bf16"], default="f32",
+                    help="precision of the replicas in device memory (arithmetic is fp32 either way)")
     ap.add_argument("--mode", choices=["rounds", "async"], default="rounds",
                     help="rounds: synchronous rounds (default); async: the paper's one-worker-per-step timeline")
     args = ap.parse_args()

@@ -49,6 +49,19 @@ typedef enum netmax_status {
 typedef struct netmax_ctx netmax_ctx; /* opaque; created and destroyed by the library */
 
 /*
+ * Precision of the state kept in device memory (netmax_config.storage).  The paper trains in
+ * fp32, which is the default.  NETMAX_STORAGE_BF16 is an option of this library: replicas and
+ * centres are held as bfloat16 (half the memory and half the traffic per element), Eq. 15 and
+ * Eq. 16 are still evaluated in fp32, in the order
+ *   t = x - c;  g = fma(sigma, z, t);  h = fma(-alpha, g, x);  x' = fma(-w, h - x_m, h),
+ * and each new parameter is rounded once to the nearest bfloat16 (ties to even) when it is
+ * stored.  An update smaller than half a bfloat16 unit of the parameter is therefore lost --
+ * the known price of narrow storage.  Host-side arrays stay fp32 in every call: values passed
+ * in are rounded to bfloat16, values read back are widened exactly.
+ */
+enum { NETMAX_STORAGE_F32 = 0, NETMAX_STORAGE_BF16 = 1 };
+
+/*
  * Full configuration of a context (Algorithm 2's inputs alpha, rho and P, plus what the
  * simulator adds: sizes, the synthetic objective, the seed and where to run).
  */
@@ -56,7 +69,8 @@ typedef struct netmax_config {
   int32_t M;                     /* workers, 2 <= M <= 16384                                          */
   int64_t d;                     /* parameters per replica, 1 <= d < 2^30 - 32                        */
   int64_t element_offset;        /* logical index of this context's first element inside a longer global
-                                    vector (a multiple of 4, offset + d < 2^30 - 32; default 0).  Only the
+                                    vector (a multiple of 4 -- of 8 with bfloat16 storage --, offset + d <
+                                    2^30 - 32; default 0).  Only the
                                     noise / initialisation counters use it: contexts that hold disjoint
                                     column ranges of one problem (one per GPU) then draw the streams the
                                     single-context run would, and never need to exchange data            */
@@ -88,13 +102,15 @@ typedef struct netmax_config {
                                     caller and kept alive until netmax_destroy.  NULL: the library
                                     allocates with cudaMalloc and frees in netmax_destroy              */
   size_t workspace_bytes;
+  int32_t storage;               /* NETMAX_STORAGE_F32 (default) or NETMAX_STORAGE_BF16: see above       */
 } netmax_config;
 
 /* Fills *cfg with defaults: rho = 0 (automatic), sigma = 0, stds 0, objective 1, seed 0,
- * device 0, stream NULL, trace_rounds 1024, policy grid 20 x 20, no workspace, offset 0. */
+ * device 0, stream NULL, trace_rounds 1024, policy grid 20 x 20, no workspace, offset 0,
+ * fp32 storage. */
 int netmax_config_init(netmax_config* cfg);
 
-/* Device bytes a context with this M, d and trace_rounds needs (only those fields are read). */
+/* Device bytes a context with this M, d, trace_rounds and storage needs (only those fields are read). */
 int netmax_workspace_size(const netmax_config* cfg, size_t* bytes);
 
 /*
@@ -121,7 +137,9 @@ int netmax_set_policy(netmax_ctx* ctx, const double* link_speed_gbps, const doub
 /* Reads back the policy in force: prob_out (host, M*M) and *rho_out; either may be NULL. */
 int netmax_get_policy(netmax_ctx* ctx, double* prob_out, double* rho_out);
 
-/* Overwrite all replicas / all centres from dense host arrays of M*d floats. */
+/* Overwrite all replicas / all centres from dense host arrays of M*d floats.  A bfloat16
+ * context rounds them on the device; the buffer of the double buffer that holds no replicas
+ * at that moment is the staging area, so nothing is allocated. */
 int netmax_set_replicas(netmax_ctx* ctx, const float* host_x);
 int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
 
@@ -141,7 +159,8 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds);
 /* Number of rounds enqueued so far. */
 int64_t netmax_rounds_done(const netmax_ctx* ctx);
 
-/* Synchronises, then copies the current replicas to host_out (M*d floats, dense). */
+/* Synchronises, then copies the current replicas to host_out (M*d floats, dense; bfloat16
+ * state is widened exactly). */
 int netmax_read_replicas(netmax_ctx* ctx, float* host_out);
 /* Same for the centres c_i. */
 int netmax_read_centres(netmax_ctx* ctx, float* host_out);
@@ -258,7 +277,9 @@ int netmax_async_ema(netmax_ctx* ctx, double* ema_out, int64_t* samples_out);
 /*
  * Device access for callers that keep working on the GPU (for example through PyTorch):
  * *x is the buffer holding the current replicas, row i at x + i * ld, ld >= d floats,
- * valid until the next netmax_round / netmax_set_* call; nothing is synchronised.
+ * valid until the next netmax_round / netmax_set_* / netmax_read_replicas call; nothing is
+ * synchronised.  In a bfloat16 context the buffer holds bfloat16 values: cast the pointer;
+ * ld then counts bfloat16 elements.
  */
 int netmax_replicas_device(netmax_ctx* ctx, const float** x, int64_t* ld);
 

@@ -253,6 +253,26 @@ void telemetry(const Sim* s, double* consensus, double* loss) {
   *loss = ls / M;
 }
 
+// bfloat16 storage: Eq. 15 and Eq. 16 on one element in fp32, one operation at a time in the
+// order the header states; `iter` is the round (or the worker's local iteration on the
+// asynchronous timeline).  Returns the fp32 value before the rounding to bfloat16.
+float update_fp32(const Sim* s, int i, uint64_t iter, int64_t e, float xv, float cv, float xmv, float alpha, float sigma,
+                  float wf) {
+  float h = xv;
+  if (s->objective == 1) {
+    uint32_t ctr[4], r[4];
+    double z[4];
+    make_ctr((uint32_t)(e >> 2), (uint32_t)i, iter, TAG_NOISE, ctr);
+    philox4x32_10(ctr, s->key, r);
+    normals4(r, z);
+    const float t = xv - cv;
+    const float g = std::fmaf(sigma, (float)z[e & 3], t);
+    h = std::fmaf(-alpha, g, xv);  // Eq. 15
+  }
+  const float diff = h - xmv;
+  return std::fmaf(-wf, diff, h);  // Eq. 16 (w = 0 on a self-draw)
+}
+
 void round_columns(Sim* s, const int32_t* peer, int64_t k0, int64_t k1) {
   const int M = s->M;
   const int64_t n = s->ncols;
@@ -267,21 +287,7 @@ void round_columns(Sim* s, const int32_t* peer, int64_t k0, int64_t k1) {
       const float alpha = (float)s->alpha, sigma = (float)s->sigma, wf = (m != i) ? s->w[(size_t)i * M + m] : 0.0f;
       float* pre = s->pre.data() + (size_t)i * n;
       for (int64_t k = k0; k < k1; ++k) {
-        const int64_t e = s->cols[k];
-        const float xv = xi[k];
-        float h = xv;
-        if (s->objective == 1) {
-          uint32_t ctr[4], r[4];
-          double z[4];
-          make_ctr((uint32_t)(e >> 2), (uint32_t)i, s->round, TAG_NOISE, ctr);
-          philox4x32_10(ctr, s->key, r);
-          normals4(r, z);
-          const float t = xv - ci[k];
-          const float g = std::fmaf(sigma, (float)z[e & 3], t);
-          h = std::fmaf(-alpha, g, xv);                          // Eq. 15
-        }
-        const float diff = h - xm[k];
-        const float xnew = std::fmaf(-wf, diff, h);              // Eq. 16 (w = 0 on a self-draw)
+        const float xnew = update_fp32(s, i, s->round, s->cols[k], xi[k], ci[k], xm[k], alpha, sigma, wf);
         pre[k] = xnew;
         out[k] = bf16_round(xnew);
       }
@@ -369,6 +375,13 @@ void async_step(Sim* s) {
   const float* ci = s->c.data() + (size_t)i * n;
   for (int64_t k = 0; k < n; ++k) {
     const int64_t e = s->cols[k];
+    if (s->storage == 1) {  // bfloat16 state: the same fp32 evaluation as in a round, rounded once
+      const float wf = (m != i) ? s->w[(size_t)i * M + m] : 0.0f;
+      const float xnew = update_fp32(s, i, (uint64_t)nloc, e, xi[k], ci[k], xm[k], (float)s->alpha, (float)s->sigma, wf);
+      s->pre[(size_t)i * n + k] = xnew;
+      xi[k] = bf16_round(xnew);
+      continue;
+    }
     const double xv = (double)xi[k];
     double g = 0.0;
     if (s->objective == 1) {

@@ -42,8 +42,10 @@ class Config(C.Structure):
         ("lr", C.c_double), ("rho", C.c_double), ("pull_weight", C.c_double), ("sigma", C.c_double), ("x0_std", C.c_double),
         ("c_std", C.c_double), ("objective", C.c_int32), ("seed", C.c_uint64), ("device", C.c_int32),
         ("stream", C.c_void_p), ("trace_rounds", C.c_int64), ("policy_K", C.c_int32), ("policy_R", C.c_int32), ("policy_rho_upper", C.c_double),
-        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("storage", C.c_int32),
     ]
+
+STORAGE = {"f32": 0, "bf16": 1}
 
 
 _lib = None
@@ -166,7 +168,8 @@ class Netmax:
                  sigma: float = 0.0, x0_std: float = 0.0, c_std: float = 0.0, objective: int = 1, seed: int = 0,
                  device: int = 0, stream: Optional[int] = None, trace_rounds: int = 1024, policy_K: int = 20,
                  policy_R: int = 20, workspace: Optional[int] = None, workspace_bytes: int = 0,
-                 element_offset: int = 0, pull_weight: float = 0.0, policy_rho_upper: float = 0.0):
+                 element_offset: int = 0, pull_weight: float = 0.0, policy_rho_upper: float = 0.0,
+                 storage: str = "f32"):
         L = lib()
         cfg = Config()
         _check(L.netmax_config_init(C.byref(cfg)))
@@ -184,15 +187,18 @@ class Netmax:
         cfg.policy_K, cfg.policy_R = int(policy_K), int(policy_R)
         cfg.policy_rho_upper = float(policy_rho_upper)
         cfg.workspace, cfg.workspace_bytes = workspace, int(workspace_bytes)
+        cfg.storage = STORAGE[storage]
+        self.storage = storage
         self.M, self.d = int(M), int(d)
         self._h = C.c_void_p()
         _check(L.netmax_create_ex(C.byref(cfg), C.byref(self._h)))
 
     @staticmethod
-    def workspace_size(M: int, d: int, trace_rounds: int = 1024) -> int:
+    def workspace_size(M: int, d: int, trace_rounds: int = 1024, storage: str = "f32") -> int:
         cfg = Config()
         _check(lib().netmax_config_init(C.byref(cfg)))
         cfg.M, cfg.d, cfg.trace_rounds = int(M), int(d), int(trace_rounds)
+        cfg.storage = STORAGE[storage]
         out = C.c_size_t()
         _check(lib().netmax_workspace_size(C.byref(cfg), C.byref(out)))
         return out.value

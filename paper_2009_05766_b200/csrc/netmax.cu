@@ -46,7 +46,9 @@ struct DeviceGuard {
 };
 
 struct Layout {
-  int64_t ld = 0, ldq = 0, nq = 0;
+  int64_t ld = 0, ldq = 0, nq = 0;  // row stride in elements / in 16-byte column groups; column groups in use
+  int elem = 4, halves = 1;         // bytes per stored element; Philox blocks (4 elements) per column group
+  size_t plane = 0;                 // bytes of one [M][ld] array
   size_t off_x0 = 0, off_x1 = 0, off_c = 0, off_thr = 0, off_last = 0, off_w = 0, off_trace = 0, off_tel = 0,
          off_partials = 0, off_ticket = 0, off_colpart = 0, off_coltick = 0, total = 0;
 };
@@ -55,14 +57,18 @@ constexpr int kMaxGrid = 148 * 16;  // upper bound on resident CTAs of the round
 constexpr int64_t kMaxRoundsPerLaunch = 4096;  // rounds one cooperative launch runs at most
 constexpr size_t kColPartBytes = (size_t)8 << 20;  // column partials of the row-split (short vector) shape
 
-Layout make_layout(int64_t M, int64_t d, int64_t trace_rounds) {
+Layout make_layout(int64_t M, int64_t d, int64_t trace_rounds, int storage) {
   Layout L;
-  L.ld = (int64_t)align_up((size_t)d, 32);  // rows start on 128-byte boundaries
-  L.ldq = L.ld / 4;
-  L.nq = (d + 3) / 4;
+  L.elem = storage == NETMAX_STORAGE_BF16 ? 2 : 4;
+  L.halves = storage == NETMAX_STORAGE_BF16 ? 2 : 1;
+  const int64_t per_group = 16 / L.elem;
+  L.ld = (int64_t)align_up((size_t)d, (size_t)(128 / L.elem));  // rows start on 128-byte boundaries
+  L.ldq = L.ld / per_group;
+  L.nq = (d + per_group - 1) / per_group;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
-  const size_t plane = (size_t)M * L.ld * sizeof(float);
+  const size_t plane = (size_t)M * L.ld * L.elem;
+  L.plane = plane;
   L.off_x0 = take(plane);
   L.off_x1 = take(plane);
   L.off_c = take(plane);
@@ -94,7 +100,8 @@ struct netmax_ctx {
   cudaStream_t stream = nullptr;
   bool own_memory = false;
   unsigned char* base = nullptr;
-  float *x[2] = {nullptr, nullptr}, *c = nullptr;
+  int storage = NETMAX_STORAGE_F32;
+  unsigned char *x[2] = {nullptr, nullptr}, *c = nullptr;  // [M][ld] fp32 or bfloat16, as `storage` says
   uint32_t* thr = nullptr;
   int32_t* last_nz = nullptr;
   float* wtab = nullptr;
@@ -313,22 +320,23 @@ int resolve_policy(netmax_ctx* ctx, const double* speed, const double* prob, dou
   return NETMAX_OK;
 }
 
-int launch_init(netmax_ctx* ctx, float* dst, double stddev, uint32_t tag) {
-  NM_CUDA(ctx, cudaMemsetAsync(dst, 0, (size_t)ctx->M * ctx->L.ld * sizeof(float), ctx->stream));
+int launch_init(netmax_ctx* ctx, unsigned char* dst, double stddev, uint32_t tag) {
+  NM_CUDA(ctx, cudaMemsetAsync(dst, 0, ctx->L.plane, ctx->stream));
   if (stddev == 0.0) return NETMAX_OK;
   InitParams p;
   p.dst = reinterpret_cast<float4*>(dst);
   p.ldq = ctx->L.ldq;
   p.nq = ctx->L.nq;
   p.M = ctx->M;
-  p.tail = (int32_t)(ctx->d % 4);
+  p.tail = (int32_t)(ctx->d % (4 * ctx->L.halves));
   p.stddev = (float)stddev;
   p.tag = tag;
   p.q_offset = ctx->q_offset;
   p.keys = ctx->keys;
   const int64_t total = (int64_t)ctx->M * ctx->L.nq;
   const int grid = (int)std::min<int64_t>((total + kThreads - 1) / kThreads, (int64_t)ctx->sm_count * 16);
-  init_normal_kernel<<<grid, kThreads, 0, ctx->stream>>>(p);
+  if (ctx->L.halves == 2) init_normal_kernel<2><<<grid, kThreads, 0, ctx->stream>>>(p);
+  else init_normal_kernel<1><<<grid, kThreads, 0, ctx->stream>>>(p);
   ctx->launches += 1;
   NM_CUDA(ctx, cudaGetLastError());
   return NETMAX_OK;
@@ -366,18 +374,30 @@ using RoundKernel = void (*)(const RoundParams);
 
 using StepKernel = void (*)(const StepParams);
 
-StepKernel pick_step_kernel(int objective) { return objective == 1 ? step_kernel<1, true> : step_kernel<0, true>; }
+// halves: 1 for fp32 state, 2 for bfloat16 state (Philox blocks per 16-byte column group)
+template <int kHalves>
+StepKernel pick_step_kernel_h(int objective) {
+  return objective == 1 ? step_kernel<1, true, kHalves> : step_kernel<0, true, kHalves>;
+}
+StepKernel pick_step_kernel(int objective, int halves) {
+  return halves == 2 ? pick_step_kernel_h<2>(objective) : pick_step_kernel_h<1>(objective);
+}
 
-RoundKernel pick_kernel(int objective, bool short_vectors) {
-  if (objective == 2) return short_vectors ? round_kernel<2, true, 4> : round_kernel<2, true, 1>;
-  if (short_vectors) return objective == 1 ? round_kernel<1, true, 4> : round_kernel<0, true, 4>;
-  return objective == 1 ? round_kernel<1, true, 1> : round_kernel<0, true, 1>;
+template <int kHalves>
+RoundKernel pick_kernel_h(int objective, bool short_vectors) {
+  if (objective == 2) return short_vectors ? round_kernel<2, true, 4, kHalves> : round_kernel<2, true, 1, kHalves>;
+  if (short_vectors) return objective == 1 ? round_kernel<1, true, 4, kHalves> : round_kernel<0, true, 4, kHalves>;
+  return objective == 1 ? round_kernel<1, true, 1, kHalves> : round_kernel<0, true, 1, kHalves>;
+}
+RoundKernel pick_kernel(int objective, bool short_vectors, int halves) {
+  return halves == 2 ? pick_kernel_h<2>(objective, short_vectors) : pick_kernel_h<1>(objective, short_vectors);
 }
 
 using MultiRoundKernel = void (*)(const MultiRoundParams);
 
-MultiRoundKernel pick_multi_kernel(int objective) {
-  return objective == 1 ? multi_round_kernel<1, true> : multi_round_kernel<0, true>;
+MultiRoundKernel pick_multi_kernel(int objective, int halves) {
+  if (halves == 2) return objective == 1 ? multi_round_kernel<1, true, 2> : multi_round_kernel<0, true, 2>;
+  return objective == 1 ? multi_round_kernel<1, true, 1> : multi_round_kernel<0, true, 1>;
 }
 
 int floor_pow2(int64_t v) {
@@ -408,7 +428,7 @@ int plan_round(netmax_ctx* ctx, RoundPlan& plan, int objective) {
       if (rl > M && cand != kThreads) continue;  // row lanes without rows
       const int64_t nct = (nq + cand - 1) / cand;
       int g = (int)std::min<int64_t>(std::min<int64_t>(32, std::max<int64_t>(1, M / rl)), floor_pow2(std::max<int64_t>(1, target / nct)));
-      while (g > 1 && (size_t)nct * g * cand * 32 > kColPartBytes) g >>= 1;
+      while (g > 1 && (size_t)nct * g * cand * 32 * ctx->L.halves > kColPartBytes) g >>= 1;
       if (nct * g > kMaxGrid) continue;
       const int64_t score = std::min<int64_t>(nct * g, target);
       if (score > best_score) {
@@ -423,15 +443,15 @@ int plan_round(netmax_ctx* ctx, RoundPlan& plan, int objective) {
   plan.rg = rg;
   plan.rows_per_group = (int)((M + rg - 1) / rg);
   plan.n_tiles = (nq + cg - 1) / cg * rg;
-  plan.smem = align_up((size_t)M * 8, 16) + (plan.rl > 1 ? (size_t)kThreads * 32 : 0) + 64 * sizeof(double);
-  RoundKernel k = pick_kernel(objective, plan.short_vectors);
+  plan.smem = align_up((size_t)M * 8, 16) + (plan.rl > 1 ? (size_t)kThreads * 32 * ctx->L.halves : 0) + 64 * sizeof(double);
+  RoundKernel k = pick_kernel(objective, plan.short_vectors, ctx->L.halves);
   if (plan.smem > 48 * 1024)
     NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
   int per_sm = 0;
   NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, plan.smem));
   if (per_sm < 1) return fail(ctx, NETMAX_CUDA_ERROR, "round kernel does not fit on an SM (smem %zu)", plan.smem);
   if (plan.short_vectors && ctx->cooperative) {  // the multi-round kernel needs all of its CTAs resident
-    MultiRoundKernel mk = pick_multi_kernel(objective == 2 ? 0 : objective);
+    MultiRoundKernel mk = pick_multi_kernel(objective == 2 ? 0 : objective, ctx->L.halves);
     if (plan.smem > 48 * 1024)
       NM_CUDA(ctx, cudaFuncSetAttribute(mk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
     int per_sm_multi = 0;
@@ -459,6 +479,10 @@ int netmax_config_init(netmax_config* cfg) {
 
 static int check_sizes(const netmax_config* cfg) {
   if (!cfg) return fail(nullptr, NETMAX_INVALID_ARG, "cfg is NULL");
+  if (cfg->storage != NETMAX_STORAGE_F32 && cfg->storage != NETMAX_STORAGE_BF16)
+    return fail(nullptr, NETMAX_INVALID_ARG, "storage = %d is neither NETMAX_STORAGE_F32 nor NETMAX_STORAGE_BF16", cfg->storage);
+  if (cfg->storage == NETMAX_STORAGE_BF16 && cfg->element_offset % 8 != 0)
+    return fail(nullptr, NETMAX_INVALID_ARG, "element_offset = %lld must be a multiple of 8 with bfloat16 storage", (long long)cfg->element_offset);
   if (cfg->M < 2 || cfg->M > kMaxM) return fail(nullptr, NETMAX_INVALID_ARG, "M = %d outside [2, %lld]", cfg->M, (long long)kMaxM);
   if (cfg->d < 1 || cfg->d >= kMaxD) return fail(nullptr, NETMAX_INVALID_ARG, "d = %lld outside [1, 2^30 - 32)", (long long)cfg->d);
   if (cfg->element_offset < 0 || cfg->element_offset % 4 != 0 || cfg->element_offset + cfg->d >= kMaxD)
@@ -471,7 +495,7 @@ int netmax_workspace_size(const netmax_config* cfg, size_t* bytes) {
   int rc = check_sizes(cfg);
   if (rc) return rc;
   if (!bytes) return fail(nullptr, NETMAX_INVALID_ARG, "bytes is NULL");
-  *bytes = make_layout(cfg->M, cfg->d, cfg->trace_rounds).total;
+  *bytes = make_layout(cfg->M, cfg->d, cfg->trace_rounds, cfg->storage).total;
   return NETMAX_OK;
 }
 
@@ -512,7 +536,8 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   ctx->policy_R = cfg->policy_R > 0 ? cfg->policy_R : 20;
   ctx->policy_rho_upper = cfg->policy_rho_upper > 0.0 ? cfg->policy_rho_upper : 0.0;
   ctx->keys = make_philox_keys(cfg->seed);
-  ctx->L = make_layout(cfg->M, cfg->d, cfg->trace_rounds);
+  ctx->storage = cfg->storage;
+  ctx->L = make_layout(cfg->M, cfg->d, cfg->trace_rounds, cfg->storage);
 
   rc = build_adjacency(ctx, cfg->M, cfg->link_speed_gbps, ctx->adj);
   if (rc) return bail(rc);
@@ -556,9 +581,9 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
     ctx->own_memory = true;
   }
   const Layout& L = ctx->L;
-  ctx->x[0] = (float*)(ctx->base + L.off_x0);
-  ctx->x[1] = (float*)(ctx->base + L.off_x1);
-  ctx->c = (float*)(ctx->base + L.off_c);
+  ctx->x[0] = ctx->base + L.off_x0;
+  ctx->x[1] = ctx->base + L.off_x1;
+  ctx->c = ctx->base + L.off_c;
   ctx->thr = (uint32_t*)(ctx->base + L.off_thr);
   ctx->last_nz = (int32_t*)(ctx->base + L.off_last);
   ctx->wtab = (float*)(ctx->base + L.off_w);
@@ -579,7 +604,7 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   };
   if (!step(cudaMemsetAsync(ctx->ticket, 0, 256, ctx->stream), "cudaMemsetAsync(ticket)")) return bail(NETMAX_CUDA_ERROR);
   if (!step(cudaMemsetAsync(ctx->coltick, 0, (size_t)kMaxGrid * sizeof(unsigned int), ctx->stream), "cudaMemsetAsync(coltick)")) return bail(NETMAX_CUDA_ERROR);
-  if (!step(cudaMemsetAsync(ctx->x[1], 0, (size_t)ctx->M * L.ld * sizeof(float), ctx->stream), "cudaMemsetAsync(x)")) return bail(NETMAX_CUDA_ERROR);
+  if (!step(cudaMemsetAsync(ctx->x[1], 0, L.plane, ctx->stream), "cudaMemsetAsync(x)")) return bail(NETMAX_CUDA_ERROR);
   if (!step(cudaMemsetAsync(ctx->tel, 0, (size_t)ctx->trace_rounds * 2 * sizeof(double), ctx->stream), "cudaMemsetAsync(tel)")) return bail(NETMAX_CUDA_ERROR);
   rc = upload_policy(ctx);
   if (rc) return bail(rc);
@@ -658,19 +683,59 @@ static int check_device_error(netmax_ctx* ctx) {
   return fail(ctx, NETMAX_CUDA_ERROR, "a multi-round launch gave up waiting at its grid barrier; replicas are not valid");
 }
 
-static int copy_in(netmax_ctx* ctx, float* dst, const float* host) {
+// Host transfers of a bfloat16 context go through fp32 on the device: the buffer of the double
+// buffer that holds no replicas at the moment serves as the staging area, a chunk of rows at a
+// time, and is cleared again afterwards.  Nothing is allocated.
+static int64_t staging_rows(const netmax_ctx* ctx) {
+  return std::max<int64_t>(1, (int64_t)(ctx->L.plane / ((size_t)ctx->d * sizeof(float))));
+}
+
+static int convert_grid(const netmax_ctx* ctx, int64_t total) {
+  return (int)std::min<int64_t>((total + kThreads - 1) / kThreads, (int64_t)ctx->sm_count * 16);
+}
+
+static int copy_in(netmax_ctx* ctx, unsigned char* dst, const float* host) {
   if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
   if (!host) return fail(ctx, NETMAX_INVALID_ARG, "host pointer is NULL");
   DeviceGuard guard(ctx->device);
+  if (ctx->storage == NETMAX_STORAGE_BF16) {
+    float* stage = reinterpret_cast<float*>(ctx->x[ctx->cur ^ 1]);
+    const int64_t chunk = staging_rows(ctx);
+    for (int64_t r0 = 0; r0 < ctx->M; r0 += chunk) {
+      const int64_t rows = std::min<int64_t>(chunk, ctx->M - r0);
+      NM_CUDA(ctx, cudaMemcpyAsync(stage, host + (size_t)r0 * ctx->d, (size_t)rows * ctx->d * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
+      narrow_rows_kernel<<<convert_grid(ctx, rows * ctx->d), kThreads, 0, ctx->stream>>>(
+          stage, reinterpret_cast<unsigned short*>(dst) + (size_t)r0 * ctx->L.ld, rows, ctx->d, ctx->L.ld);
+      ctx->launches += 1;
+      NM_CUDA(ctx, cudaGetLastError());
+    }
+    NM_CUDA(ctx, cudaMemsetAsync(stage, 0, ctx->L.plane, ctx->stream));
+    return NETMAX_OK;
+  }
   NM_CUDA(ctx, cudaMemcpy2DAsync(dst, (size_t)ctx->L.ld * sizeof(float), host, (size_t)ctx->d * sizeof(float),
                                  (size_t)ctx->d * sizeof(float), (size_t)ctx->M, cudaMemcpyHostToDevice, ctx->stream));
   return NETMAX_OK;
 }
 
-static int copy_out(netmax_ctx* ctx, const float* src, float* host) {
+static int copy_out(netmax_ctx* ctx, const unsigned char* src, float* host) {
   if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
   if (!host) return fail(ctx, NETMAX_INVALID_ARG, "host pointer is NULL");
   DeviceGuard guard(ctx->device);
+  if (ctx->storage == NETMAX_STORAGE_BF16) {
+    float* stage = reinterpret_cast<float*>(ctx->x[ctx->cur ^ 1]);
+    const int64_t chunk = staging_rows(ctx);
+    for (int64_t r0 = 0; r0 < ctx->M; r0 += chunk) {
+      const int64_t rows = std::min<int64_t>(chunk, ctx->M - r0);
+      widen_rows_kernel<<<convert_grid(ctx, rows * ctx->d), kThreads, 0, ctx->stream>>>(
+          reinterpret_cast<const unsigned short*>(src) + (size_t)r0 * ctx->L.ld, stage, rows, ctx->d, ctx->L.ld);
+      ctx->launches += 1;
+      NM_CUDA(ctx, cudaGetLastError());
+      NM_CUDA(ctx, cudaMemcpyAsync(host + (size_t)r0 * ctx->d, stage, (size_t)rows * ctx->d * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+    }
+    NM_CUDA(ctx, cudaMemsetAsync(stage, 0, ctx->L.plane, ctx->stream));
+    NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return check_device_error(ctx);
+  }
   NM_CUDA(ctx, cudaMemcpy2DAsync(host, (size_t)ctx->d * sizeof(float), src, (size_t)ctx->L.ld * sizeof(float),
                                  (size_t)ctx->d * sizeof(float), (size_t)ctx->M, cudaMemcpyDeviceToHost, ctx->stream));
   NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
@@ -692,7 +757,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   RoundPlan plan;
   int rc = plan_round(ctx, plan, ctx->objective);
   if (rc) return rc;
-  RoundKernel kernel = pick_kernel(ctx->objective, plan.short_vectors);
+  RoundKernel kernel = pick_kernel(ctx->objective, plan.short_vectors, ctx->L.halves);
 
   RoundParams p;
   p.c = reinterpret_cast<const float4*>(ctx->c);
@@ -700,11 +765,11 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   p.partials = ctx->partials;
   p.ticket = ctx->ticket;
   p.ldq = ctx->L.ldq;
-  p.row_bytes = (uint32_t)(ctx->L.ld * sizeof(float));
+  p.row_bytes = (uint32_t)(ctx->L.ld * ctx->L.elem);
   p.nq = ctx->L.nq;
   p.n_tiles = plan.n_tiles;
   p.M = ctx->M;
-  p.tail = (int32_t)(ctx->d % 4);
+  p.tail = (int32_t)(ctx->d % (4 * ctx->L.halves));
   p.cg = plan.cg;
   p.rl = plan.rl;
   p.rg = plan.rg;
@@ -748,7 +813,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
         ctx->inject_absent_ctas = 0;
         NM_CUDA(ctx, cudaMemsetAsync(ctx->grid_barrier, 0, sizeof(unsigned int), ctx->stream));
         void* args[] = {&mp};
-        NM_CUDA(ctx, cudaLaunchCooperativeKernel((const void*)pick_multi_kernel(ctx->objective), dim3(plan.grid), dim3(kThreads),
+        NM_CUDA(ctx, cudaLaunchCooperativeKernel((const void*)pick_multi_kernel(ctx->objective, ctx->L.halves), dim3(plan.grid), dim3(kThreads),
                                                  args, plan.smem, ctx->stream));
         ctx->launches += 1;
         ctx->cur ^= (int)(chunk & 1);
@@ -797,7 +862,7 @@ int netmax_read_columns(netmax_ctx* ctx, const int64_t* host_cols, int64_t n_col
   const int grid = (int)std::min<int64_t>((total + kThreads - 1) / kThreads, 4096);
   e = cudaMemcpyAsync(d_cols, host_cols, (size_t)n_cols * sizeof(int64_t), cudaMemcpyHostToDevice, ctx->stream);
   if (e == cudaSuccess) {
-    gather_columns_kernel<<<grid, kThreads, 0, ctx->stream>>>(ctx->x[ctx->cur], ctx->L.ld, ctx->M, d_cols, n_cols, d_out);
+    gather_columns_kernel<<<grid, kThreads, 0, ctx->stream>>>(ctx->x[ctx->cur], ctx->storage == NETMAX_STORAGE_BF16, ctx->L.ld, ctx->M, d_cols, n_cols, d_out);
     ctx->launches += 1;
     e = cudaGetLastError();
   }
@@ -858,7 +923,7 @@ int netmax_read_columns_static(netmax_ctx* ctx, const int64_t* host_cols, int64_
   const int64_t total = n_cols * ctx->M;
   const int grid = (int)std::min<int64_t>((total + kThreads - 1) / kThreads, 4096);
   NM_CUDA(ctx, cudaMemcpyAsync(scratch->cols, host_cols, (size_t)n_cols * sizeof(int64_t), cudaMemcpyHostToDevice, ctx->stream));
-  gather_columns_kernel<<<grid, kThreads, 0, ctx->stream>>>(ctx->x[ctx->cur], ctx->L.ld, ctx->M, scratch->cols, n_cols, scratch->values);
+  gather_columns_kernel<<<grid, kThreads, 0, ctx->stream>>>(ctx->x[ctx->cur], ctx->storage == NETMAX_STORAGE_BF16, ctx->L.ld, ctx->M, scratch->cols, n_cols, scratch->values);
   ctx->launches += 1;
   NM_CUDA(ctx, cudaGetLastError());
   NM_CUDA(ctx, cudaMemcpyAsync(host_out, scratch->values, (size_t)total * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
@@ -916,7 +981,7 @@ int netmax_telemetry(netmax_ctx* ctx, int64_t first_round, int64_t n, double* ho
 int netmax_replicas_device(netmax_ctx* ctx, const float** x, int64_t* ld) {
   if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
   if (!x || !ld) return fail(ctx, NETMAX_INVALID_ARG, "output pointer is NULL");
-  *x = ctx->x[ctx->cur];
+  *x = reinterpret_cast<const float*>(ctx->x[ctx->cur]);
   *ld = ctx->L.ld;
   return NETMAX_OK;
 }
@@ -935,7 +1000,7 @@ int netmax_measure(netmax_ctx* ctx, double* consensus, double* loss) {
   RoundPlan plan;
   int rc = plan_round(ctx, plan, 2);  // 2: the measuring instantiation of the round kernel
   if (rc) return rc;
-  RoundKernel kernel = pick_kernel(2, plan.short_vectors);
+  RoundKernel kernel = pick_kernel(2, plan.short_vectors, ctx->L.halves);
   RoundParams p;
   std::memset(&p, 0, sizeof p);
   p.x_cur = reinterpret_cast<const float4*>(ctx->x[ctx->cur]);
@@ -947,11 +1012,11 @@ int netmax_measure(netmax_ctx* ctx, double* consensus, double* loss) {
   p.ticket = ctx->ticket;
   p.tel_out = ctx->measure_out;
   p.ldq = ctx->L.ldq;
-  p.row_bytes = (uint32_t)(ctx->L.ld * sizeof(float));
+  p.row_bytes = (uint32_t)(ctx->L.ld * ctx->L.elem);
   p.nq = ctx->L.nq;
   p.n_tiles = plan.n_tiles;
   p.M = ctx->M;
-  p.tail = (int32_t)(ctx->d % 4);
+  p.tail = (int32_t)(ctx->d % (4 * ctx->L.halves));
   p.cg = plan.cg;
   p.rl = plan.rl;
   p.rg = plan.rg;
@@ -1089,13 +1154,13 @@ int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps) {
   if (n_steps < 0) return fail(ctx, NETMAX_INVALID_ARG, "n_steps = %lld < 0", (long long)n_steps);
   DeviceGuard guard(ctx->device);
   const int32_t M = ctx->M;
-  StepKernel kernel = pick_step_kernel(ctx->objective);
+  StepKernel kernel = pick_step_kernel(ctx->objective, ctx->L.halves);
   StepParams p;
   p.x = reinterpret_cast<float4*>(ctx->x[ctx->cur]);
   p.c = reinterpret_cast<const float4*>(ctx->c);
   p.nq = ctx->L.nq;
-  p.row_bytes = (uint32_t)(ctx->L.ld * sizeof(float));
-  p.tail = (int32_t)(ctx->d % 4);
+  p.row_bytes = (uint32_t)(ctx->L.ld * ctx->L.elem);
+  p.tail = (int32_t)(ctx->d % (4 * ctx->L.halves));
   p.alpha = (float)ctx->alpha;
   p.sigma = (float)ctx->sigma;
   p.q_offset = ctx->q_offset;

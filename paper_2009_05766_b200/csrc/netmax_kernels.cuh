@@ -7,6 +7,12 @@
 //                         with the round's telemetry; reads one buffer, writes the other.
 //   init_normal_kernel    x(0) and c from the seed.
 //   gather_columns_kernel sampled read-back.
+//
+// State precision.  The replicas and centres are stored as fp32 (kHalves == 1) or, as an option
+// the paper does not have, as bfloat16 (kHalves == 2).  Either way a thread moves 16-byte column
+// groups -- 4 fp32 or 8 bfloat16 values, i.e. kHalves Philox blocks of four normals -- and all
+// arithmetic is fp32: bfloat16 values are widened exactly on load, and each new parameter is
+// rounded once, to the nearest bfloat16 (ties to even), at the store.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -49,7 +55,7 @@ __global__ void __launch_bounds__(256) sample_peers_kernel(const SampleParams p)
 
 // ------------------------------------------------------------------------- round
 struct RoundParams {
-  const float4* x_cur;   // [M][ldq] round-start replicas
+  const float4* x_cur;   // [M][ldq] round-start replicas (16-byte column groups: 4 fp32 or 8 bfloat16)
   float4* x_nxt;         // [M][ldq] next replicas
   const float4* c;       // [M][ldq] centres
   const int32_t* peers;  // [M] this round's draws
@@ -57,42 +63,73 @@ struct RoundParams {
   double* partials;      // [gridDim.x][2] per-CTA telemetry sums
   unsigned int* ticket;  // last-CTA-done counter (0 between launches)
   double* tel_out;       // [2] this round's (consensus, loss)
-  int64_t ldq;           // row stride, in float4
+  int64_t ldq;           // row stride, in column groups
   uint32_t row_bytes;    // row stride, in bytes (< 2^32)
-  int64_t nq;            // column groups per row = ceil(d / 4)
+  int64_t nq;            // column groups per row = ceil(d / (4 kHalves))
   int64_t n_tiles;       // ceil(nq / cg)
   int32_t M;
-  int32_t tail;          // d % 4: live lanes of the last column group (0 = all four)
+  int32_t tail;          // d % (4 kHalves): live lanes of the last column group (0 = all of them)
   int32_t cg;            // column groups per tile   (cg * rl == blockDim.x, both powers of two)
   int32_t rl;            // row lanes per tile
   int32_t rg;            // row groups: tile t covers column tile t / rg, rows of group t % rg
   int32_t rows_per_group;  // ceil(M / rg)
-  float4* colpart;       // rg > 1: per tile, per column group: (sum, sum of squares) partials
+  float4* colpart;       // rg > 1: per tile, per column group, per half: (sum, sum of squares) partials
   unsigned int* coltick; // rg > 1: arrivals per column tile (0 between launches)
   float alpha, sigma;
   float inv_M;
   uint32_t round_lo, ctr3;
-  uint32_t q_offset;     // column-group index of the context's first element in the global vector
+  uint32_t q_offset;     // Philox block index (element / 4) of the context's first element in the global vector
   PhiloxKeys keys;
 };
 
-// Per-thread telemetry accumulators of one column group (4 columns as two fp32 pairs):
-// sum (x - pivot), sum (x - pivot)^2 and sum (x - c)^2 over the rows the thread has seen.
-struct RowAcc {
-  pair_t s1a = 0ull, s1b = 0ull, s2a = 0ull, s2b = 0ull, la = 0ull, lb = 0ull;  // +0.0f pairs
+// Per-thread telemetry accumulators.  ColAcc: four columns as two fp32 pairs, sum (x - pivot)
+// and sum (x - pivot)^2 over the rows the thread has seen.  LossAcc: sum (x - c)^2 over all of
+// the thread's elements.
+struct ColAcc {
+  pair_t s1a = 0ull, s1b = 0ull, s2a = 0ull, s2b = 0ull;  // +0.0f pairs
 };
+struct LossAcc {
+  pair_t la = 0ull, lb = 0ull;
+};
+
+// Four bfloat16 values in a 64-bit word (element 0 in the lowest 16 bits) <-> two fp32 pairs.
+// Widening is exact; narrowing rounds to nearest, ties to even.
+__device__ __forceinline__ ulonglong2 widen_bf16x4(unsigned long long v) {
+  const uint32_t lo = (uint32_t)v, hi = (uint32_t)(v >> 32);
+  return make_ulonglong2(pack2(__uint_as_float(lo << 16), __uint_as_float(lo & 0xFFFF0000u)),
+                         pack2(__uint_as_float(hi << 16), __uint_as_float(hi & 0xFFFF0000u)));
+}
+__device__ __forceinline__ unsigned long long narrow_bf16x4(ulonglong2 v) {
+  float e0, e1, e2, e3;
+  unpack2(v.x, e0, e1);
+  unpack2(v.y, e2, e3);
+  uint32_t lo, hi;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo) : "f"(e1), "f"(e0));  // first operand -> upper half
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hi) : "f"(e3), "f"(e2));
+  return ((unsigned long long)hi << 32) | lo;
+}
+// Half h (four elements, as two fp32 pairs) of a 16-byte column group.
+template <int kHalves>
+__device__ __forceinline__ ulonglong2 group_half(ulonglong2 raw, int h) {
+  if (kHalves == 1) return raw;
+  return widen_bf16x4(h == 0 ? raw.x : raw.y);
+}
+// Live lanes of half h of a column group: 4 everywhere but in a row's last, ragged group.
+__device__ __forceinline__ int live_lanes(bool ragged, int tail, int h) {
+  return ragged ? min(4, max(0, tail - 4 * h)) : 4;
+}
 
 // Eq. 15 and Eq. 16 on one column group of one worker, on packed fp32 pairs:
 //   g = (x - c) + sigma z,  h = x - alpha g                                       (Eq. 15)
 //   x' = h - w (h - x_m),   w = alpha rho gamma_im  (w = 0 on a self-draw)          (Eq. 16)
-// q32 is the global column-group index (first Philox counter word), iter_lo / ctr3 carry the
-// round (or, on the asynchronous timeline, the worker's local iteration); `ragged` marks the
-// last group of a row whose padding lanes (beyond `tail` live ones) must stay zero.  ta, tb
-// return x - c for the caller's loss statistic.
+// q32 is the global index of the four elements' Philox block (first counter word), iter_lo /
+// ctr3 carry the round (or, on the asynchronous timeline, the worker's local iteration); `live`
+// is the number of real elements among the four (4 except in the last group of a row, whose
+// padding lanes must stay zero).  ta, tb return x - c for the caller's loss statistic.
 template <int kObjective, bool kFastNoise>
-__device__ __forceinline__ ulonglong2 update_core(float alpha, float sigma, int32_t tail, const PhiloxKeys& keys,
+__device__ __forceinline__ ulonglong2 update_core(float alpha, float sigma, const PhiloxKeys& keys,
                                                   uint32_t iter_lo, uint32_t ctr3, uint32_t q32, uint32_t worker,
-                                                  ulonglong2 xv, ulonglong2 cv, ulonglong2 xm, float w, bool ragged,
+                                                  ulonglong2 xv, ulonglong2 cv, ulonglong2 xm, float w, int live,
                                                   pair_t& ta, pair_t& tb) {
   const pair_t neg1 = pack2(-1.0f, -1.0f);
   const pair_t nw2 = pack2(-w, -w);
@@ -117,12 +154,13 @@ __device__ __forceinline__ ulonglong2 update_core(float alpha, float sigma, int3
   }
   pair_t oa = fma2(nw2, fma2(xm.x, neg1, ha), ha);
   pair_t ob = fma2(nw2, fma2(xm.y, neg1, hb), hb);
-  if (ragged) {  // keep the padding lanes of the last group at zero
+  if (live < 4) {  // keep the padding lanes of the last group at zero
     float o0, o1, o2, o3;
     unpack2(oa, o0, o1);
     unpack2(ob, o2, o3);
-    if (tail < 2) o1 = 0.f;
-    if (tail < 3) o2 = 0.f;
+    if (live < 1) o0 = 0.f;
+    if (live < 2) o1 = 0.f;
+    if (live < 3) o2 = 0.f;
     oa = pack2(o0, o1);
     ob = pack2(o2, 0.f);
   }
@@ -133,7 +171,7 @@ __device__ __forceinline__ ulonglong2 update_core(float alpha, float sigma, int3
 template <int kObjective, bool kFastNoise>
 __device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t round_lo, uint32_t ctr3, uint32_t q32,
                                                  uint32_t worker, ulonglong2 xv, ulonglong2 cv, ulonglong2 xm,
-                                                 ulonglong2 pivot, float w, bool ragged, RowAcc& acc) {
+                                                 ulonglong2 pivot, float w, int live, ColAcc& acc, LossAcc& lacc) {
   const pair_t neg1 = pack2(-1.0f, -1.0f);
   pair_t ta, tb;
   ulonglong2 o = xv;
@@ -141,16 +179,16 @@ __device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t 
     ta = fma2(cv.x, neg1, xv.x);
     tb = fma2(cv.y, neg1, xv.y);
   } else {
-    o = update_core<kObjective, kFastNoise>(p.alpha, p.sigma, p.tail, p.keys, round_lo, ctr3, q32, worker, xv, cv, xm, w,
-                                            ragged, ta, tb);
+    o = update_core<kObjective, kFastNoise>(p.alpha, p.sigma, p.keys, round_lo, ctr3, q32, worker, xv, cv, xm, w, live,
+                                            ta, tb);
   }
   const pair_t da = fma2(pivot.x, neg1, xv.x), db = fma2(pivot.y, neg1, xv.y);  // x - pivot
   acc.s1a = add2(acc.s1a, da);
   acc.s1b = add2(acc.s1b, db);
   acc.s2a = fma2(da, da, acc.s2a);
   acc.s2b = fma2(db, db, acc.s2b);
-  acc.la = fma2(ta, ta, acc.la);
-  acc.lb = fma2(tb, tb, acc.lb);
+  lacc.la = fma2(ta, ta, lacc.la);
+  lacc.lb = fma2(tb, tb, lacc.lb);
   return o;
 }
 
@@ -236,10 +274,13 @@ __device__ __forceinline__ void finalize_telemetry(const RoundParams& p, double 
 // the resident CTAs.  All accesses are plain cacheable 128-bit loads and
 // stores: the peer read (a row this tile reads anyway) then hits L1/L2, and streaming hints on
 // c and on the output measured slower.
-// Dynamic shared memory: (peer, weight) int2[M], then (rl > 1) 2 * blockDim float4 of
+// Dynamic shared memory: (peer, weight) int2[M], then (rl > 1) 2 * kHalves * blockDim float4 of
 // column-sum scratch, then 64 doubles for the block reduction.
 #ifndef NETMAX_ROUND_MIN_CTAS
 #define NETMAX_ROUND_MIN_CTAS 4  // CTAs per SM the register allocation leaves room for
+#endif
+#ifndef NETMAX_ROUND_MIN_CTAS_BF16
+#define NETMAX_ROUND_MIN_CTAS_BF16 3  // bfloat16 state: eight elements per thread need more registers
 #endif
 
 // kRowsInFlight = 1 (64 registers, 4 CTAs/SM) is the streaming shape for long vectors, where
@@ -262,10 +303,11 @@ __device__ __forceinline__ ulonglong2 ld_x(const char* ptr) {
 }
 
 // All tiles of this CTA for one round.  Every thread of the CTA must call this.
-template <int kObjective, bool kFastNoise, int kRowsInFlight, bool kCoherent>
+template <int kObjective, bool kFastNoise, int kRowsInFlight, bool kCoherent, int kHalves>
 __device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* x_cur, float4* x_nxt, const int32_t* peers,
                                             uint32_t round_lo, uint32_t ctr3, int2* s_pw, float4* s_col,
                                             double& acc_cons, double& acc_loss) {
+  constexpr int kStats = 2 * kHalves;  // float4 column statistics per thread: (sum, sum of squares) per half
   const int tid = threadIdx.x;
   const int G = p.rg;
   __shared__ bool s_lastcol;
@@ -291,16 +333,19 @@ __device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* 
     const int64_t q = ct * p.cg + cgi;
     const bool live = q < p.nq;
     const bool ragged = (p.tail != 0) && (q == p.nq - 1);
-    float4 s1 = make_float4(0.f, 0.f, 0.f, 0.f), s2 = s1;
+    float4 st[kStats];  // st[2h] = sum (x - pivot), st[2h + 1] = sum (x - pivot)^2 of half h's columns
+#pragma unroll
+    for (int a = 0; a < kStats; ++a) st[a] = make_float4(0.f, 0.f, 0.f, 0.f);
     float loss = 0.f;
     if (live) {
       // byte pointers to this thread's column group in row 0; row i is i * row_bytes further
       const char* xq = reinterpret_cast<const char*>(x_cur + q);
       const char* cq = reinterpret_cast<const char*>(p.c + q);
       char* oq = reinterpret_cast<char*>(x_nxt + q);
-      const uint32_t q32 = (uint32_t)q + p.q_offset;
+      const uint32_t q32 = (uint32_t)q * kHalves + p.q_offset;
       const ulonglong2 pivot = ld_x<kCoherent>(xq);  // row 0: pivot of the one-pass variance
-      RowAcc acc;
+      ColAcc acc[kHalves];
+      LossAcc lacc;
       for (int i0 = r0 + rli; i0 < r1; i0 += step * kRowsInFlight) {
         ulonglong2 xv[kRowsInFlight], xm[kRowsInFlight], cv[kRowsInFlight];
         int2 pw[kRowsInFlight];
@@ -324,38 +369,51 @@ __device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* 
         for (int u = 0; u < kRowsInFlight; ++u) {
           const int i = i0 + u * step;
           if (kRowsInFlight == 1 || i < r1) {
-            const ulonglong2 o = row_update<kObjective, kFastNoise>(p, round_lo, ctr3, q32, (uint32_t)i, xv[u], cv[u],
-                                                                    xm[u], pivot, __int_as_float(pw[u].y), ragged, acc);
+            ulonglong2 o;
+#pragma unroll
+            for (int h = 0; h < kHalves; ++h) {
+              const ulonglong2 oh = row_update<kObjective, kFastNoise>(
+                  p, round_lo, ctr3, q32 + h, (uint32_t)i, group_half<kHalves>(xv[u], h), group_half<kHalves>(cv[u], h),
+                  group_half<kHalves>(xm[u], h), group_half<kHalves>(pivot, h), __int_as_float(pw[u].y),
+                  live_lanes(ragged, p.tail, h), acc[h], lacc);
+              if (kHalves == 1) o = oh;
+              else if (h == 0) o.x = narrow_bf16x4(oh);
+              else o.y = narrow_bf16x4(oh);
+            }
             if (kObjective != 2) *reinterpret_cast<ulonglong2*>(oq + (uint64_t)(uint32_t)i * p.row_bytes) = o;
           }
         }
       }
-      unpack2(acc.s1a, s1.x, s1.y);
-      unpack2(acc.s1b, s1.z, s1.w);
-      unpack2(acc.s2a, s2.x, s2.y);
-      unpack2(acc.s2b, s2.z, s2.w);
+#pragma unroll
+      for (int h = 0; h < kHalves; ++h) {
+        unpack2(acc[h].s1a, st[2 * h].x, st[2 * h].y);
+        unpack2(acc[h].s1b, st[2 * h].z, st[2 * h].w);
+        unpack2(acc[h].s2a, st[2 * h + 1].x, st[2 * h + 1].y);
+        unpack2(acc[h].s2b, st[2 * h + 1].z, st[2 * h + 1].w);
+      }
       float l0, l1, l2, l3;
-      unpack2(acc.la, l0, l1);
-      unpack2(acc.lb, l2, l3);
+      unpack2(lacc.la, l0, l1);
+      unpack2(lacc.lb, l2, l3);
       loss = (l0 + l1) + (l2 + l3);
     }
     if (p.rl > 1) {  // sum the column statistics over the row lanes (stride cg in tid)
-      s_col[tid] = s1;
-      s_col[blockDim.x + tid] = s2;
+#pragma unroll
+      for (int a = 0; a < kStats; ++a) s_col[a * blockDim.x + tid] = st[a];
       __syncthreads();
       for (int s = blockDim.x >> 1; s >= p.cg; s >>= 1) {
         if (tid < s) {
-          float4 a = s_col[tid], b = s_col[tid + s];
-          a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-          s_col[tid] = a;
-          a = s_col[blockDim.x + tid]; b = s_col[blockDim.x + tid + s];
-          a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-          s_col[blockDim.x + tid] = a;
+#pragma unroll
+          for (int a = 0; a < kStats; ++a) {
+            float4 v = s_col[a * blockDim.x + tid];
+            const float4 b = s_col[a * blockDim.x + tid + s];
+            v.x += b.x; v.y += b.y; v.z += b.z; v.w += b.w;
+            s_col[a * blockDim.x + tid] = v;
+          }
         }
         __syncthreads();
       }
-      s1 = s_col[cgi];
-      s2 = s_col[blockDim.x + cgi];
+#pragma unroll
+      for (int a = 0; a < kStats; ++a) st[a] = s_col[a * blockDim.x + cgi];
       __syncthreads();
     }
     bool owner = true;  // does this CTA hold the complete column sums of the tile?
@@ -363,8 +421,8 @@ __device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* 
       // rows are split over rg CTAs: publish this CTA's column partials; the last of the rg
       // CTAs of a column tile to arrive adds them up in group order (deterministic)
       if (rli == 0) {
-        p.colpart[((size_t)tile * p.cg + cgi) * 2] = s1;
-        p.colpart[((size_t)tile * p.cg + cgi) * 2 + 1] = s2;
+#pragma unroll
+        for (int a = 0; a < kStats; ++a) p.colpart[((size_t)tile * p.cg + cgi) * kStats + a] = st[a];
       }
       __threadfence();
       __syncthreads();
@@ -377,21 +435,26 @@ __device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* 
       owner = s_lastcol;
       if (owner && rli == 0) {
         __threadfence();
-        s1 = make_float4(0.f, 0.f, 0.f, 0.f);
-        s2 = s1;
+#pragma unroll
+        for (int a = 0; a < kStats; ++a) st[a] = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int gg = 0; gg < G; ++gg) {
-          const float4 a = __ldcg(p.colpart + (((size_t)ct * G + gg) * p.cg + cgi) * 2);
-          const float4 b = __ldcg(p.colpart + (((size_t)ct * G + gg) * p.cg + cgi) * 2 + 1);
-          s1.x += a.x; s1.y += a.y; s1.z += a.z; s1.w += a.w;
-          s2.x += b.x; s2.y += b.y; s2.z += b.z; s2.w += b.w;
+#pragma unroll
+          for (int a = 0; a < kStats; ++a) {
+            const float4 b = __ldcg(p.colpart + (((size_t)ct * G + gg) * p.cg + cgi) * kStats + a);
+            st[a].x += b.x; st[a].y += b.y; st[a].z += b.z; st[a].w += b.w;
+          }
         }
       }
     }
     if (rli == 0 && owner) {
       // sum_i (x_i - xbar)^2 = sum_i (x_i - a)^2 - (sum_i (x_i - a))^2 / M   per column
-      const float cons = (s2.x - s1.x * s1.x * p.inv_M) + (s2.y - s1.y * s1.y * p.inv_M) +
-                         (s2.z - s1.z * s1.z * p.inv_M) + (s2.w - s1.w * s1.w * p.inv_M);
-      acc_cons += (double)cons;
+#pragma unroll
+      for (int h = 0; h < kHalves; ++h) {
+        const float4 s1 = st[2 * h], s2 = st[2 * h + 1];
+        const float cons = (s2.x - s1.x * s1.x * p.inv_M) + (s2.y - s1.y * s1.y * p.inv_M) +
+                           (s2.z - s1.z * s1.z * p.inv_M) + (s2.w - s1.w * s1.w * p.inv_M);
+        acc_cons += (double)cons;
+      }
     }
     acc_loss += (double)loss;
   }
@@ -400,16 +463,17 @@ __device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* 
 // kRowsInFlight = 1 (64 registers, 4 CTAs/SM) is the streaming shape for long vectors, where
 // occupancy hides the HBM latency; kRowsInFlight = 4 (2 CTAs/SM) serves short, L2-resident
 // problems, where a thread's chain of dependent row loads is what takes the time.
-template <int kObjective, bool kFastNoise, int kRowsInFlight>
-__global__ void __launch_bounds__(256, kRowsInFlight == 1 ? NETMAX_ROUND_MIN_CTAS : 2) round_kernel(const RoundParams p) {
+template <int kObjective, bool kFastNoise, int kRowsInFlight, int kHalves>
+__global__ void __launch_bounds__(256, kRowsInFlight != 1 ? 2 : kHalves == 1 ? NETMAX_ROUND_MIN_CTAS : NETMAX_ROUND_MIN_CTAS_BF16)
+    round_kernel(const RoundParams p) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   int2* s_pw = reinterpret_cast<int2*>(smem_raw);  // (peer, bits of the pull weight) per worker
   const size_t head = (((size_t)p.M * 8) + 15) & ~(size_t)15;
   float4* s_col = reinterpret_cast<float4*>(smem_raw + head);
-  double* s_red = reinterpret_cast<double*>(smem_raw + head + (p.rl > 1 ? (size_t)blockDim.x * 32 : 0));
+  double* s_red = reinterpret_cast<double*>(smem_raw + head + (p.rl > 1 ? (size_t)blockDim.x * 32 * kHalves : 0));
   double acc_cons = 0.0, acc_loss = 0.0;
-  round_tiles<kObjective, kFastNoise, kRowsInFlight, false>(p, p.x_cur, p.x_nxt, p.peers, p.round_lo, p.ctr3, s_pw, s_col,
-                                                            acc_cons, acc_loss);
+  round_tiles<kObjective, kFastNoise, kRowsInFlight, false, kHalves>(p, p.x_cur, p.x_nxt, p.peers, p.round_lo, p.ctr3, s_pw,
+                                                                     s_col, acc_cons, acc_loss);
   finalize_telemetry(p, acc_cons, acc_loss, s_red);
 }
 
@@ -459,14 +523,14 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int
   return s_ok != 0;
 }
 
-template <int kObjective, bool kFastNoise>
+template <int kObjective, bool kFastNoise, int kHalves>
 __global__ void __launch_bounds__(256, 2) multi_round_kernel(const MultiRoundParams mp) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const RoundParams& p = mp.r;
   int2* s_pw = reinterpret_cast<int2*>(smem_raw);
   const size_t head = (((size_t)p.M * 8) + 15) & ~(size_t)15;
   float4* s_col = reinterpret_cast<float4*>(smem_raw + head);
-  double* s_red = reinterpret_cast<double*>(smem_raw + head + (p.rl > 1 ? (size_t)blockDim.x * 32 : 0));
+  double* s_red = reinterpret_cast<double*>(smem_raw + head + (p.rl > 1 ? (size_t)blockDim.x * 32 * kHalves : 0));
   const float4* x_cur = p.x_cur;
   float4* x_nxt = p.x_nxt;
   for (int k = 0; k < mp.n_rounds; ++k) {
@@ -474,8 +538,8 @@ __global__ void __launch_bounds__(256, 2) multi_round_kernel(const MultiRoundPar
     const int64_t slot = (mp.slot0 + k) % mp.ring;
     double* partials = mp.partials2 + (size_t)(k & 1) * 2 * gridDim.x;
     double acc_cons = 0.0, acc_loss = 0.0;
-    round_tiles<kObjective, kFastNoise, 4, true>(p, x_cur, x_nxt, mp.trace + slot * p.M, (uint32_t)round,
-                                                 philox_ctr3(kTagNoise, round), s_pw, s_col, acc_cons, acc_loss);
+    round_tiles<kObjective, kFastNoise, 4, true, kHalves>(p, x_cur, x_nxt, mp.trace + slot * p.M, (uint32_t)round,
+                                                          philox_ctr3(kTagNoise, round), s_pw, s_col, acc_cons, acc_loss);
     block_partials(partials, acc_cons, acc_loss, s_red);
     if (!grid_barrier(mp.barrier, (unsigned int)(k + 1), mp.error, mp.absent_ctas)) return;
     // round k is complete everywhere: one CTA publishes its telemetry while the rest move on
@@ -502,11 +566,11 @@ struct StepEvent {
 };
 
 struct StepParams {
-  float4* x;        // [M][ldq] replicas, updated in place
+  float4* x;        // [M][ldq] replicas (16-byte column groups), updated in place
   const float4* c;  // [M][ldq]
   int64_t nq;
   uint32_t row_bytes;
-  int32_t tail;
+  int32_t tail;     // d % (4 kHalves)
   float alpha, sigma;
   uint32_t q_offset;
   int32_t n_events;
@@ -514,7 +578,7 @@ struct StepParams {
   PhiloxKeys keys;
 };
 
-template <int kObjective, bool kFastNoise>
+template <int kObjective, bool kFastNoise, int kHalves>
 __global__ void __launch_bounds__(256) step_kernel(const StepParams p) {
   const StepEvent& e = p.ev[blockIdx.y];
   const uint64_t row_i = (uint64_t)(uint32_t)e.worker * p.row_bytes;
@@ -527,48 +591,97 @@ __global__ void __launch_bounds__(256) step_kernel(const StepParams p) {
     const ulonglong2 xm = *reinterpret_cast<const ulonglong2*>(xb + row_m + off);
     ulonglong2 cv = make_ulonglong2(0ull, 0ull);
     if (kObjective == 1) cv = __ldg(reinterpret_cast<const ulonglong2*>(cb + row_i + off));
-    pair_t ta, tb;
-    const ulonglong2 o = update_core<kObjective, kFastNoise>(p.alpha, p.sigma, p.tail, p.keys, e.iter_lo, e.ctr3,
-                                                             (uint32_t)q + p.q_offset, (uint32_t)e.worker, xv, cv, xm, e.w,
-                                                             (p.tail != 0) && (q == p.nq - 1), ta, tb);
+    const bool ragged = (p.tail != 0) && (q == p.nq - 1);
+    ulonglong2 o;
+#pragma unroll
+    for (int h = 0; h < kHalves; ++h) {
+      pair_t ta, tb;
+      const ulonglong2 oh = update_core<kObjective, kFastNoise>(
+          p.alpha, p.sigma, p.keys, e.iter_lo, e.ctr3, (uint32_t)q * kHalves + h + p.q_offset, (uint32_t)e.worker,
+          group_half<kHalves>(xv, h), group_half<kHalves>(cv, h), group_half<kHalves>(xm, h), e.w,
+          live_lanes(ragged, p.tail, h), ta, tb);
+      if (kHalves == 1) o = oh;
+      else if (h == 0) o.x = narrow_bf16x4(oh);
+      else o.y = narrow_bf16x4(oh);
+    }
     *reinterpret_cast<ulonglong2*>(xb + row_i + off) = o;
   }
 }
 
 // ------------------------------------------------------------------------- init / IO
 struct InitParams {
-  float4* dst;  // [M][ldq]
+  float4* dst;  // [M][ldq] column groups
   int64_t ldq, nq;
-  int32_t M, tail;
+  int32_t M, tail;  // tail = d % (4 kHalves)
   float stddev;
   uint32_t tag;
   uint32_t q_offset;
   PhiloxKeys keys;
 };
 
+template <int kHalves>
 __global__ void __launch_bounds__(256) init_normal_kernel(const InitParams p) {
   const int64_t total = (int64_t)p.M * p.nq;
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
        idx += (int64_t)gridDim.x * blockDim.x) {
     const int64_t i = idx / p.nq, q = idx - i * p.nq;
-    float4 z = normals4<false>(philox4x32_10((uint32_t)q + p.q_offset, (uint32_t)i, 0u, p.tag, p.keys));
-    z.x *= p.stddev; z.y *= p.stddev; z.z *= p.stddev; z.w *= p.stddev;
-    if (p.tail != 0 && q == p.nq - 1) {
-      if (p.tail < 2) z.y = 0.f;
-      if (p.tail < 3) z.z = 0.f;
-      z.w = 0.f;
+    const bool ragged = p.tail != 0 && q == p.nq - 1;
+    ulonglong2 o;
+#pragma unroll
+    for (int h = 0; h < kHalves; ++h) {
+      float4 z = normals4<false>(philox4x32_10((uint32_t)q * kHalves + h + p.q_offset, (uint32_t)i, 0u, p.tag, p.keys));
+      z.x *= p.stddev; z.y *= p.stddev; z.z *= p.stddev; z.w *= p.stddev;
+      const int live = live_lanes(ragged, p.tail, h);
+      if (live < 1) z.x = 0.f;
+      if (live < 2) z.y = 0.f;
+      if (live < 3) z.z = 0.f;
+      if (live < 4) z.w = 0.f;
+      const ulonglong2 v = make_ulonglong2(pack2(z.x, z.y), pack2(z.z, z.w));
+      if (kHalves == 1) o = v;
+      else if (h == 0) o.x = narrow_bf16x4(v);
+      else o.y = narrow_bf16x4(v);
     }
-    p.dst[(size_t)i * p.ldq + q] = z;
+    *reinterpret_cast<ulonglong2*>(p.dst + (size_t)i * p.ldq + q) = o;
   }
 }
 
-__global__ void __launch_bounds__(256) gather_columns_kernel(const float* x, int64_t ld, int32_t M, const int64_t* cols,
-                                                             int64_t n_cols, float* out) {
+// One stored element as fp32 (bfloat16 widens exactly).
+__device__ __forceinline__ float load_element(const void* plane, size_t index, bool bf16) {
+  if (bf16) return __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(plane)[index] << 16);
+  return reinterpret_cast<const float*>(plane)[index];
+}
+
+__global__ void __launch_bounds__(256) gather_columns_kernel(const void* x, bool bf16, int64_t ld, int32_t M,
+                                                             const int64_t* cols, int64_t n_cols, float* out) {
   const int64_t total = (int64_t)M * n_cols;
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
        idx += (int64_t)gridDim.x * blockDim.x) {
     const int64_t i = idx / n_cols, k = idx - i * n_cols;
-    out[idx] = x[(size_t)i * ld + cols[k]];
+    out[idx] = load_element(x, (size_t)i * ld + cols[k], bf16);
+  }
+}
+
+// bfloat16 state <-> dense fp32 rows (host transfers of a bfloat16 context are staged in fp32
+// on the device): `rows` rows of d elements; the bfloat16 side has row stride ld.
+__global__ void __launch_bounds__(256) narrow_rows_kernel(const float* src, unsigned short* dst, int64_t rows, int64_t d,
+                                                          int64_t ld) {
+  const int64_t total = rows * d;
+  for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
+       idx += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = idx / d, e = idx - i * d;
+    unsigned short v;
+    asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(v) : "f"(src[idx]));
+    dst[(size_t)i * ld + e] = v;
+  }
+}
+
+__global__ void __launch_bounds__(256) widen_rows_kernel(const unsigned short* src, float* dst, int64_t rows, int64_t d,
+                                                         int64_t ld) {
+  const int64_t total = rows * d;
+  for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
+       idx += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = idx / d, e = idx - i * d;
+    dst[idx] = __uint_as_float((uint32_t)src[(size_t)i * ld + e] << 16);
   }
 }
 

@@ -64,6 +64,18 @@ __device__ __forceinline__ float radius_uniform(uint32_t a) {
   return __uint_as_float(0x3F800000u | (a >> 9)) - 0.99999994039535522461f;
 }
 
+// Hardware log2 of a normal number (u1 >= 2^-24 here, so flushing subnormals changes nothing
+// and saves the subnormal-input handling around the instruction).
+__device__ __forceinline__ float log2_fast(float v) {
+#ifdef NETMAX_LG2_NO_FTZ
+  return __log2f(v);
+#else
+  float r;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+  return r;
+#endif
+}
+
 // Fast pair: hardware log2 / sin / cos / sqrt approximations.  The absolute error of each
 // normal is about 2e-7 for typical radii and is bounded by 6e-4 for radii below 1e-3
 // (probability 5e-7), far inside the replica tolerance after scaling by alpha*sigma.
@@ -71,7 +83,7 @@ __device__ __forceinline__ void normal_pair_fast(uint32_t a, uint32_t b, float& 
   const float u1 = radius_uniform(a);
   // angle = 2 pi u2 with u2 = top24(b)/2^24 taken modulo 1 into [-1/2, 1/2)
   const float ang = (float)((int32_t)b >> 8) * 3.74507028e-07f;  // 2 pi / 2^24
-  const float r2 = fmaxf(-1.38629436111989f * __log2f(u1), 0.0f);  // -2 ln 2 * log2(u1)
+  const float r2 = fmaxf(-1.38629436111989f * log2_fast(u1), 0.0f);  // -2 ln 2 * log2(u1)
   float rad;
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(r2));
   float s, c;
@@ -122,7 +134,7 @@ __device__ __forceinline__ pair_t add2(pair_t a, pair_t b) {
 __device__ __forceinline__ pair_t normal_pair_fast_packed(uint32_t a, uint32_t b) {
   const float u1 = radius_uniform(a);
   const float ang = (float)((int32_t)b >> 8) * 3.74507028e-07f;
-  const float r2 = fmaxf(-1.38629436111989f * __log2f(u1), 0.0f);
+  const float r2 = fmaxf(-1.38629436111989f * log2_fast(u1), 0.0f);
   float rad;
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(r2));
   float s, c;

@@ -144,3 +144,33 @@ def test_consensus_still_contracts_to_the_grid_floor():
     x = s.x()
     assert ((x.max(axis=0) <= hi0 + bf16_ulp(hi0)) & (x.min(axis=0) >= lo0 - bf16_ulp(lo0))).all()
     assert (x.max(axis=0) - x.min(axis=0)).mean() < 0.05 * spread0
+
+
+def test_asynchronous_step_is_the_double_precision_step_rounded_once():
+    """One global step of the asynchronous timeline from a common bfloat16 state: the bf16-mode
+    step and the double-mode step change the same single replica and agree to half a bfloat16
+    unit plus fp32 rounding noise; every other replica is untouched, bit for bit."""
+    rng = np.random.default_rng(9)
+    M, d, lr, sigma = 5, 777, 0.06, 0.2
+    P = policy(M, rng)
+    t = rng.uniform(1.0, 3.0, (M, M))
+    x0 = oracle.bf16_round(rng.standard_normal((M, d)).astype(np.float32))
+    c0 = oracle.bf16_round(rng.standard_normal((M, d)).astype(np.float32))
+    sims = {}
+    for storage in ("bf16", "f32"):
+        s = oracle.Sim(M, d, P, np.ones((M, M), np.uint8), lr, 0.3, sigma, 1, 21, storage=storage)
+        s.set_x(x0)
+        s.set_c(c0)
+        s.async_begin(t, 0.5)
+        s.async_steps(1)
+        sims[storage] = s
+    wb, wd = sims["bf16"].async_trace(), sims["f32"].async_trace()
+    assert all((a == b).all() for a, b in zip(wb, wd))
+    i = int(wb[0][0])
+    xb, xd = sims["bf16"].x(), sims["f32"].x()
+    others = np.arange(M) != i
+    assert (xb[others] == x0[others]).all() and (xd[others] == x0[others]).all()
+    assert (xb[i].view(np.uint32) & 0xFFFF == 0).all() and (xb[i] != x0[i]).mean() > 0.5
+    scale = 1.0 + np.abs(x0[i]).astype(np.float64) + np.abs(c0[i]) + 4.0 * sigma
+    assert (np.abs(xb[i].astype(np.float64) - xd[i]) <= 0.5 * bf16_ulp(xb[i]) + 6 * 2.0 ** -24 * scale).all()
+    assert (oracle.bf16_round(sims["bf16"].unrounded()[i]) == xb[i]).all()
