@@ -4,9 +4,14 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl ours|reference]
 
 A step is one round: every worker of the workload draws a peer, takes its noisy SGD step and
-pulls from the peer's round-start replica, over all M x d elements (one fused kernel launch).
-The metric is replica GB/s = 16 bytes x M x d x rounds / time (reads of x_i, x_peer and c_i
-plus the write of x_i', 4 bytes each).  One JSON line is printed by rank 0.
+pulls from the peer's round-start replica, over all M x d elements.  The metric is replica
+GB/s = 16 bytes x M x d x rounds / time (reads of x_i, x_peer and c_i plus the write of x_i',
+4 bytes each).  One JSON line is printed by rank 0.
+
+The library advances up to four rounds per launch where all M rows of a column tile fit in
+shared memory (M <= 18, fp32 state); that launch is bound by instruction issue, not by HBM,
+and the line's `roofline` says so.  The same workload with one launch per round (the HBM-bound
+kernel) is timed as well and reported under `one_launch_per_round`.
 
 With --gpus N > 1 (launched under torch.distributed.run) the replicas are sharded by columns:
 every rank holds d columns of an N*d-long problem (weak scaling), draws the same peers from
@@ -41,7 +46,10 @@ FALLBACK_HBM_GBS = 6650.0
 KERNEL_SOURCES = ("netmax_kernels.cuh", "netmax_rng.cuh")
 # dram__bytes_read.sum + dram__bytes_write.sum of one round-kernel launch, from an ncu capture
 # (see profiles/); only reported while the kernel sources still hash to the value captured.
-NCU_TRAFFIC = {("b613ba2052dedcf1", "cfg2_M8_resnet18"): 1_041_897_000}
+NCU_TRAFFIC = {}
+# smsp__inst_executed.sum of one launch / (elements x rounds of the launch), from the same captures
+NCU_WARP_INST_PER_ELEMENT_ROUND = {}
+SM_COUNT, SCHEDULERS_PER_SM = 148, 4     # one warp instruction per scheduler and clock at most
 
 
 def kernel_source_hash() -> str:
@@ -250,7 +258,7 @@ def run_ours(args, w):
     g = binding.Netmax(M=w.M, d=w.d, lr=w.lr, link_speed_gbps=speeds, prob=P, rho=rho, sigma=w.sigma,
                        x0_std=w.x0_std, c_std=w.c_std, objective=1, seed=w.seed, device=local,
                        stream=stream.cuda_stream, trace_rounds=ring, workspace=ws_ptr, workspace_bytes=size,
-                       element_offset=plan["element_offset"], storage=args.storage)
+                       element_offset=plan["element_offset"], storage=args.storage, fuse_rounds=args.fuse_rounds)
 
     def barrier():
         torch.cuda.synchronize()
@@ -283,16 +291,29 @@ def run_ours(args, w):
 
     # five more untimed-by-the-contract repeats of a shorter run: best and median per round
     rep_rounds = max(1, min(args.steps, 200))
-    rep_ms = []
-    for _ in range(5):
-        barrier()
-        with torch.cuda.stream(stream):
-            start.record()
-        g.round(rep_rounds)
-        with torch.cuda.stream(stream):
-            stop.record()
-        stop.synchronize()
-        rep_ms.append(start.elapsed_time(stop) / rep_rounds)
+
+    def repeats():
+        out = []
+        for _ in range(5):
+            barrier()
+            with torch.cuda.stream(stream):
+                start.record()
+            g.round(rep_rounds)
+            with torch.cuda.stream(stream):
+                stop.record()
+            stop.synchronize()
+            out.append(start.elapsed_time(stop) / rep_rounds)
+        return out
+
+    rep_ms = repeats()
+    rounds_per_launch = args.steps / max(1, launches - (args.steps + ring - 1) // ring)   # sampler launches excluded
+    fused = 1.5 < rounds_per_launch <= 4.5      # (short vectors run thousands of rounds per cooperative launch)
+    single_ms = None
+    if fused:                       # the same rounds, one launch each: the HBM-bound kernel
+        g.set_fuse_rounds(1)
+        g.round(args.warmup)
+        single_ms = repeats()
+        g.set_fuse_rounds(args.fuse_rounds)
 
     # end to end through the C ABI with host buffers: upload x and c, one round, download x'
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -347,7 +368,26 @@ def run_ours(args, w):
     peak, peak_kind = measured_peak()
     per_launch_ms = ms / args.steps
     achieved = bytes_per_element * elements / (per_launch_ms / 1e3) / 1e9
-    traffic = NCU_TRAFFIC.get((kernel_source_hash(), w.name + ("/bf16" if bf16 else "")))
+    tag = w.name + ("/bf16" if bf16 else "")
+    khash = kernel_source_hash()
+    if fused:
+        # several rounds per launch over a resident tile: bound by instruction issue
+        ipe = NCU_WARP_INST_PER_ELEMENT_ROUND.get((khash, tag + "/fused"))
+        sm_max_ghz = (clocks.summary()["sm_max_mhz"] or 1965) / 1e3
+        alu_peak = SM_COUNT * SCHEDULERS_PER_SM * sm_max_ghz           # G warp instructions / s
+        alu_achieved = None if ipe is None else ipe * elements / (per_launch_ms / 1e3) / 1e9
+        roofline = {"bound": "alu", "achieved": alu_achieved, "peak": alu_peak, "unit": "Gwarp-inst/s",
+                    "frac": None if alu_achieved is None else alu_achieved / alu_peak,
+                    "traffic": NCU_TRAFFIC.get((khash, tag + "/fused")),
+                    "peak_kind": "148 SMs x 4 schedulers x 1 warp instruction per clock x clocks.max.sm",
+                    "kernel": "fused_rounds_kernel", "rounds_per_launch": rounds_per_launch,
+                    "warp_inst_per_element_round": ipe,
+                    "bytes_per_launch": bytes_per_element * elements * rounds_per_launch,
+                    "replica_GBs_over_hbm_peak": achieved / peak, "hbm_peak": peak, "hbm_peak_kind": f"of {peak_kind}"}
+    else:
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": NCU_TRAFFIC.get((khash, tag)), "peak_kind": f"of {peak_kind}", "kernel": "round_kernel",
+                    "bytes_per_launch": bytes_per_element * elements, "frac_of_nominal_8TBs": achieved / 8000.0}
     line = {
         "metric": "replica GB/s", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": per_launch_ms, "higher_is_better": True, "scaling": "weak",
@@ -361,10 +401,7 @@ def run_ours(args, w):
         "hbm_footprint_bytes": int(size),
         "rounds_per_s": args.steps / sec, "peer_draws_per_s": w.M * world * args.steps / sec,
         "sampler_only_draws_per_s": sampler_draws_per_s,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "round_kernel",
-                     "bytes_per_launch": bytes_per_element * elements,
-                     "frac_of_nominal_8TBs": achieved / 8000.0},
+        "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": 2 * elements * 4,
                 "d2h_bytes_per_step": elements * 4, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
                 "wall_ms_per_step": e2e_wall * 1e3 / e2e_steps},
@@ -374,6 +411,14 @@ def run_ours(args, w):
         "paper_context": "paper: 3.7x/3.4x/1.9x faster convergence than Prague/Allreduce-SGD/AD-PSGD "
                          "(ResNet18, 8x RTX 2080 Ti, throttled 1 GbE); not comparable to this metric",
     }
+    if single_ms is not None:
+        one = bytes_per_element * elements / (min(single_ms) / 1e3) / 1e9
+        line["one_launch_per_round"] = {
+            "ms_per_step_best": min(single_ms), "ms_per_step_median": statistics.median(single_ms),
+            "roofline": {"bound": "hbm", "achieved": one, "peak": peak, "unit": "GB/s", "frac": one / peak,
+                         "traffic": NCU_TRAFFIC.get((khash, tag)), "peak_kind": f"of {peak_kind}",
+                         "kernel": "round_kernel", "bytes_per_launch": bytes_per_element * elements,
+                         "frac_of_nominal_8TBs": one / 8000.0}}
     if base is not None:
         line["cpu_baseline"] = base
     g.close()
@@ -448,6 +493,8 @@ def main():
     ap.add_argument("--d", type=int, default=0, help="override the workload's vector length (profiling on a smaller case)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fuse-rounds", type=int, default=0,
+                    help="rounds per launch over a resident tile: 0 automatic, 1 one launch per round, 2..4")
     ap.add_argument("--storage", choices=["f32", "bf16"], default="f32",
                     help="precision of the replicas in device memory (arithmetic is fp32 either way)")
     ap.add_argument("--mode", choices=["rounds", "async"], default="rounds",

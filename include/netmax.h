@@ -103,6 +103,10 @@ typedef struct netmax_config {
                                     allocates with cudaMalloc and frees in netmax_destroy              */
   size_t workspace_bytes;
   int32_t storage;               /* NETMAX_STORAGE_F32 (default) or NETMAX_STORAGE_BF16: see above       */
+  int32_t fuse_rounds;           /* rounds that one launch may advance a tile of long vectors while it is
+                                    resident on chip (see netmax_round): 0 (default) automatic, 1 never
+                                    (one launch per round), 2..4 at most that many.  Replicas and peer
+                                    traces do not depend on it                                           */
 } netmax_config;
 
 /* Fills *cfg with defaults: rho = 0 (automatic), sigma = 0, stds 0, objective 1, seed 0,
@@ -152,9 +156,20 @@ int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
  * Short vectors (a round of a few microseconds) run all rounds of a call in one cooperative
  * launch with a grid-wide barrier per round; its waits are bounded, and one that runs out is
  * reported by the next synchronising call as NETMAX_CUDA_ERROR (the replicas are then not
- * valid).  Either way the results are the same, bit for bit, however a run is split into calls.
+ * valid).
+ * Long vectors with at most 18 workers and fp32 state advance up to four rounds per launch
+ * (netmax_config.fuse_rounds): given the draws, Eq. 16 acts on every column separately, so a
+ * tile holding all M rows of a column range stays in shared memory for those rounds and HBM
+ * sees x and c once per launch instead of once per round.
+ * Whatever the launch shape and however a run is split into calls, replicas and peer traces
+ * are the same bit for bit; telemetry sums are accumulated in double precision in an order
+ * that depends on the launch shape and agree to rounding (1e-12 relative).
  */
 int netmax_round(netmax_ctx* ctx, int64_t n_rounds);
+
+/* Changes netmax_config.fuse_rounds for the rounds that follow (0 automatic, 1 one launch per
+ * round, 2..4 at most that many rounds per launch). */
+int netmax_set_fuse_rounds(netmax_ctx* ctx, int32_t fuse_rounds);
 
 /* Number of rounds enqueued so far. */
 int64_t netmax_rounds_done(const netmax_ctx* ctx);

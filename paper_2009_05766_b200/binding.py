@@ -21,7 +21,7 @@ STATUS = {0: "OK", -1: "INVALID_ARG", -2: "BAD_PROB_ROW", -3: "OOM", -4: "CUDA_E
 EXPORTS = [
     "netmax_config_init", "netmax_workspace_size", "netmax_create_ex", "netmax_create", "netmax_destroy",
     "netmax_set_policy", "netmax_get_policy", "netmax_set_replicas", "netmax_set_centres", "netmax_round",
-    "netmax_rounds_done", "netmax_read_replicas", "netmax_read_centres", "netmax_read_columns",
+    "netmax_rounds_done", "netmax_set_fuse_rounds", "netmax_read_replicas", "netmax_read_centres", "netmax_read_columns",
     "netmax_read_columns_static",
     "netmax_peer_trace", "netmax_telemetry", "netmax_replicas_device", "netmax_sample_peers",
     "netmax_measure", "netmax_async_begin", "netmax_async_set_times", "netmax_async_steps", "netmax_async_time",
@@ -43,6 +43,7 @@ class Config(C.Structure):
         ("c_std", C.c_double), ("objective", C.c_int32), ("seed", C.c_uint64), ("device", C.c_int32),
         ("stream", C.c_void_p), ("trace_rounds", C.c_int64), ("policy_K", C.c_int32), ("policy_R", C.c_int32), ("policy_rho_upper", C.c_double),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("storage", C.c_int32),
+        ("fuse_rounds", C.c_int32),
     ]
 
 STORAGE = {"f32": 0, "bf16": 1}
@@ -76,6 +77,7 @@ def lib():
             "netmax_set_centres": ([vp, vp], C.c_int),
             "netmax_round": ([vp, i64], C.c_int),
             "netmax_rounds_done": ([vp], i64),
+            "netmax_set_fuse_rounds": ([vp, i32], C.c_int),
             "netmax_read_replicas": ([vp, vp], C.c_int),
             "netmax_read_centres": ([vp, vp], C.c_int),
             "netmax_read_columns": ([vp, vp, i64, vp], C.c_int),
@@ -169,7 +171,7 @@ class Netmax:
                  device: int = 0, stream: Optional[int] = None, trace_rounds: int = 1024, policy_K: int = 20,
                  policy_R: int = 20, workspace: Optional[int] = None, workspace_bytes: int = 0,
                  element_offset: int = 0, pull_weight: float = 0.0, policy_rho_upper: float = 0.0,
-                 storage: str = "f32"):
+                 storage: str = "f32", fuse_rounds: int = 0):
         L = lib()
         cfg = Config()
         _check(L.netmax_config_init(C.byref(cfg)))
@@ -188,6 +190,7 @@ class Netmax:
         cfg.policy_rho_upper = float(policy_rho_upper)
         cfg.workspace, cfg.workspace_bytes = workspace, int(workspace_bytes)
         cfg.storage = STORAGE[storage]
+        cfg.fuse_rounds = int(fuse_rounds)
         self.storage = storage
         self.M, self.d = int(M), int(d)
         self._h = C.c_void_p()
@@ -249,6 +252,9 @@ class Netmax:
 
     def round(self, n_rounds: int = 1):
         _check(lib().netmax_round(self._h, int(n_rounds)), self._h)
+
+    def set_fuse_rounds(self, fuse_rounds: int):
+        _check(lib().netmax_set_fuse_rounds(self._h, int(fuse_rounds)), self._h)
 
     @property
     def rounds_done(self) -> int:

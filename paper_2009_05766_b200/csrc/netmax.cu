@@ -148,6 +148,7 @@ struct netmax_ctx {
   uint64_t seed = 0;
   int policy_K = 20, policy_R = 20;
   double policy_rho_upper = 0.0;
+  int fuse_rounds = 0;  // 0: automatic, 1: one launch per round, 2..kFusedMaxRounds: rounds per fused launch
   PhiloxKeys keys;
   std::vector<double> P;      // policy in force
   std::vector<uint8_t> adj;   // link graph in force
@@ -387,6 +388,9 @@ template <int kHalves>
 RoundKernel pick_kernel_h(int objective, bool short_vectors) {
   if (objective == 2) return short_vectors ? round_kernel<2, true, 4, kHalves> : round_kernel<2, true, 1, kHalves>;
   if (short_vectors) return objective == 1 ? round_kernel<1, true, 4, kHalves> : round_kernel<0, true, 4, kHalves>;
+#ifdef NETMAX_BF16_LONG_RIF
+  if (kHalves == 2) return objective == 1 ? round_kernel<1, true, NETMAX_BF16_LONG_RIF, kHalves> : round_kernel<0, true, NETMAX_BF16_LONG_RIF, kHalves>;
+#endif
   return objective == 1 ? round_kernel<1, true, 1, kHalves> : round_kernel<0, true, 1, kHalves>;
 }
 RoundKernel pick_kernel(int objective, bool short_vectors, int halves) {
@@ -398,6 +402,12 @@ using MultiRoundKernel = void (*)(const MultiRoundParams);
 MultiRoundKernel pick_multi_kernel(int objective, int halves) {
   if (halves == 2) return objective == 1 ? multi_round_kernel<1, true, 2> : multi_round_kernel<0, true, 2>;
   return objective == 1 ? multi_round_kernel<1, true, 1> : multi_round_kernel<0, true, 1>;
+}
+
+using FusedKernel = void (*)(const FusedParams);
+
+FusedKernel pick_fused_kernel(int objective) {
+  return objective == 1 ? fused_rounds_kernel<1, true> : fused_rounds_kernel<0, true>;
 }
 
 int floor_pow2(int64_t v) {
@@ -463,6 +473,40 @@ int plan_round(netmax_ctx* ctx, RoundPlan& plan, int objective) {
   return NETMAX_OK;
 }
 
+// Several rounds per launch over shared-memory-resident tiles (fused_rounds_kernel): long
+// vectors, fp32 state, and few enough workers that two CTAs' slabs (48 bytes per worker and
+// thread) fit on an SM.
+struct FusedPlan {
+  bool ok = false;
+  int threads = 0, grid = 0, max_rounds = 0;
+  size_t smem = 0;
+  int64_t n_tiles = 0;
+};
+
+int plan_fused(netmax_ctx* ctx, const RoundPlan& plan, FusedPlan& f) {
+  f.ok = false;
+  if (ctx->fuse_rounds == 1 || plan.short_vectors || ctx->storage != NETMAX_STORAGE_F32) return NETMAX_OK;
+  const int64_t M = ctx->M;
+  const size_t head = align_up((size_t)kFusedMaxRounds * M * 8, 128);
+  const size_t budget = 113 * 1024;  // two CTAs per SM
+  int threads = 0;
+  for (int cand : {256, 128})
+    if (head + (size_t)48 * M * cand + 64 * sizeof(double) <= budget) { threads = cand; break; }
+  if (threads == 0) return NETMAX_OK;
+  f.threads = threads;
+  f.smem = head + (size_t)48 * M * threads + 64 * sizeof(double);
+  f.max_rounds = ctx->fuse_rounds >= 2 ? std::min(ctx->fuse_rounds, kFusedMaxRounds) : kFusedMaxRounds;
+  f.n_tiles = (ctx->L.nq + threads - 1) / threads;
+  FusedKernel k = pick_fused_kernel(ctx->objective);
+  NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)f.smem));
+  int per_sm = 0;
+  NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, threads, f.smem));
+  if (per_sm < 1) return NETMAX_OK;
+  f.grid = (int)std::min<int64_t>(f.n_tiles, std::min<int64_t>((int64_t)per_sm * ctx->sm_count, kMaxGrid));
+  f.ok = true;
+  return NETMAX_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -488,6 +532,8 @@ static int check_sizes(const netmax_config* cfg) {
   if (cfg->element_offset < 0 || cfg->element_offset % 4 != 0 || cfg->element_offset + cfg->d >= kMaxD)
     return fail(nullptr, NETMAX_INVALID_ARG, "element_offset = %lld must be a non-negative multiple of 4 with offset + d < 2^30 - 32", (long long)cfg->element_offset);
   if (cfg->trace_rounds < 1) return fail(nullptr, NETMAX_INVALID_ARG, "trace_rounds = %lld < 1", (long long)cfg->trace_rounds);
+  if (cfg->fuse_rounds < 0 || cfg->fuse_rounds > kFusedMaxRounds)
+    return fail(nullptr, NETMAX_INVALID_ARG, "fuse_rounds = %d outside [0, %d]", cfg->fuse_rounds, kFusedMaxRounds);
   return NETMAX_OK;
 }
 
@@ -537,6 +583,7 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   ctx->policy_rho_upper = cfg->policy_rho_upper > 0.0 ? cfg->policy_rho_upper : 0.0;
   ctx->keys = make_philox_keys(cfg->seed);
   ctx->storage = cfg->storage;
+  ctx->fuse_rounds = cfg->fuse_rounds;
   ctx->L = make_layout(cfg->M, cfg->d, cfg->trace_rounds, cfg->storage);
 
   rc = build_adjacency(ctx, cfg->M, cfg->link_speed_gbps, ctx->adj);
@@ -758,6 +805,9 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   int rc = plan_round(ctx, plan, ctx->objective);
   if (rc) return rc;
   RoundKernel kernel = pick_kernel(ctx->objective, plan.short_vectors, ctx->L.halves);
+  FusedPlan fused;
+  rc = plan_fused(ctx, plan, fused);
+  if (rc) return rc;
 
   RoundParams p;
   p.c = reinterpret_cast<const float4*>(ctx->c);
@@ -823,7 +873,40 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
       done += batch;
       continue;
     }
-    for (int64_t b = 0; b < batch; ++b) {
+    for (int64_t b = 0; b < batch;) {
+      if (fused.ok && batch - b >= 2) {  // the next rounds in one launch over resident tiles
+        const int chunk = (int)std::min<int64_t>(batch - b, fused.max_rounds);
+        FusedParams fp;
+        fp.x_cur = reinterpret_cast<const float4*>(ctx->x[ctx->cur]);
+        fp.x_nxt = reinterpret_cast<float4*>(ctx->x[ctx->cur ^ 1]);
+        fp.c = p.c;
+        fp.trace = ctx->trace;
+        fp.wtab = ctx->wtab;
+        fp.tel = ctx->tel;
+        fp.partials = ctx->partials;
+        fp.ticket = ctx->ticket;
+        fp.slot0 = ctx->rounds % ctx->trace_rounds;
+        fp.ring = ctx->trace_rounds;
+        fp.first_round = (uint64_t)ctx->rounds;
+        fp.n_rounds = chunk;
+        fp.ldq = p.ldq;
+        fp.nq = p.nq;
+        fp.n_tiles = fused.n_tiles;
+        fp.row_bytes = p.row_bytes;
+        fp.M = p.M;
+        fp.tail = p.tail;
+        fp.alpha = p.alpha;
+        fp.sigma = p.sigma;
+        fp.inv_M = p.inv_M;
+        fp.q_offset = p.q_offset;
+        fp.keys = p.keys;
+        pick_fused_kernel(ctx->objective)<<<fused.grid, fused.threads, fused.smem, ctx->stream>>>(fp);
+        ctx->launches += 1;
+        ctx->cur ^= 1;
+        ctx->rounds += chunk;
+        b += chunk;
+        continue;
+      }
       const uint64_t r = (uint64_t)ctx->rounds;
       const int64_t slot = (int64_t)(r % (uint64_t)ctx->trace_rounds);
       p.x_cur = reinterpret_cast<const float4*>(ctx->x[ctx->cur]);
@@ -836,6 +919,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
       ctx->launches += 1;
       ctx->cur ^= 1;
       ctx->rounds += 1;
+      b += 1;
     }
     NM_CUDA(ctx, cudaGetLastError());
     done += batch;
@@ -844,6 +928,14 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
 }
 
 int64_t netmax_rounds_done(const netmax_ctx* ctx) { return ctx ? ctx->rounds : -1; }
+
+int netmax_set_fuse_rounds(netmax_ctx* ctx, int32_t fuse_rounds) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (fuse_rounds < 0 || fuse_rounds > kFusedMaxRounds)
+    return fail(ctx, NETMAX_INVALID_ARG, "fuse_rounds = %d outside [0, %d]", fuse_rounds, kFusedMaxRounds);
+  ctx->fuse_rounds = fuse_rounds;
+  return NETMAX_OK;
+}
 
 int netmax_read_columns(netmax_ctx* ctx, const int64_t* host_cols, int64_t n_cols, float* host_out) {
   if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");

@@ -169,9 +169,10 @@ __device__ __forceinline__ ulonglong2 update_core(float alpha, float sigma, cons
 
 // update_core plus the telemetry sums of the round-start values.  kObjective == 2 measures only.
 template <int kObjective, bool kFastNoise>
-__device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t round_lo, uint32_t ctr3, uint32_t q32,
-                                                 uint32_t worker, ulonglong2 xv, ulonglong2 cv, ulonglong2 xm,
-                                                 ulonglong2 pivot, float w, int live, ColAcc& acc, LossAcc& lacc) {
+__device__ __forceinline__ ulonglong2 row_update(float alpha, float sigma, const PhiloxKeys& keys, uint32_t round_lo,
+                                                 uint32_t ctr3, uint32_t q32, uint32_t worker, ulonglong2 xv, ulonglong2 cv,
+                                                 ulonglong2 xm, ulonglong2 pivot, float w, int live, ColAcc& acc,
+                                                 LossAcc& lacc) {
   const pair_t neg1 = pack2(-1.0f, -1.0f);
   pair_t ta, tb;
   ulonglong2 o = xv;
@@ -179,8 +180,7 @@ __device__ __forceinline__ ulonglong2 row_update(const RoundParams& p, uint32_t 
     ta = fma2(cv.x, neg1, xv.x);
     tb = fma2(cv.y, neg1, xv.y);
   } else {
-    o = update_core<kObjective, kFastNoise>(p.alpha, p.sigma, p.keys, round_lo, ctr3, q32, worker, xv, cv, xm, w, live,
-                                            ta, tb);
+    o = update_core<kObjective, kFastNoise>(alpha, sigma, keys, round_lo, ctr3, q32, worker, xv, cv, xm, w, live, ta, tb);
   }
   const pair_t da = fma2(pivot.x, neg1, xv.x), db = fma2(pivot.y, neg1, xv.y);  // x - pivot
   acc.s1a = add2(acc.s1a, da);
@@ -280,7 +280,7 @@ __device__ __forceinline__ void finalize_telemetry(const RoundParams& p, double 
 #define NETMAX_ROUND_MIN_CTAS 4  // CTAs per SM the register allocation leaves room for
 #endif
 #ifndef NETMAX_ROUND_MIN_CTAS_BF16
-#define NETMAX_ROUND_MIN_CTAS_BF16 3  // bfloat16 state: eight elements per thread need more registers
+#define NETMAX_ROUND_MIN_CTAS_BF16 2  // bfloat16 state: eight elements per thread; measured 152 us (2), 161 (3), 157 (4) per cfg2 round
 #endif
 
 // kRowsInFlight = 1 (64 registers, 4 CTAs/SM) is the streaming shape for long vectors, where
@@ -373,7 +373,7 @@ __device__ __forceinline__ void round_tiles(const RoundParams& p, const float4* 
 #pragma unroll
             for (int h = 0; h < kHalves; ++h) {
               const ulonglong2 oh = row_update<kObjective, kFastNoise>(
-                  p, round_lo, ctr3, q32 + h, (uint32_t)i, group_half<kHalves>(xv[u], h), group_half<kHalves>(cv[u], h),
+                  p.alpha, p.sigma, p.keys, round_lo, ctr3, q32 + h, (uint32_t)i, group_half<kHalves>(xv[u], h), group_half<kHalves>(cv[u], h),
                   group_half<kHalves>(xm[u], h), group_half<kHalves>(pivot, h), __int_as_float(pw[u].y),
                   live_lanes(ragged, p.tail, h), acc[h], lacc);
               if (kHalves == 1) o = oh;
@@ -548,6 +548,150 @@ __global__ void __launch_bounds__(256, 2) multi_round_kernel(const MultiRoundPar
     const float4* t = x_cur;
     x_cur = x_nxt;
     x_nxt = const_cast<float4*>(t);
+  }
+}
+
+// ---- several rounds over one resident tile (long vectors, few workers) -----------------------
+// Given the peer draws, every column of the M x d state evolves on its own (Eq. 16 is
+// elementwise), so a tile that holds ALL M rows of a column range can be advanced several
+// rounds without touching global memory in between: the HBM traffic per element drops from
+// 12 bytes per round (x and c read, x' written; the peer read is a cache hit) to 12 bytes per
+// kFusedMaxRounds rounds, and the kernel becomes bound by its arithmetic instead.
+//
+// A thread owns one 16-byte column group for all M rows.  Its slab of shared memory
+// ([2][M] replica values, double-buffered by round, and [M] centres, each entry 16 bytes,
+// laid out [row][thread] so that a warp's accesses are conflict-free) is private to the thread:
+// the peer's value of the same column group was written by this very thread a round earlier,
+// so the rounds need no barrier.  Per-element arithmetic is row_update's, hence the replicas
+// are bit-identical to one launch per round; telemetry sums only differ in the order of their
+// double-precision accumulation.  fp32 state only.
+#ifndef NETMAX_FUSED_MAX_ROUNDS
+#define NETMAX_FUSED_MAX_ROUNDS 4
+#endif
+#ifndef NETMAX_FUSED_UNROLL
+#define NETMAX_FUSED_UNROLL 2
+#endif
+constexpr int kFusedMaxRounds = NETMAX_FUSED_MAX_ROUNDS;
+constexpr int kFusedUnroll = NETMAX_FUSED_UNROLL;  // rows of a round in flight per thread
+
+struct FusedParams {
+  const float4* x_cur;   // [M][ldq] replicas at the start of the first round
+  float4* x_nxt;         // [M][ldq] replicas after the last round
+  const float4* c;       // [M][ldq]
+  const int32_t* trace;  // peer-trace ring [ring][M], filled for these rounds
+  const float* wtab;     // [M][M]
+  double* tel;           // telemetry ring [ring][2]
+  double* partials;      // [kFusedMaxRounds][gridDim.x][2]
+  unsigned int* ticket;  // last-CTA-done counter (0 between launches)
+  int64_t slot0, ring;   // ring slot of the first round
+  uint64_t first_round;
+  int32_t n_rounds;      // 1 .. kFusedMaxRounds
+  int64_t ldq, nq, n_tiles;
+  uint32_t row_bytes;
+  int32_t M, tail;
+  float alpha, sigma, inv_M;
+  uint32_t q_offset;
+  PhiloxKeys keys;
+};
+
+// Dynamic shared memory: (peer, weight) int2[kFusedMaxRounds][M], then the slabs
+// float4[3][M][blockDim] (replicas of even rounds, of odd rounds, centres), then 64 doubles.
+template <int kObjective, bool kFastNoise>
+__global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams p) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int tid = threadIdx.x, T = blockDim.x, M = p.M;
+  int2* s_pw = reinterpret_cast<int2*>(smem_raw);
+  const size_t head = (((size_t)kFusedMaxRounds * M * 8) + 127) & ~(size_t)127;
+  ulonglong2* s_x = reinterpret_cast<ulonglong2*>(smem_raw + head);  // [2][M][T]
+  ulonglong2* s_c = s_x + (size_t)2 * M * T;                        // [M][T]
+  double* s_red = reinterpret_cast<double*>(s_c + (size_t)M * T);
+
+  for (int k = 0; k < p.n_rounds; ++k) {
+    const int32_t* peers = p.trace + ((p.slot0 + k) % p.ring) * M;
+    for (int i = tid; i < M; i += T) {
+      const int32_t m = __ldg(peers + i);
+      s_pw[k * M + i] = make_int2(m, __float_as_int((m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * M + m)));
+    }
+  }
+  __syncthreads();
+
+  double acc_cons[kFusedMaxRounds], acc_loss[kFusedMaxRounds];
+#pragma unroll
+  for (int k = 0; k < kFusedMaxRounds; ++k) acc_cons[k] = acc_loss[k] = 0.0;
+
+  for (int64_t tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x) {
+    const int64_t q = tile * T + tid;
+    if (q >= p.nq) continue;  // no barrier below: threads are independent
+    const int live_lo = live_lanes((p.tail != 0) && (q == p.nq - 1), p.tail, 0);
+    const uint32_t q32 = (uint32_t)q + p.q_offset;
+    {  // all rows of this column group into the thread's slab
+      const char* xq = reinterpret_cast<const char*>(p.x_cur + q);
+      const char* cq = reinterpret_cast<const char*>(p.c + q);
+#pragma unroll 4
+      for (int i = 0; i < M; ++i) {
+        const uint64_t row = (uint64_t)(uint32_t)i * p.row_bytes;
+        s_x[(size_t)i * T + tid] = __ldg(reinterpret_cast<const ulonglong2*>(xq + row));
+        s_c[(size_t)i * T + tid] = __ldg(reinterpret_cast<const ulonglong2*>(cq + row));
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < kFusedMaxRounds; ++k) {
+      if (k < p.n_rounds) {
+        const uint64_t round = p.first_round + (uint64_t)k;
+        const uint32_t round_lo = (uint32_t)round, ctr3 = philox_ctr3(kTagNoise, round);
+        const ulonglong2* cur = s_x + (size_t)(k & 1) * M * T;
+        ulonglong2* nxt = s_x + (size_t)((k & 1) ^ 1) * M * T;
+        const int2* pw = s_pw + k * M;
+        const ulonglong2 pivot = cur[tid];
+        ColAcc acc;
+        LossAcc lacc;
+#pragma unroll kFusedUnroll
+        for (int i = 0; i < M; ++i) {
+          const int2 d = pw[i];
+          const ulonglong2 o = row_update<kObjective, kFastNoise>(
+              p.alpha, p.sigma, p.keys, round_lo, ctr3, q32, (uint32_t)i, cur[(size_t)i * T + tid], s_c[(size_t)i * T + tid],
+              cur[(size_t)d.x * T + tid], pivot, __int_as_float(d.y), live_lo, acc, lacc);
+          nxt[(size_t)i * T + tid] = o;
+        }
+        float4 s1, s2;
+        unpack2(acc.s1a, s1.x, s1.y);
+        unpack2(acc.s1b, s1.z, s1.w);
+        unpack2(acc.s2a, s2.x, s2.y);
+        unpack2(acc.s2b, s2.z, s2.w);
+        float l0, l1, l2, l3;
+        unpack2(lacc.la, l0, l1);
+        unpack2(lacc.lb, l2, l3);
+        const float cons = (s2.x - s1.x * s1.x * p.inv_M) + (s2.y - s1.y * s1.y * p.inv_M) +
+                           (s2.z - s1.z * s1.z * p.inv_M) + (s2.w - s1.w * s1.w * p.inv_M);
+        acc_cons[k] += (double)cons;
+        acc_loss[k] += (double)((l0 + l1) + (l2 + l3));
+      }
+    }
+    {
+      const ulonglong2* fin = s_x + (size_t)(p.n_rounds & 1) * M * T;
+      char* oq = reinterpret_cast<char*>(p.x_nxt + q);
+#pragma unroll 4
+      for (int i = 0; i < M; ++i)
+        *reinterpret_cast<ulonglong2*>(oq + (uint64_t)(uint32_t)i * p.row_bytes) = fin[(size_t)i * T + tid];
+    }
+  }
+
+  // telemetry: per round, CTA partials; the last CTA to finish sums them in index order
+#pragma unroll
+  for (int k = 0; k < kFusedMaxRounds; ++k)
+    if (k < p.n_rounds) block_partials(p.partials + (size_t)k * 2 * gridDim.x, acc_cons[k], acc_loss[k], s_red);
+  __shared__ bool s_last;
+  if (tid == 0) {
+    __threadfence();
+    const unsigned int t = atomicAdd(p.ticket, 1u);
+    s_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    for (int k = 0; k < p.n_rounds; ++k)
+      sum_partials(p.partials + (size_t)k * 2 * gridDim.x, (double)p.inv_M, p.tel + 2 * ((p.slot0 + k) % p.ring), s_red);
+    if (tid == 0) *p.ticket = 0u;
   }
 }
 

@@ -1,0 +1,101 @@
+"""GPU parity of the launch shape that advances a resident tile several rounds (long vectors,
+few workers; netmax_config.fuse_rounds).  Columns evolve independently given the peer draws, so
+fusing rounds must not change a bit of the replicas or of the peer trace: checked against one
+launch per round on the same context inputs, and against the CPU oracle within the fp32
+tolerance.  Telemetry sums are accumulated in a different order and agree to rounding."""
+import numpy as np
+import pytest
+
+from oracle import oracle
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def nm():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    from paper_2009_05766_b200 import binding
+    binding.lib()
+    return binding
+
+
+def full_adj(M):
+    return (1 - np.eye(M)).astype(np.uint8)
+
+
+def random_policy(M, rng, zeros=0.0):
+    P = rng.random((M, M)) + 0.05
+    if zeros > 0:
+        mask = rng.random((M, M)) < zeros
+        mask[np.arange(M), (np.arange(M) + 1) % M] = False
+        P[mask] = 0.0
+    return P / P.sum(axis=1, keepdims=True)
+
+
+# long vectors: at least two 4 KB-wide tiles per SM, so that the streaming launch shapes are chosen
+@pytest.mark.parametrize("M,d,fuse", [(2, 400_003, 0), (5, 320_001, 0), (8, 400_002, 0), (9, 310_000, 3), (8, 400_001, 2),
+                                      (16, 320_001, 4), (18, 310_003, 4)])
+@pytest.mark.parametrize("objective", [0, 1])
+def test_fused_rounds_change_no_bit(nm, M, d, fuse, objective):
+    rng = np.random.default_rng(M * 11 + d)
+    P = random_policy(M, rng, zeros=0.2 if M > 4 else 0.0)
+    kw = dict(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=objective, seed=d + M, trace_rounds=64)
+    one = nm.Netmax(fuse_rounds=1, **kw)         # one launch per round
+    many = nm.Netmax(fuse_rounds=fuse, **kw)
+    rounds = 0
+    for n in (11, 1, 2, 4, 3):                   # chunks of every length, a lone round in between, ring wrap-around
+        launches = many.kernel_launches
+        one.round(n)
+        many.round(n)
+        rounds += n
+        if n >= 2:
+            assert many.kernel_launches - launches < n + 1, "rounds were not fused"
+    xa, xb = one.read_replicas(), many.read_replicas()
+    assert (xa.view(np.uint32) == xb.view(np.uint32)).all()
+    assert (one.peer_trace(0, rounds) == many.peer_trace(0, rounds)).all()
+    (ca, la), (cb, lb) = one.telemetry(0, rounds), many.telemetry(0, rounds)
+    np.testing.assert_allclose(cb, ca, rtol=1e-12)
+    np.testing.assert_allclose(lb, la, rtol=1e-12)
+    # padding lanes of the rows stay zero
+    import torch
+    ptr, ld = many.replicas_device()
+
+    class _Holder:
+        pass
+
+    h = _Holder()
+    h.__cuda_array_interface__ = {"shape": (M, ld), "typestr": "<f4", "data": (ptr, False), "version": 3, "strides": None}
+    assert float(torch.as_tensor(h, device="cuda")[:, d:].abs().max().item()) == 0.0
+    one.close()
+    many.close()
+
+
+@pytest.mark.parametrize("M,d", [(3, 400_003), (8, 303_107)])
+def test_fused_rounds_match_the_oracle(nm, M, d):
+    rng = np.random.default_rng(M + d)
+    P = random_policy(M, rng)
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=1, seed=7, trace_rounds=32)
+    o = oracle.Sim(M, d, P, full_adj(M), alpha=0.05, rho=g.get_policy()[1], sigma=0.1, objective=1, seed=7)
+    o.init(1.0, 1.0)
+    rounds = 14
+    launches = g.kernel_launches
+    g.round(rounds)
+    assert g.kernel_launches - launches <= 1 + (rounds + 3) // 4     # the sampler and fused launches of four rounds
+    o.round(rounds, threads=8)
+    assert (g.peer_trace() == o.trace()).all()
+    got, want = g.read_replicas().astype(np.float64), o.x().astype(np.float64)
+    assert (np.abs(got - want) <= TOL * (1.0 + np.abs(want))).all()
+    gc, gl = g.telemetry()
+    oc, ol = o.telemetry()
+    np.testing.assert_allclose(gc, oc, rtol=1e-4)
+    np.testing.assert_allclose(gl, ol, rtol=1e-4)
+    g.close()
+
+
+def test_fuse_rounds_out_of_range_is_refused(nm):
+    with pytest.raises(nm.NetmaxError) as e:
+        nm.Netmax(M=2, d=64, lr=0.1, fuse_rounds=5)
+    assert e.value.code == -1
