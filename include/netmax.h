@@ -157,13 +157,14 @@ int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
  * launch with a grid-wide barrier per round; its waits are bounded, and one that runs out is
  * reported by the next synchronising call as NETMAX_CUDA_ERROR (the replicas are then not
  * valid).
- * Long vectors with at most 18 workers and fp32 state advance up to four rounds per launch
+ * Long vectors with at most 18 workers advance up to four rounds per launch
  * (netmax_config.fuse_rounds): given the draws, Eq. 16 acts on every column separately, so a
  * tile holding all M rows of a column range stays in shared memory for those rounds and HBM
  * sees x and c once per launch instead of once per round.
  * Whatever the launch shape and however a run is split into calls, replicas and peer traces
- * are the same bit for bit; telemetry sums are accumulated in double precision in an order
- * that depends on the launch shape and agree to rounding (1e-12 relative).
+ * are the same bit for bit; telemetry sums are accumulated in an order that depends on the
+ * launch shape and agree to rounding (1e-12 relative with fp32 state, 1e-6 with bfloat16
+ * state, whose per-thread fp32 partial sums span eight or four columns).
  */
 int netmax_round(netmax_ctx* ctx, int64_t n_rounds);
 

@@ -45,6 +45,13 @@ struct DeviceGuard {
   }
 };
 
+struct FusedPlan {  // launch shape of fused_rounds_kernel
+  bool ok = false;
+  int threads = 0, grid = 0, max_rounds = 0;
+  size_t smem = 0;
+  int64_t n_tiles = 0;
+};
+
 struct Layout {
   int64_t ld = 0, ldq = 0, nq = 0;  // row stride in elements / in 16-byte column groups; column groups in use
   int elem = 4, halves = 1;         // bytes per stored element; Philox blocks (4 elements) per column group
@@ -149,6 +156,8 @@ struct netmax_ctx {
   int policy_K = 20, policy_R = 20;
   double policy_rho_upper = 0.0;
   int fuse_rounds = 0;  // 0: automatic, 1: one launch per round, 2..kFusedMaxRounds: rounds per fused launch
+  bool fused_planned = false;
+  FusedPlan fused;
   PhiloxKeys keys;
   std::vector<double> P;      // policy in force
   std::vector<uint8_t> adj;   // link graph in force
@@ -406,8 +415,9 @@ MultiRoundKernel pick_multi_kernel(int objective, int halves) {
 
 using FusedKernel = void (*)(const FusedParams);
 
-FusedKernel pick_fused_kernel(int objective) {
-  return objective == 1 ? fused_rounds_kernel<1, true> : fused_rounds_kernel<0, true>;
+FusedKernel pick_fused_kernel(int objective, int halves) {
+  if (halves == 2) return objective == 1 ? fused_rounds_kernel<1, true, true> : fused_rounds_kernel<0, true, true>;
+  return objective == 1 ? fused_rounds_kernel<1, true, false> : fused_rounds_kernel<0, true, false>;
 }
 
 int floor_pow2(int64_t v) {
@@ -473,38 +483,55 @@ int plan_round(netmax_ctx* ctx, RoundPlan& plan, int objective) {
   return NETMAX_OK;
 }
 
-// Several rounds per launch over shared-memory-resident tiles (fused_rounds_kernel): long
-// vectors, fp32 state, and few enough workers that two CTAs' slabs (48 bytes per worker and
-// thread) fit on an SM.
-struct FusedPlan {
-  bool ok = false;
-  int threads = 0, grid = 0, max_rounds = 0;
-  size_t smem = 0;
-  int64_t n_tiles = 0;
-};
-
-int plan_fused(netmax_ctx* ctx, const RoundPlan& plan, FusedPlan& f) {
-  f.ok = false;
-  if (ctx->fuse_rounds == 1 || plan.short_vectors || ctx->storage != NETMAX_STORAGE_F32) return NETMAX_OK;
+int plan_fused_uncached(netmax_ctx* ctx, const RoundPlan& plan, FusedPlan& f) {
+  f = FusedPlan();
+  if (ctx->fuse_rounds == 1 || plan.short_vectors) return NETMAX_OK;
   const int64_t M = ctx->M;
   const size_t head = align_up((size_t)kFusedMaxRounds * M * 8, 128);
-  const size_t budget = 113 * 1024;  // two CTAs per SM
-  int threads = 0;
-  for (int cand : {256, 128})
-    if (head + (size_t)48 * M * cand + 64 * sizeof(double) <= budget) { threads = cand; break; }
-  if (threads == 0) return NETMAX_OK;
+  const size_t fixed = head + 64 * sizeof(double);
+  // 256 or 128 threads per CTA (a multiple of four warps keeps the SM's four schedulers evenly
+  // loaded: 3 x 96 threads measured 587 us per cfg3 round against 508 for 2 x 128), whichever
+  // puts more threads on an SM with at least two CTAs (one loads its tile while the other
+  // computes; M = 16: 1 x 256 threads 529 us).  Every thread needs 48 M bytes of shared memory,
+  // and the kernel's ~100 registers cap an SM at 16 warps (capping it at 96 or 80 registers for
+  // 18-20 warps measured slower: 135 and 157 us against 128 per cfg2 round).
+  FusedKernel k = pick_fused_kernel(ctx->objective, ctx->L.halves);
+  NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
+  int threads = 0, per_sm = 0;
+  for (int cand : {256, 128}) {
+    const size_t smem = fixed + (size_t)48 * M * cand;
+    if (smem > (size_t)227 * 1024) continue;
+    NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int n = 0;
+    NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k, cand, smem));
+    const bool better = (n >= 2) != (per_sm >= 2) ? n >= 2 : n * cand > per_sm * threads;
+    if (n >= 1 && (threads == 0 || better)) { threads = cand; per_sm = n; }
+  }
+  if (threads == 0 || per_sm * threads < 256) return NETMAX_OK;  // too few warps to hide the arithmetic latency
   f.threads = threads;
-  f.smem = head + (size_t)48 * M * threads + 64 * sizeof(double);
+  f.smem = fixed + (size_t)48 * M * threads;
   f.max_rounds = ctx->fuse_rounds >= 2 ? std::min(ctx->fuse_rounds, kFusedMaxRounds) : kFusedMaxRounds;
-  f.n_tiles = (ctx->L.nq + threads - 1) / threads;
-  FusedKernel k = pick_fused_kernel(ctx->objective);
+  f.n_tiles = ((ctx->d + 3) / 4 + threads - 1) / threads;
   NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)f.smem));
-  int per_sm = 0;
-  NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, threads, f.smem));
-  if (per_sm < 1) return NETMAX_OK;
   f.grid = (int)std::min<int64_t>(f.n_tiles, std::min<int64_t>((int64_t)per_sm * ctx->sm_count, kMaxGrid));
   f.ok = true;
   return NETMAX_OK;
+}
+
+// Several rounds per launch over shared-memory-resident tiles (fused_rounds_kernel): long
+// vectors, fp32 state, and few enough workers that the slabs (48 bytes per worker and thread)
+// of at least eight warps fit on an SM.  The plan is kept until fuse_rounds changes.
+int plan_fused(netmax_ctx* ctx, const RoundPlan& plan, FusedPlan& f) {
+  if (ctx->fused_planned) {
+    f = ctx->fused;
+    return NETMAX_OK;
+  }
+  int rc = plan_fused_uncached(ctx, plan, f);
+  if (rc == NETMAX_OK) {
+    ctx->fused = f;
+    ctx->fused_planned = true;
+  }
+  return rc;
 }
 
 }  // namespace
@@ -889,18 +916,20 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
         fp.ring = ctx->trace_rounds;
         fp.first_round = (uint64_t)ctx->rounds;
         fp.n_rounds = chunk;
-        fp.ldq = p.ldq;
-        fp.nq = p.nq;
+        fp.nq = (ctx->d + 3) / 4;
         fp.n_tiles = fused.n_tiles;
         fp.row_bytes = p.row_bytes;
         fp.M = p.M;
-        fp.tail = p.tail;
+        fp.tail = (int32_t)(ctx->d % 4);
         fp.alpha = p.alpha;
         fp.sigma = p.sigma;
         fp.inv_M = p.inv_M;
         fp.q_offset = p.q_offset;
         fp.keys = p.keys;
-        pick_fused_kernel(ctx->objective)<<<fused.grid, fused.threads, fused.smem, ctx->stream>>>(fp);
+        // (the attribute belongs to the kernel, not to this context: another context may have lowered it)
+        FusedKernel fk = pick_fused_kernel(ctx->objective, ctx->L.halves);
+        NM_CUDA(ctx, cudaFuncSetAttribute(fk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fused.smem));
+        fk<<<fused.grid, fused.threads, fused.smem, ctx->stream>>>(fp);
         ctx->launches += 1;
         ctx->cur ^= 1;
         ctx->rounds += chunk;
@@ -934,6 +963,7 @@ int netmax_set_fuse_rounds(netmax_ctx* ctx, int32_t fuse_rounds) {
   if (fuse_rounds < 0 || fuse_rounds > kFusedMaxRounds)
     return fail(ctx, NETMAX_INVALID_ARG, "fuse_rounds = %d outside [0, %d]", fuse_rounds, kFusedMaxRounds);
   ctx->fuse_rounds = fuse_rounds;
+  ctx->fused_planned = false;
   return NETMAX_OK;
 }
 

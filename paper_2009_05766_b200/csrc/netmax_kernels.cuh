@@ -564,7 +564,10 @@ __global__ void __launch_bounds__(256, 2) multi_round_kernel(const MultiRoundPar
 // the peer's value of the same column group was written by this very thread a round earlier,
 // so the rounds need no barrier.  Per-element arithmetic is row_update's, hence the replicas
 // are bit-identical to one launch per round; telemetry sums only differ in the order of their
-// double-precision accumulation.  fp32 state only.
+// double-precision accumulation.  The slabs always hold fp32; with bfloat16 state (kBf16) a
+// thread's column group is four bfloat16 values (8 bytes of global memory), widened on the way
+// in, and every round's result is rounded to bfloat16 before it is written to the slab, exactly
+// as a store to and a load from the bfloat16 state would.
 #ifndef NETMAX_FUSED_MAX_ROUNDS
 #define NETMAX_FUSED_MAX_ROUNDS 4
 #endif
@@ -586,31 +589,34 @@ struct FusedParams {
   int64_t slot0, ring;   // ring slot of the first round
   uint64_t first_round;
   int32_t n_rounds;      // 1 .. kFusedMaxRounds
-  int64_t ldq, nq, n_tiles;
+  int64_t nq, n_tiles;   // column groups of FOUR elements per row (whatever the storage), tiles of blockDim of them
   uint32_t row_bytes;
-  int32_t M, tail;
+  int32_t M, tail;       // tail = d % 4
   float alpha, sigma, inv_M;
   uint32_t q_offset;
   PhiloxKeys keys;
 };
 
-// Dynamic shared memory: (peer, weight) int2[kFusedMaxRounds][M], then the slabs
+// Dynamic shared memory: (peer row offset, weight) int2[kFusedMaxRounds][M], then the slabs
 // float4[3][M][blockDim] (replicas of even rounds, of odd rounds, centres), then 64 doubles.
-template <int kObjective, bool kFastNoise>
+// Any block size that is a multiple of 32 up to 256 works.
+template <int kObjective, bool kFastNoise, bool kBf16>
 __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams p) {
+  constexpr uint32_t kGroupBytes = kBf16 ? 8u : 16u;  // four elements in global memory
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int tid = threadIdx.x, T = blockDim.x, M = p.M;
-  int2* s_pw = reinterpret_cast<int2*>(smem_raw);
-  const size_t head = (((size_t)kFusedMaxRounds * M * 8) + 127) & ~(size_t)127;
-  ulonglong2* s_x = reinterpret_cast<ulonglong2*>(smem_raw + head);  // [2][M][T]
-  ulonglong2* s_c = s_x + (size_t)2 * M * T;                        // [M][T]
-  double* s_red = reinterpret_cast<double*>(s_c + (size_t)M * T);
+  int2* s_pw = reinterpret_cast<int2*>(smem_raw);  // (byte offset of the peer's row in a slab, weight bits)
+  const uint32_t head = ((uint32_t)(kFusedMaxRounds * M * 8) + 127u) & ~127u;
+  const uint32_t stride = (uint32_t)T * 16u;     // bytes between consecutive rows of a slab
+  const uint32_t plane = (uint32_t)M * stride;   // bytes of one [M][T] slab
+  unsigned char* slab = smem_raw + head + (uint32_t)tid * 16u;  // this thread's column: slabs 0, 1 (replicas), 2 (centres)
+  double* s_red = reinterpret_cast<double*>(smem_raw + head + 3u * plane);
 
   for (int k = 0; k < p.n_rounds; ++k) {
     const int32_t* peers = p.trace + ((p.slot0 + k) % p.ring) * M;
     for (int i = tid; i < M; i += T) {
       const int32_t m = __ldg(peers + i);
-      s_pw[k * M + i] = make_int2(m, __float_as_int((m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * M + m)));
+      s_pw[k * M + i] = make_int2((int)((uint32_t)m * stride), __float_as_int((m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * M + m)));
     }
   }
   __syncthreads();
@@ -624,14 +630,24 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
     if (q >= p.nq) continue;  // no barrier below: threads are independent
     const int live_lo = live_lanes((p.tail != 0) && (q == p.nq - 1), p.tail, 0);
     const uint32_t q32 = (uint32_t)q + p.q_offset;
-    {  // all rows of this column group into the thread's slab
-      const char* xq = reinterpret_cast<const char*>(p.x_cur + q);
-      const char* cq = reinterpret_cast<const char*>(p.c + q);
+    {  // all rows of this column group into the thread's slabs
+      const char* xq = reinterpret_cast<const char*>(p.x_cur) + (uint64_t)q * kGroupBytes;
+      const char* cq = reinterpret_cast<const char*>(p.c) + (uint64_t)q * kGroupBytes;
+      unsigned char* sx = slab;
+      unsigned char* sc = slab + 2u * plane;
 #pragma unroll 4
       for (int i = 0; i < M; ++i) {
-        const uint64_t row = (uint64_t)(uint32_t)i * p.row_bytes;
-        s_x[(size_t)i * T + tid] = __ldg(reinterpret_cast<const ulonglong2*>(xq + row));
-        s_c[(size_t)i * T + tid] = __ldg(reinterpret_cast<const ulonglong2*>(cq + row));
+        if (kBf16) {
+          *reinterpret_cast<ulonglong2*>(sx) = widen_bf16x4(__ldg(reinterpret_cast<const unsigned long long*>(xq)));
+          *reinterpret_cast<ulonglong2*>(sc) = widen_bf16x4(__ldg(reinterpret_cast<const unsigned long long*>(cq)));
+        } else {
+          *reinterpret_cast<ulonglong2*>(sx) = __ldg(reinterpret_cast<const ulonglong2*>(xq));
+          *reinterpret_cast<ulonglong2*>(sc) = __ldg(reinterpret_cast<const ulonglong2*>(cq));
+        }
+        xq += p.row_bytes;
+        cq += p.row_bytes;
+        sx += stride;
+        sc += stride;
       }
     }
 #pragma unroll
@@ -639,19 +655,23 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
       if (k < p.n_rounds) {
         const uint64_t round = p.first_round + (uint64_t)k;
         const uint32_t round_lo = (uint32_t)round, ctr3 = philox_ctr3(kTagNoise, round);
-        const ulonglong2* cur = s_x + (size_t)(k & 1) * M * T;
-        ulonglong2* nxt = s_x + (size_t)((k & 1) ^ 1) * M * T;
+        const unsigned char* cur = slab + (uint32_t)(k & 1) * plane;
+        unsigned char* nxt = slab + (uint32_t)((k & 1) ^ 1) * plane;
+        const unsigned char* cen = slab + 2u * plane;
         const int2* pw = s_pw + k * M;
-        const ulonglong2 pivot = cur[tid];
+        const ulonglong2 pivot = *reinterpret_cast<const ulonglong2*>(cur);
         ColAcc acc;
         LossAcc lacc;
+        uint32_t off = 0;
 #pragma unroll kFusedUnroll
         for (int i = 0; i < M; ++i) {
           const int2 d = pw[i];
           const ulonglong2 o = row_update<kObjective, kFastNoise>(
-              p.alpha, p.sigma, p.keys, round_lo, ctr3, q32, (uint32_t)i, cur[(size_t)i * T + tid], s_c[(size_t)i * T + tid],
-              cur[(size_t)d.x * T + tid], pivot, __int_as_float(d.y), live_lo, acc, lacc);
-          nxt[(size_t)i * T + tid] = o;
+              p.alpha, p.sigma, p.keys, round_lo, ctr3, q32, (uint32_t)i, *reinterpret_cast<const ulonglong2*>(cur + off),
+              *reinterpret_cast<const ulonglong2*>(cen + off), *reinterpret_cast<const ulonglong2*>(cur + (uint32_t)d.x), pivot,
+              __int_as_float(d.y), live_lo, acc, lacc);
+          *reinterpret_cast<ulonglong2*>(nxt + off) = kBf16 ? widen_bf16x4(narrow_bf16x4(o)) : o;
+          off += stride;
         }
         float4 s1, s2;
         unpack2(acc.s1a, s1.x, s1.y);
@@ -668,11 +688,15 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
       }
     }
     {
-      const ulonglong2* fin = s_x + (size_t)(p.n_rounds & 1) * M * T;
-      char* oq = reinterpret_cast<char*>(p.x_nxt + q);
+      const unsigned char* fin = slab + (uint32_t)(p.n_rounds & 1) * plane;
+      char* oq = reinterpret_cast<char*>(p.x_nxt) + (uint64_t)q * kGroupBytes;
 #pragma unroll 4
-      for (int i = 0; i < M; ++i)
-        *reinterpret_cast<ulonglong2*>(oq + (uint64_t)(uint32_t)i * p.row_bytes) = fin[(size_t)i * T + tid];
+      for (int i = 0; i < M; ++i) {
+        if (kBf16) *reinterpret_cast<unsigned long long*>(oq) = narrow_bf16x4(*reinterpret_cast<const ulonglong2*>(fin));
+        else *reinterpret_cast<ulonglong2*>(oq) = *reinterpret_cast<const ulonglong2*>(fin);
+        oq += p.row_bytes;
+        fin += stride;
+      }
     }
   }
 

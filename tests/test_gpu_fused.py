@@ -36,13 +36,16 @@ def random_policy(M, rng, zeros=0.0):
 
 
 # long vectors: at least two 4 KB-wide tiles per SM, so that the streaming launch shapes are chosen
-@pytest.mark.parametrize("M,d,fuse", [(2, 400_003, 0), (5, 320_001, 0), (8, 400_002, 0), (9, 310_000, 3), (8, 400_001, 2),
-                                      (16, 320_001, 4), (18, 310_003, 4)])
+@pytest.mark.parametrize("M,d,fuse,storage", [(2, 400_003, 0, "f32"), (5, 320_001, 0, "f32"), (8, 400_002, 0, "f32"),
+                                              (9, 310_000, 3, "f32"), (8, 400_001, 2, "f32"), (16, 320_001, 4, "f32"),
+                                              (18, 310_003, 4, "f32"), (8, 700_003, 0, "bf16"), (3, 650_001, 4, "bf16"),
+                                              (16, 620_006, 3, "bf16")])
 @pytest.mark.parametrize("objective", [0, 1])
-def test_fused_rounds_change_no_bit(nm, M, d, fuse, objective):
+def test_fused_rounds_change_no_bit(nm, M, d, fuse, storage, objective):
     rng = np.random.default_rng(M * 11 + d)
     P = random_policy(M, rng, zeros=0.2 if M > 4 else 0.0)
-    kw = dict(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=objective, seed=d + M, trace_rounds=64)
+    kw = dict(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=objective, seed=d + M, trace_rounds=64,
+              storage=storage)
     one = nm.Netmax(fuse_rounds=1, **kw)         # one launch per round
     many = nm.Netmax(fuse_rounds=fuse, **kw)
     rounds = 0
@@ -57,8 +60,10 @@ def test_fused_rounds_change_no_bit(nm, M, d, fuse, objective):
     assert (xa.view(np.uint32) == xb.view(np.uint32)).all()
     assert (one.peer_trace(0, rounds) == many.peer_trace(0, rounds)).all()
     (ca, la), (cb, lb) = one.telemetry(0, rounds), many.telemetry(0, rounds)
-    np.testing.assert_allclose(cb, ca, rtol=1e-12)
-    np.testing.assert_allclose(lb, la, rtol=1e-12)
+    # (with bfloat16 state the two launch shapes group a thread's fp32 partial sums by 8 and by 4 columns)
+    rtol = 1e-12 if storage == "f32" else 1e-6
+    np.testing.assert_allclose(cb, ca, rtol=rtol)
+    np.testing.assert_allclose(lb, la, rtol=rtol)
     # padding lanes of the rows stay zero
     import torch
     ptr, ld = many.replicas_device()
@@ -67,8 +72,9 @@ def test_fused_rounds_change_no_bit(nm, M, d, fuse, objective):
         pass
 
     h = _Holder()
-    h.__cuda_array_interface__ = {"shape": (M, ld), "typestr": "<f4", "data": (ptr, False), "version": 3, "strides": None}
-    assert float(torch.as_tensor(h, device="cuda")[:, d:].abs().max().item()) == 0.0
+    h.__cuda_array_interface__ = {"shape": (M, ld), "typestr": "<f4" if storage == "f32" else "<i2", "data": (ptr, False),
+                                  "version": 3, "strides": None}
+    assert int(torch.as_tensor(h, device="cuda")[:, d:].abs().max().item()) == 0
     one.close()
     many.close()
 
