@@ -45,6 +45,13 @@ struct DeviceGuard {
   }
 };
 
+struct ResidentPlan {  // launch shape of resident_rounds_kernel
+  bool ok = false;
+  int threads = 0, grid = 0, G = 0, log2G = 0, draws_in_smem = 0;
+  size_t smem = 0;
+  int64_t n_tiles = 0, max_rounds = 0;
+};
+
 struct FusedPlan {  // launch shape of fused_rounds_kernel
   bool ok = false;
   int threads = 0, grid = 0, max_rounds = 0;
@@ -56,7 +63,7 @@ struct Layout {
   int64_t ld = 0, ldq = 0, nq = 0;  // row stride in elements / in 16-byte column groups; column groups in use
   int elem = 4, halves = 1;         // bytes per stored element; Philox blocks (4 elements) per column group
   size_t plane = 0;                 // bytes of one [M][ld] array
-  size_t off_x0 = 0, off_x1 = 0, off_c = 0, off_thr = 0, off_last = 0, off_w = 0, off_trace = 0, off_tel = 0,
+  size_t off_x0 = 0, off_x1 = 0, off_c = 0, off_thr = 0, off_last = 0, off_w = 0, off_trace = 0, off_wring = 0, off_tel = 0,
          off_partials = 0, off_ticket = 0, off_colpart = 0, off_coltick = 0, total = 0;
 };
 
@@ -83,6 +90,7 @@ Layout make_layout(int64_t M, int64_t d, int64_t trace_rounds, int storage) {
   L.off_last = take((size_t)M * sizeof(int32_t));
   L.off_w = take((size_t)M * M * sizeof(float));
   L.off_trace = take((size_t)trace_rounds * M * sizeof(int32_t));
+  L.off_wring = take((size_t)trace_rounds * M * sizeof(float));  // pull weight of every draw in the trace ring
   L.off_tel = take((size_t)trace_rounds * 2 * sizeof(double));
   L.off_partials = take((size_t)kMaxGrid * 2 * sizeof(double) * 2);  // two sets: multi-round launches alternate
   L.off_ticket = take(256);
@@ -113,6 +121,7 @@ struct netmax_ctx {
   int32_t* last_nz = nullptr;
   float* wtab = nullptr;
   int32_t* trace = nullptr;
+  float* wring = nullptr;
   double* tel = nullptr;
   double* partials = nullptr;
   unsigned int* ticket = nullptr;
@@ -158,6 +167,8 @@ struct netmax_ctx {
   int fuse_rounds = 0;  // 0: automatic, 1: one launch per round, 2..kFusedMaxRounds: rounds per fused launch
   bool fused_planned = false;
   FusedPlan fused;
+  bool resident_planned = false;
+  ResidentPlan resident;
   PhiloxKeys keys;
   std::vector<double> P;      // policy in force
   std::vector<uint8_t> adj;   // link graph in force
@@ -352,12 +363,15 @@ int launch_init(netmax_ctx* ctx, unsigned char* dst, double stddev, uint32_t tag
   return NETMAX_OK;
 }
 
-int launch_sampler(netmax_ctx* ctx, uint64_t first_round, int64_t n_rounds, int32_t* out, int64_t slot0, int64_t ring) {
+int launch_sampler(netmax_ctx* ctx, uint64_t first_round, int64_t n_rounds, int32_t* out, float* w_out, int64_t slot0,
+                   int64_t ring) {
   if (n_rounds <= 0) return NETMAX_OK;
   SampleParams p;
   p.thresholds = ctx->thr;
   p.last_nz = ctx->last_nz;
   p.out = out;
+  p.w_out = w_out;
+  p.wtab = ctx->wtab;
   p.slot0 = slot0;
   p.ring = ring;
   p.first_round = first_round;
@@ -418,6 +432,13 @@ using FusedKernel = void (*)(const FusedParams);
 FusedKernel pick_fused_kernel(int objective, int halves) {
   if (halves == 2) return objective == 1 ? fused_rounds_kernel<1, true, true> : fused_rounds_kernel<0, true, true>;
   return objective == 1 ? fused_rounds_kernel<1, true, false> : fused_rounds_kernel<0, true, false>;
+}
+
+using ResidentKernel = void (*)(const ResidentParams);
+
+ResidentKernel pick_resident_kernel(int objective, int halves) {
+  if (halves == 2) return objective == 1 ? resident_rounds_kernel<1, true, true> : resident_rounds_kernel<0, true, true>;
+  return objective == 1 ? resident_rounds_kernel<1, true, false> : resident_rounds_kernel<0, true, false>;
 }
 
 int floor_pow2(int64_t v) {
@@ -481,6 +502,67 @@ int plan_round(netmax_ctx* ctx, RoundPlan& plan, int objective) {
   }
   plan.grid = (int)std::min<int64_t>(plan.n_tiles, std::min<int64_t>((int64_t)per_sm * ctx->sm_count, kMaxGrid));
   return NETMAX_OK;
+}
+
+size_t resident_smem(int64_t M, int threads, int G, bool draws) {
+  return (size_t)48 * M * G + 2 * sizeof(float) * resident_scratch_floats(threads, G) + 128 * sizeof(double) +
+         (draws ? (size_t)16 * M : 0);
+}
+
+// Short vectors whose M rows of at least one column group fit in a CTA's shared memory run all
+// rounds of a call on resident columns (resident_rounds_kernel).  Small M: a thread per column
+// group, as few threads per CTA as keep the CTA count within a few per SM (the problem is
+// latency-bound: spread it over the SMs).  Larger M: G column groups per CTA, the rows of each
+// split over the threads; G as large as fits, but no larger than leaves every SM a tile.
+int plan_resident_uncached(netmax_ctx* ctx, const RoundPlan& plan, ResidentPlan& f) {
+  f = ResidentPlan();
+  if (!plan.short_vectors) return NETMAX_OK;
+  const int64_t M = ctx->M, nq = (ctx->d + 3) / 4;
+  const size_t limit = (size_t)224 * 1024;
+  int threads = 0, G = 0;
+  for (int cand : {32, 64, 128, 256}) {  // a thread per column group
+    if (resident_smem(M, cand, cand, M <= cand) > (size_t)100 * 1024) break;
+    threads = G = cand;
+    if ((nq + cand - 1) / cand <= (int64_t)8 * ctx->sm_count) break;
+  }
+  if (threads == 0) {  // rows of a group split over the threads
+    G = 32;
+    while (G > 1 && (size_t)48 * M * G > (size_t)190 * 1024) G >>= 1;
+    while (G > 1 && (nq + G - 1) / G < ctx->sm_count) G >>= 1;
+    threads = (int)std::min<int64_t>(512, std::max<int64_t>(64, floor_pow2(M * G / 2)));
+    threads = std::max(threads, G);
+    if (resident_smem(M, threads, G, M <= threads) > limit) return NETMAX_OK;
+  }
+  f.threads = threads;
+  f.G = G;
+  f.log2G = 0;
+  while ((1 << f.log2G) < G) ++f.log2G;
+  f.draws_in_smem = M <= threads ? 1 : 0;
+  f.smem = resident_smem(M, threads, G, f.draws_in_smem != 0);
+  f.n_tiles = (nq + G - 1) / G;
+  f.max_rounds = std::max<int64_t>(1, std::min<int64_t>(kMaxRoundsPerLaunch, (int64_t)(kColPartBytes / 16) / f.n_tiles));
+  ResidentKernel k = pick_resident_kernel(ctx->objective, ctx->L.halves);
+  NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
+  NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)f.smem));
+  int per_sm = 0;
+  NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, threads, f.smem));
+  if (per_sm < 1) return NETMAX_OK;
+  f.grid = (int)std::min<int64_t>(f.n_tiles, (int64_t)per_sm * ctx->sm_count);
+  f.ok = true;
+  return NETMAX_OK;
+}
+
+int plan_resident(netmax_ctx* ctx, const RoundPlan& plan, ResidentPlan& f) {
+  if (ctx->resident_planned) {
+    f = ctx->resident;
+    return NETMAX_OK;
+  }
+  int rc = plan_resident_uncached(ctx, plan, f);
+  if (rc == NETMAX_OK) {
+    ctx->resident = f;
+    ctx->resident_planned = true;
+  }
+  return rc;
 }
 
 int plan_fused_uncached(netmax_ctx* ctx, const RoundPlan& plan, FusedPlan& f) {
@@ -662,6 +744,7 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   ctx->last_nz = (int32_t*)(ctx->base + L.off_last);
   ctx->wtab = (float*)(ctx->base + L.off_w);
   ctx->trace = (int32_t*)(ctx->base + L.off_trace);
+  ctx->wring = (float*)(ctx->base + L.off_wring);
   ctx->tel = (double*)(ctx->base + L.off_tel);
   ctx->partials = (double*)(ctx->base + L.off_partials);
   ctx->ticket = (unsigned int*)(ctx->base + L.off_ticket);
@@ -835,6 +918,10 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   FusedPlan fused;
   rc = plan_fused(ctx, plan, fused);
   if (rc) return rc;
+  ResidentPlan resident;
+  rc = plan_resident(ctx, plan, resident);
+  if (rc) return rc;
+  if (ctx->fuse_rounds == 1) resident.ok = false;  // one launch per round was asked for
 
   RoundParams p;
   p.c = reinterpret_cast<const float4*>(ctx->c);
@@ -864,8 +951,53 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
     // peers of a batch of rounds in one launch (counter-based draws do not depend on x),
     // at most one lap of the ring at a time
     const int64_t batch = std::min<int64_t>(n_rounds - done, ctx->trace_rounds);
-    rc = launch_sampler(ctx, (uint64_t)ctx->rounds, batch, ctx->trace, ctx->rounds % ctx->trace_rounds, ctx->trace_rounds);
+    rc = launch_sampler(ctx, (uint64_t)ctx->rounds, batch, ctx->trace, ctx->wring, ctx->rounds % ctx->trace_rounds,
+                        ctx->trace_rounds);
     if (rc) return rc;
+    if (resident.ok) {
+      // short vectors: every round of the batch on shared-memory-resident columns
+      ResidentKernel rk = pick_resident_kernel(ctx->objective, ctx->L.halves);
+      int64_t b = 0;
+      while (b < batch) {
+        const int64_t chunk = std::min<int64_t>(batch - b, resident.max_rounds);
+        ResidentParams rp;
+        rp.x_cur = reinterpret_cast<const char*>(ctx->x[ctx->cur]);
+        rp.x_nxt = reinterpret_cast<char*>(ctx->x[ctx->cur ^ 1]);
+        rp.c = reinterpret_cast<const char*>(ctx->c);
+        rp.trace = ctx->trace;
+        rp.wring = ctx->wring;
+        rp.partials = reinterpret_cast<double*>(ctx->colpart);
+        rp.slot0 = ctx->rounds % ctx->trace_rounds;
+        rp.ring = ctx->trace_rounds;
+        rp.first_round = (uint64_t)ctx->rounds;
+        rp.n_rounds = (int32_t)chunk;
+        rp.nq = (ctx->d + 3) / 4;
+        rp.n_tiles = resident.n_tiles;
+        rp.row_bytes = p.row_bytes;
+        rp.M = p.M;
+        rp.tail = (int32_t)(ctx->d % 4);
+        rp.G = resident.G;
+        rp.log2G = resident.log2G;
+        rp.draws_in_smem = resident.draws_in_smem;
+        rp.alpha = p.alpha;
+        rp.sigma = p.sigma;
+        rp.inv_M = p.inv_M;
+        rp.q_offset = p.q_offset;
+        rp.keys = p.keys;
+        NM_CUDA(ctx, cudaFuncSetAttribute(rk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)resident.smem));
+        rk<<<resident.grid, resident.threads, resident.smem, ctx->stream>>>(rp);
+        const int warps_per_block = kThreads / 32;
+        sum_tile_partials_kernel<<<(unsigned)((chunk + warps_per_block - 1) / warps_per_block), kThreads, 0, ctx->stream>>>(
+            rp.partials, rp.n_tiles, rp.n_rounds, (double)p.inv_M, ctx->tel, rp.slot0, rp.ring);
+        ctx->launches += 2;
+        NM_CUDA(ctx, cudaGetLastError());
+        ctx->cur ^= 1;
+        ctx->rounds += chunk;
+        b += chunk;
+      }
+      done += batch;
+      continue;
+    }
     if (plan.short_vectors && ctx->cooperative && batch >= 2) {
       // short, L2-resident problem: all rounds of the batch in cooperative launches
       int64_t b = 0;
@@ -1112,7 +1244,7 @@ int netmax_sample_peers(netmax_ctx* ctx, int64_t first_round, int64_t n_rounds, 
   if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
   if (first_round < 0 || n_rounds < 0 || (n_rounds > 0 && !device_out)) return fail(ctx, NETMAX_INVALID_ARG, "bad range or NULL output");
   DeviceGuard guard(ctx->device);
-  return launch_sampler(ctx, (uint64_t)first_round, n_rounds, device_out, 0, INT64_MAX);
+  return launch_sampler(ctx, (uint64_t)first_round, n_rounds, device_out, nullptr, 0, INT64_MAX);
 }
 
 // ---- telemetry on demand --------------------------------------------------------------------

@@ -26,6 +26,8 @@ struct SampleParams {
   const uint32_t* thresholds;  // [M][M] non-decreasing per row
   const int32_t* last_nz;      // [M] last index with p > 0
   int32_t* out;                // slot s of round r is out + ((slot0 + r) % ring) * M
+  float* w_out;                // same indexing: pull weight of the draw (0 on a self-draw); may be NULL
+  const float* wtab;           // [M][M] pull weights (read when w_out is given)
   int64_t slot0, ring;
   uint64_t first_round;
   int64_t n_rounds;
@@ -49,7 +51,9 @@ __global__ void __launch_bounds__(256) sample_peers_kernel(const SampleParams p)
       if (__ldg(row + mid) <= u) lo = mid + 1; else hi = mid;
     }
     const int32_t m = min(lo, __ldg(p.last_nz + i));
-    p.out[((p.slot0 + r) % p.ring) * p.M + i] = m;
+    const int64_t at = ((p.slot0 + r) % p.ring) * p.M + i;
+    p.out[at] = m;
+    if (p.w_out) p.w_out[at] = (m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * p.M + m);
   }
 }
 
@@ -716,6 +720,222 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
     for (int k = 0; k < p.n_rounds; ++k)
       sum_partials(p.partials + (size_t)k * 2 * gridDim.x, (double)p.inv_M, p.tel + 2 * ((p.slot0 + k) % p.ring), s_red);
     if (tid == 0) *p.ticket = 0u;
+  }
+}
+
+// ---- all rounds of a call over resident columns (short vectors) -------------------------------
+// The same independence of columns serves the opposite shape: when the whole problem is a few
+// megabytes, a round takes microseconds and what costs time is every launch and every grid-wide
+// exchange.  Here a CTA keeps ALL M rows of G column groups (four elements each) in shared
+// memory, fp32, double-buffered by round, together with their centres, and runs every round of
+// the call on them; CTAs never talk to each other.  Two thread mappings:
+//   G == blockDim  a thread owns a column group and walks all M rows (small M): no barrier is
+//                  needed for the data, only the per-round telemetry reduction synchronises;
+//   G <= 32        thread (g, r) owns the rows r, r + blockDim / G, ... of group g (large M):
+//                  a peer's row belongs to another thread, so rounds are separated by a barrier.
+// Per round every CTA writes its two telemetry sums to partials[round][tile]; a second small
+// kernel adds the tiles of each round in index order.  Arithmetic per element is row_update's,
+// so replicas are bit-identical to the other launch shapes.
+struct ResidentParams {
+  const char* x_cur;      // replicas at the start of the first round, row stride row_bytes
+  char* x_nxt;            // replicas after the last round
+  const char* c;
+  const int32_t* trace;   // peer-trace ring [ring][M]
+  const float* wring;     // pull weight of every draw, same ring
+  double* partials;       // [n_rounds][n_tiles][2]
+  int64_t slot0, ring;
+  uint64_t first_round;
+  int32_t n_rounds;
+  int64_t nq, n_tiles;    // column groups of four elements per row; tiles of G of them
+  uint32_t row_bytes;
+  int32_t M, tail;        // tail = d % 4
+  int32_t G, log2G;       // column groups per tile (a power of two)
+  int32_t draws_in_smem;  // 1: the round's (peer, weight) pairs are staged in shared memory, one round ahead
+  float alpha, sigma, inv_M;
+  uint32_t q_offset;
+  PhiloxKeys keys;
+};
+
+// Dynamic shared memory: slabs float4[3][M][G]; then (G < blockDim) two reduction scratch
+// buffers float[warps][G][9] (padded to 16 bytes); then 2 x 64 doubles; then (draws_in_smem,
+// which needs M <= blockDim) int2[2][M].
+#ifndef NETMAX_RESIDENT_UNROLL
+#define NETMAX_RESIDENT_UNROLL 2
+#endif
+constexpr int kResidentUnroll = NETMAX_RESIDENT_UNROLL;  // rows of a round in flight per thread
+__host__ __device__ inline uint32_t resident_scratch_floats(int threads, int G) {
+  return G < threads ? (uint32_t)(((threads >> 5) * G * 9 + 3) & ~3) : 0u;
+}
+template <int kObjective, bool kFastNoise, bool kBf16>
+__global__ void __launch_bounds__(512) resident_rounds_kernel(const ResidentParams p) {
+  constexpr uint32_t kGroupBytes = kBf16 ? 8u : 16u;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int tid = threadIdx.x, T = blockDim.x, M = p.M, G = p.G;
+  const int g = tid & (G - 1), r = tid >> p.log2G, RL = T >> p.log2G;
+  const int lane = tid & 31, warp = tid >> 5, nwarps = T >> 5;
+  const uint32_t stride = (uint32_t)G * 16u;    // bytes between consecutive rows of a slab
+  const uint32_t plane = (uint32_t)M * stride;
+  unsigned char* slab = smem_raw + (uint32_t)g * 16u;
+  float* s_scratch = reinterpret_cast<float*>(smem_raw + 3u * plane);
+  const uint32_t scratch_floats = resident_scratch_floats(T, G);
+  double* s_red = reinterpret_cast<double*>(s_scratch + 2 * scratch_floats);
+  int2* s_pw = reinterpret_cast<int2*>(s_red + 128);
+
+  for (int64_t tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x) {
+    const int64_t q = tile * G + g;
+    const bool live = q < p.nq;
+    const int live_lo = live_lanes((p.tail != 0) && (q == p.nq - 1), p.tail, 0);
+    const uint32_t q32 = (uint32_t)q + p.q_offset;
+    __syncthreads();  // the previous tile is stored
+    for (int i = r; i < M; i += RL) {
+      ulonglong2 xv = make_ulonglong2(0ull, 0ull), cv = xv;
+      if (live) {
+        const char* xq = p.x_cur + (uint64_t)(uint32_t)i * p.row_bytes + (uint64_t)q * kGroupBytes;
+        const char* cq = p.c + (uint64_t)(uint32_t)i * p.row_bytes + (uint64_t)q * kGroupBytes;
+        if (kBf16) {
+          xv = widen_bf16x4(__ldg(reinterpret_cast<const unsigned long long*>(xq)));
+          cv = widen_bf16x4(__ldg(reinterpret_cast<const unsigned long long*>(cq)));
+        } else {
+          xv = __ldg(reinterpret_cast<const ulonglong2*>(xq));
+          cv = __ldg(reinterpret_cast<const ulonglong2*>(cq));
+        }
+      }
+      *reinterpret_cast<ulonglong2*>(slab + (uint32_t)i * stride) = xv;
+      *reinterpret_cast<ulonglong2*>(slab + 2u * plane + (uint32_t)i * stride) = cv;
+    }
+    if (p.draws_in_smem) {  // the first round's draws
+      const int64_t at = (p.slot0 % p.ring) * M;
+      for (int i = tid; i < M; i += T) s_pw[i] = make_int2(__ldg(p.trace + at + i), __float_as_int(__ldg(p.wring + at + i)));
+    }
+    __syncthreads();
+
+    for (int k = 0; k < p.n_rounds; ++k) {
+      const uint64_t round = p.first_round + (uint64_t)k;
+      const uint32_t round_lo = (uint32_t)round, ctr3 = philox_ctr3(kTagNoise, round);
+      const int64_t at = ((p.slot0 + k) % p.ring) * M;
+      const unsigned char* cur = slab + (uint32_t)(k & 1) * plane;
+      unsigned char* nxt = slab + (uint32_t)((k & 1) ^ 1) * plane;
+      const unsigned char* cen = slab + 2u * plane;
+      const int2* pw = s_pw + (k & 1) * M;
+      // next round's draws: issue the loads now, park them in shared memory after the arithmetic
+      int2 ahead = make_int2(0, 0);
+      const bool fetch = p.draws_in_smem && k + 1 < p.n_rounds && tid < M;
+      if (fetch) {
+        const int64_t at1 = ((p.slot0 + k + 1) % p.ring) * M;
+        ahead = make_int2(__ldg(p.trace + at1 + tid), __float_as_int(__ldg(p.wring + at1 + tid)));
+      }
+      ColAcc acc;
+      LossAcc lacc;
+      if (live) {
+        const ulonglong2 pivot = *reinterpret_cast<const ulonglong2*>(cur);
+#pragma unroll kResidentUnroll
+        for (int i = r; i < M; i += RL) {
+          int2 d;
+          if (p.draws_in_smem) d = pw[i];
+          else d = make_int2(__ldg(p.trace + at + i), __float_as_int(__ldg(p.wring + at + i)));
+          const uint32_t off = (uint32_t)i * stride;
+          ulonglong2 o = row_update<kObjective, kFastNoise>(
+              p.alpha, p.sigma, p.keys, round_lo, ctr3, q32, (uint32_t)i, *reinterpret_cast<const ulonglong2*>(cur + off),
+              *reinterpret_cast<const ulonglong2*>(cen + off), *reinterpret_cast<const ulonglong2*>(cur + (uint32_t)d.x * stride),
+              pivot, __int_as_float(d.y), live_lo, acc, lacc);
+          if (kBf16) o = widen_bf16x4(narrow_bf16x4(o));
+          *reinterpret_cast<ulonglong2*>(nxt + off) = o;
+        }
+      }
+      if (fetch) s_pw[((k & 1) ^ 1) * M + tid] = ahead;  // (M <= blockDim in this mode: one entry per thread)
+      // ---- telemetry of the round: column sums over the row lanes, then over the tile
+      float v[9];
+      unpack2(acc.s1a, v[0], v[1]);
+      unpack2(acc.s1b, v[2], v[3]);
+      unpack2(acc.s2a, v[4], v[5]);
+      unpack2(acc.s2b, v[6], v[7]);
+      {
+        float l0, l1, l2, l3;
+        unpack2(lacc.la, l0, l1);
+        unpack2(lacc.lb, l2, l3);
+        v[8] = (l0 + l1) + (l2 + l3);
+      }
+      float* scratch = s_scratch + (k & 1) * scratch_floats;
+      double* red = s_red + (k & 1) * 64;
+      bool owner = true;  // does this thread hold the complete sums of its column group?
+      if (RL > 1) {
+        for (int off = 16; off >= G; off >>= 1) {
+#pragma unroll
+          for (int a = 0; a < 9; ++a) v[a] += __shfl_xor_sync(0xffffffffu, v[a], off);
+        }
+        if (lane < G) {
+#pragma unroll
+          for (int a = 0; a < 9; ++a) scratch[(warp * G + lane) * 9 + a] = v[a];
+        }
+        __syncthreads();
+        owner = tid < G;
+        if (owner) {
+#pragma unroll
+          for (int a = 0; a < 9; ++a) v[a] = 0.f;
+          for (int w = 0; w < nwarps; ++w) {  // (G <= 32: every warp holds rows of every group)
+#pragma unroll
+            for (int a = 0; a < 9; ++a) v[a] += scratch[(w * G + tid) * 9 + a];
+          }
+        }
+      }
+      double cons = 0.0, loss = 0.0;
+      if (owner) {
+        cons = (double)((v[4] - v[0] * v[0] * p.inv_M) + (v[5] - v[1] * v[1] * p.inv_M) + (v[6] - v[2] * v[2] * p.inv_M) +
+                        (v[7] - v[3] * v[3] * p.inv_M));
+        loss = 0.5 * (double)v[8];
+      }
+      for (int off = 16; off > 0; off >>= 1) {
+        cons += __shfl_down_sync(0xffffffffu, cons, off);
+        loss += __shfl_down_sync(0xffffffffu, loss, off);
+      }
+      if (lane == 0) {
+        red[warp] = cons;
+        red[32 + warp] = loss;
+      }
+      __syncthreads();  // also: every row of the round is written before the next round reads it
+      if (tid == 0) {
+        double a = 0.0, b = 0.0;
+        for (int w = 0; w < nwarps; ++w) {
+          a += red[w];
+          b += red[32 + w];
+        }
+        double* out = p.partials + ((size_t)k * p.n_tiles + tile) * 2;
+        out[0] = a;
+        out[1] = b;
+      }
+    }
+
+    if (live) {
+      const unsigned char* fin = slab + (uint32_t)(p.n_rounds & 1) * plane;
+      for (int i = r; i < M; i += RL) {
+        char* oq = p.x_nxt + (uint64_t)(uint32_t)i * p.row_bytes + (uint64_t)q * kGroupBytes;
+        const ulonglong2 o = *reinterpret_cast<const ulonglong2*>(fin + (uint32_t)i * stride);
+        if (kBf16) *reinterpret_cast<unsigned long long*>(oq) = narrow_bf16x4(o);
+        else *reinterpret_cast<ulonglong2*>(oq) = o;
+      }
+    }
+  }
+}
+
+// tel[slot of round k] = (sum over tiles of partials[k][tile]) / M, one warp per round, tiles in a fixed order.
+__global__ void __launch_bounds__(256) sum_tile_partials_kernel(const double* partials, int64_t n_tiles, int32_t n_rounds,
+                                                                double inv_M, double* tel, int64_t slot0, int64_t ring) {
+  const int lane = threadIdx.x & 31;
+  const int k = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+  if (k >= n_rounds) return;
+  double a = 0.0, b = 0.0;
+  for (int64_t t = lane; t < n_tiles; t += 32) {
+    a += partials[((size_t)k * n_tiles + t) * 2];
+    b += partials[((size_t)k * n_tiles + t) * 2 + 1];
+  }
+  for (int off = 16; off > 0; off >>= 1) {
+    a += __shfl_down_sync(0xffffffffu, a, off);
+    b += __shfl_down_sync(0xffffffffu, b, off);
+  }
+  if (lane == 0) {
+    double* out = tel + 2 * ((slot0 + k) % ring);
+    out[0] = a * inv_M;
+    out[1] = b * inv_M;
   }
 }
 

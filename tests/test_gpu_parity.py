@@ -388,7 +388,9 @@ def test_a_barrier_wait_that_runs_out_is_reported_and_the_context_survives(nm):
     rng = np.random.default_rng(33)
     P = random_policy(M, rng)
     x0 = rng.standard_normal((M, d)).astype(np.float32)
-    kw = dict(M=M, d=d, lr=0.05, prob=P, sigma=0.1, c_std=1.0, seed=3)
+    # fuse_rounds = 1 keeps nothing resident on chip across rounds, which is what sends a short-vector
+    # batch through the cooperative launch whose grid barrier is under test
+    kw = dict(M=M, d=d, lr=0.05, prob=P, sigma=0.1, c_std=1.0, seed=3, fuse_rounds=1)
     g, ref = nm.Netmax(**kw), nm.Netmax(**kw)
     g.set_replicas(x0)
     g.debug_absent_ctas(1)

@@ -1,0 +1,107 @@
+"""GPU parity of the launch shape for short vectors that keeps whole columns (all M rows of a few
+column groups) resident in shared memory for every round of a call.  Replicas and peer traces
+must equal, bit for bit, those of the launch shapes that keep nothing on chip across rounds
+(fuse_rounds = 1), and match the CPU oracle within the fp32 tolerance; telemetry sums are
+accumulated in a different order and agree to fp32 rounding."""
+import numpy as np
+import pytest
+
+from oracle import oracle
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def nm():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    from paper_2009_05766_b200 import binding
+    binding.lib()
+    return binding
+
+
+def full_adj(M):
+    return (1 - np.eye(M)).astype(np.uint8)
+
+
+def random_policy(M, rng, zeros=0.0):
+    P = rng.random((M, M)) + 0.05
+    if zeros > 0:
+        mask = rng.random((M, M)) < zeros
+        mask[np.arange(M), (np.arange(M) + 1) % M] = False
+        P[mask] = 0.0
+    return P / P.sum(axis=1, keepdims=True)
+
+
+# a thread per column group (small M), rows split over threads (larger M), ragged tails, one column,
+# more tiles than resident CTAs, the largest M that still fits (a 4-element column of 4700 rows)
+SHAPES = [(2, 1), (3, 9), (4, 4096), (7, 4099), (5, 67), (2, 280_001), (66, 515), (67, 515), (130, 37), (300, 1030),
+          (512, 1024), (1000, 131), (4096, 64), (4700, 7)]
+
+
+@pytest.mark.parametrize("storage", ["f32", "bf16"])
+@pytest.mark.parametrize("M,d", SHAPES)
+def test_resident_columns_change_no_bit(nm, M, d, storage):
+    rng = np.random.default_rng(M * 5 + d)
+    P = random_policy(M, rng, zeros=0.3 if M > 4 else 0.0)
+    kw = dict(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=1, seed=d + M, trace_rounds=16,
+              storage=storage)
+    plain = nm.Netmax(fuse_rounds=1, **kw)
+    res = nm.Netmax(**kw)
+    rounds = 0
+    for n in (1, 7, 16, 2, 11):              # single rounds, batches, a full lap of the ring and a wrap
+        launches = res.kernel_launches
+        plain.round(n)
+        res.round(n)
+        rounds += n
+        assert res.kernel_launches - launches == 3, "the rounds did not run on resident columns"
+    xa, xb = plain.read_replicas(), res.read_replicas()
+    assert (xa.view(np.uint32) == xb.view(np.uint32)).all()
+    assert (plain.peer_trace(rounds - 16, 16) == res.peer_trace(rounds - 16, 16)).all()
+    (ca, la), (cb, lb) = plain.telemetry(rounds - 16, 16), res.telemetry(rounds - 16, 16)
+    np.testing.assert_allclose(cb, ca, rtol=2e-5)
+    np.testing.assert_allclose(lb, la, rtol=2e-5)
+    plain.close()
+    res.close()
+
+
+@pytest.mark.parametrize("objective", [0, 1])
+@pytest.mark.parametrize("M,d", [(4, 4096), (6, 4099), (64, 515), (130, 37), (1000, 131)])
+def test_resident_columns_match_the_oracle(nm, M, d, objective):
+    rng = np.random.default_rng(M + d)
+    P = random_policy(M, rng, zeros=0.2)
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=objective, seed=9, trace_rounds=64)
+    o = oracle.Sim(M, d, P, full_adj(M), alpha=0.05, rho=g.get_policy()[1], sigma=0.1, objective=objective, seed=9)
+    o.init(1.0, 1.0)
+    x0, c0 = g.read_replicas(), g.read_centres()       # (the two sides' initial normals differ in the last bit)
+    o.set_x(x0)
+    o.set_c(c0)
+    for n in (30, 1, 9):
+        g.round(n)
+        o.round(n)
+    assert (g.peer_trace() == o.trace()).all()
+    got, want = g.read_replicas().astype(np.float64), o.x().astype(np.float64)
+    assert (np.abs(got - want) <= TOL * (1.0 + np.abs(want))).all()
+    gc, gl = g.telemetry()
+    oc, ol = o.telemetry()
+    np.testing.assert_allclose(gc, oc, rtol=1e-4, atol=1e-9)
+    np.testing.assert_allclose(gl, ol, rtol=1e-4, atol=1e-9)
+    g.close()
+
+
+def test_split_calls_change_no_bit_of_replicas_trace_or_telemetry(nm):
+    """Every round runs on resident columns whatever the call pattern, so even telemetry is bit-identical."""
+    rng = np.random.default_rng(8)
+    M, d = 5, 2051
+    kw = dict(M=M, d=d, lr=0.05, prob=random_policy(M, rng), sigma=0.1, x0_std=1.0, c_std=1.0, seed=11, trace_rounds=16)
+    a, b = nm.Netmax(**kw), nm.Netmax(**kw)
+    a.round(37)
+    for n in (1, 0, 15, 16, 5):
+        b.round(n)
+    assert (a.read_replicas() == b.read_replicas()).all()
+    ta, tb = a.telemetry(21, 16), b.telemetry(21, 16)
+    assert (ta[0] == tb[0]).all() and (ta[1] == tb[1]).all()
+    a.close()
+    b.close()
