@@ -47,7 +47,7 @@ struct DeviceGuard {
 
 struct ResidentPlan {  // launch shape of resident_rounds_kernel
   bool ok = false;
-  int threads = 0, grid = 0, G = 0, log2G = 0, draws_in_smem = 0;
+  int threads = 0, grid = 0, G = 0, log2G = 0, draw_chunk = 0;
   size_t smem = 0;
   int64_t n_tiles = 0, max_rounds = 0;
 };
@@ -504,9 +504,13 @@ int plan_round(netmax_ctx* ctx, RoundPlan& plan, int objective) {
   return NETMAX_OK;
 }
 
-size_t resident_smem(int64_t M, int threads, int G, bool draws) {
-  return (size_t)48 * M * G + 2 * sizeof(float) * resident_scratch_floats(threads, G) + 128 * sizeof(double) +
-         (draws ? (size_t)16 * M : 0);
+// Rounds whose draws the resident kernel stages in shared memory at a time: about 8 KB worth
+// for up to 512 workers, none beyond (threads then fetch the draws of their own rows).
+int resident_draw_chunk(int64_t M) { return M <= 512 ? (int)std::max<int64_t>(2, 1024 / M) : 0; }
+
+size_t resident_smem(int64_t M, int threads, int G) {
+  return (size_t)48 * M * G + 2 * sizeof(float) * resident_scratch_floats(threads, G) + 128 * sizeof(float) +
+         (size_t)resident_draw_chunk(M) * M * 8;
 }
 
 // Short vectors whose M rows of at least one column group fit in a CTA's shared memory run all
@@ -520,10 +524,21 @@ int plan_resident_uncached(netmax_ctx* ctx, const RoundPlan& plan, ResidentPlan&
   const int64_t M = ctx->M, nq = (ctx->d + 3) / 4;
   const size_t limit = (size_t)224 * 1024;
   int threads = 0, G = 0;
-  for (int cand : {32, 64, 128, 256}) {  // a thread per column group
-    if (resident_smem(M, cand, cand, M <= cand) > (size_t)100 * 1024) break;
-    threads = G = cand;
-    if ((nq + cand - 1) / cand <= (int64_t)8 * ctx->sm_count) break;
+  if (resident_smem(M, 32, 32) <= (size_t)100 * 1024) {
+    // small M.  The problem is latency-bound: give a thread as few rows as still leaves about two
+    // warps per scheduler busy, i.e. split the rows of a group over RL lanes (a power of two)
+    const int64_t target_threads = (int64_t)ctx->sm_count * 256;
+    const int64_t rows_per_thread = std::max<int64_t>(1, M * nq / target_threads);
+    int RL = 1;
+    while (RL < 32 && RL < M && (M + RL - 1) / RL > rows_per_thread) RL <<= 1;
+    for (int cand : {32, 64, 128, 256}) {
+      const int g = cand / RL;
+      if (g < 1 || (RL > 1 && g > 32)) break;
+      if (resident_smem(M, cand, g) > (size_t)100 * 1024) break;
+      threads = cand;
+      G = g;
+      if ((nq + g - 1) / g <= (int64_t)8 * ctx->sm_count) break;
+    }
   }
   if (threads == 0) {  // rows of a group split over the threads
     G = 32;
@@ -531,14 +546,14 @@ int plan_resident_uncached(netmax_ctx* ctx, const RoundPlan& plan, ResidentPlan&
     while (G > 1 && (nq + G - 1) / G < ctx->sm_count) G >>= 1;
     threads = (int)std::min<int64_t>(512, std::max<int64_t>(64, floor_pow2(M * G / 2)));
     threads = std::max(threads, G);
-    if (resident_smem(M, threads, G, M <= threads) > limit) return NETMAX_OK;
+    if (resident_smem(M, threads, G) > limit) return NETMAX_OK;
   }
   f.threads = threads;
   f.G = G;
   f.log2G = 0;
   while ((1 << f.log2G) < G) ++f.log2G;
-  f.draws_in_smem = M <= threads ? 1 : 0;
-  f.smem = resident_smem(M, threads, G, f.draws_in_smem != 0);
+  f.draw_chunk = (int)std::min<int64_t>(resident_draw_chunk(M), ctx->trace_rounds);
+  f.smem = resident_smem(M, threads, G);
   f.n_tiles = (nq + G - 1) / G;
   f.max_rounds = std::max<int64_t>(1, std::min<int64_t>(kMaxRoundsPerLaunch, (int64_t)(kColPartBytes / 16) / f.n_tiles));
   ResidentKernel k = pick_resident_kernel(ctx->objective, ctx->L.halves);
@@ -978,7 +993,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
         rp.tail = (int32_t)(ctx->d % 4);
         rp.G = resident.G;
         rp.log2G = resident.log2G;
-        rp.draws_in_smem = resident.draws_in_smem;
+        rp.draw_chunk = resident.draw_chunk;
         rp.alpha = p.alpha;
         rp.sigma = p.sigma;
         rp.inv_M = p.inv_M;

@@ -750,15 +750,16 @@ struct ResidentParams {
   uint32_t row_bytes;
   int32_t M, tail;        // tail = d % 4
   int32_t G, log2G;       // column groups per tile (a power of two)
-  int32_t draws_in_smem;  // 1: the round's (peer, weight) pairs are staged in shared memory, one round ahead
+  int32_t draw_chunk;     // > 0: the (peer, weight) pairs of this many rounds at a time are staged in shared
+                          // memory; 0 (large M): every thread loads the draws of its own rows, a round ahead
   float alpha, sigma, inv_M;
   uint32_t q_offset;
   PhiloxKeys keys;
 };
 
 // Dynamic shared memory: slabs float4[3][M][G]; then (G < blockDim) two reduction scratch
-// buffers float[warps][G][9] (padded to 16 bytes); then 2 x 64 doubles; then (draws_in_smem,
-// which needs M <= blockDim) int2[2][M].
+// buffers float[warps][G][9] (padded to 16 bytes); then 2 x 64 floats; then int2[draw_chunk][M].
+constexpr int kDrawRegs = 8;  // large M: draws of a thread's first rows that are fetched a round ahead
 #ifndef NETMAX_RESIDENT_UNROLL
 #define NETMAX_RESIDENT_UNROLL 2
 #endif
@@ -778,7 +779,7 @@ __global__ void __launch_bounds__(512) resident_rounds_kernel(const ResidentPara
   unsigned char* slab = smem_raw + (uint32_t)g * 16u;
   float* s_scratch = reinterpret_cast<float*>(smem_raw + 3u * plane);
   const uint32_t scratch_floats = resident_scratch_floats(T, G);
-  double* s_red = reinterpret_cast<double*>(s_scratch + 2 * scratch_floats);
+  float* s_red = s_scratch + 2 * scratch_floats;  // 2 x 64 floats
   int2* s_pw = reinterpret_cast<int2*>(s_red + 128);
 
   for (int64_t tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x) {
@@ -803,36 +804,45 @@ __global__ void __launch_bounds__(512) resident_rounds_kernel(const ResidentPara
       *reinterpret_cast<ulonglong2*>(slab + (uint32_t)i * stride) = xv;
       *reinterpret_cast<ulonglong2*>(slab + 2u * plane + (uint32_t)i * stride) = cv;
     }
-    if (p.draws_in_smem) {  // the first round's draws
-      const int64_t at = (p.slot0 % p.ring) * M;
-      for (int i = tid; i < M; i += T) s_pw[i] = make_int2(__ldg(p.trace + at + i), __float_as_int(__ldg(p.wring + at + i)));
+    int64_t slot = p.slot0 % p.ring;  // ring slot of round k, stepped along with k
+    const int KC = p.draw_chunk;      // rounds whose draws are staged in shared memory at a time (0: none)
+    int2 dreg[kDrawRegs];             // KC == 0: the draws of this thread's first rows, loaded a round ahead
+    if (KC == 0 && live) {
+#pragma unroll
+      for (int j = 0; j < kDrawRegs; ++j) {
+        const int i = r + j * RL;
+        if (i < M) dreg[j] = make_int2(__ldg(p.trace + slot * M + i), __float_as_int(__ldg(p.wring + slot * M + i)));
+      }
     }
     __syncthreads();
 
     for (int k = 0; k < p.n_rounds; ++k) {
       const uint64_t round = p.first_round + (uint64_t)k;
       const uint32_t round_lo = (uint32_t)round, ctr3 = philox_ctr3(kTagNoise, round);
-      const int64_t at = ((p.slot0 + k) % p.ring) * M;
+      const int kc = KC > 0 ? k % KC : 0;
+      if (KC > 0 && kc == 0) {
+        // stage the draws of the next KC rounds (the previous round's barrier has retired their predecessors)
+        const int n = min(KC, p.n_rounds - k) * M;
+#pragma unroll 4
+        for (int idx = tid; idx < n; idx += T) {
+          const int ahead = idx / M;  // rounds ahead of round k
+          int64_t s2 = slot + ahead;
+          if (s2 >= p.ring) s2 -= p.ring;  // (a chunk is never longer than the ring)
+          const int64_t src = s2 * M + (idx - ahead * M);
+          s_pw[idx] = make_int2(__ldg(p.trace + src), __float_as_int(__ldg(p.wring + src)));
+        }
+        __syncthreads();
+      }
+      const int64_t at = slot * M;
+      slot = slot + 1 == p.ring ? 0 : slot + 1;
       const unsigned char* cur = slab + (uint32_t)(k & 1) * plane;
       unsigned char* nxt = slab + (uint32_t)((k & 1) ^ 1) * plane;
       const unsigned char* cen = slab + 2u * plane;
-      const int2* pw = s_pw + (k & 1) * M;
-      // next round's draws: issue the loads now, park them in shared memory after the arithmetic
-      int2 ahead = make_int2(0, 0);
-      const bool fetch = p.draws_in_smem && k + 1 < p.n_rounds && tid < M;
-      if (fetch) {
-        const int64_t at1 = ((p.slot0 + k + 1) % p.ring) * M;
-        ahead = make_int2(__ldg(p.trace + at1 + tid), __float_as_int(__ldg(p.wring + at1 + tid)));
-      }
       ColAcc acc;
       LossAcc lacc;
       if (live) {
         const ulonglong2 pivot = *reinterpret_cast<const ulonglong2*>(cur);
-#pragma unroll kResidentUnroll
-        for (int i = r; i < M; i += RL) {
-          int2 d;
-          if (p.draws_in_smem) d = pw[i];
-          else d = make_int2(__ldg(p.trace + at + i), __float_as_int(__ldg(p.wring + at + i)));
+        auto do_row = [&](int i, int2 d) {
           const uint32_t off = (uint32_t)i * stride;
           ulonglong2 o = row_update<kObjective, kFastNoise>(
               p.alpha, p.sigma, p.keys, round_lo, ctr3, q32, (uint32_t)i, *reinterpret_cast<const ulonglong2*>(cur + off),
@@ -840,9 +850,28 @@ __global__ void __launch_bounds__(512) resident_rounds_kernel(const ResidentPara
               pivot, __int_as_float(d.y), live_lo, acc, lacc);
           if (kBf16) o = widen_bf16x4(narrow_bf16x4(o));
           *reinterpret_cast<ulonglong2*>(nxt + off) = o;
+        };
+        if (KC > 0) {
+          const int2* pw = s_pw + kc * M;
+#pragma unroll kResidentUnroll
+          for (int i = r; i < M; i += RL) do_row(i, pw[i]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < kDrawRegs; ++j) {
+            const int i = r + j * RL;
+            if (i < M) do_row(i, dreg[j]);
+          }
+          for (int i = r + kDrawRegs * RL; i < M; i += RL)
+            do_row(i, make_int2(__ldg(p.trace + at + i), __float_as_int(__ldg(p.wring + at + i))));
+          if (k + 1 < p.n_rounds) {  // next round's draws: in flight during the reduction below
+#pragma unroll
+            for (int j = 0; j < kDrawRegs; ++j) {
+              const int i = r + j * RL;
+              if (i < M) dreg[j] = make_int2(__ldg(p.trace + slot * M + i), __float_as_int(__ldg(p.wring + slot * M + i)));
+            }
+          }
         }
       }
-      if (fetch) s_pw[((k & 1) ^ 1) * M + tid] = ahead;  // (M <= blockDim in this mode: one entry per thread)
       // ---- telemetry of the round: column sums over the row lanes, then over the tile
       float v[9];
       unpack2(acc.s1a, v[0], v[1]);
@@ -856,13 +885,16 @@ __global__ void __launch_bounds__(512) resident_rounds_kernel(const ResidentPara
         v[8] = (l0 + l1) + (l2 + l3);
       }
       float* scratch = s_scratch + (k & 1) * scratch_floats;
-      double* red = s_red + (k & 1) * 64;
+      float* red = s_red + (k & 1) * 64;
       bool owner = true;  // does this thread hold the complete sums of its column group?
       if (RL > 1) {
         for (int off = 16; off >= G; off >>= 1) {
 #pragma unroll
           for (int a = 0; a < 9; ++a) v[a] += __shfl_xor_sync(0xffffffffu, v[a], off);
         }
+        owner = lane < G;  // a single warp: its lanes 0 .. G-1 now hold the sums of their groups
+      }
+      if (RL > 1 && nwarps > 1) {
         if (lane < G) {
 #pragma unroll
           for (int a = 0; a < 9; ++a) scratch[(warp * G + lane) * 9 + a] = v[a];
@@ -878,11 +910,11 @@ __global__ void __launch_bounds__(512) resident_rounds_kernel(const ResidentPara
           }
         }
       }
-      double cons = 0.0, loss = 0.0;
+      float cons = 0.f, loss = 0.f;
       if (owner) {
-        cons = (double)((v[4] - v[0] * v[0] * p.inv_M) + (v[5] - v[1] * v[1] * p.inv_M) + (v[6] - v[2] * v[2] * p.inv_M) +
-                        (v[7] - v[3] * v[3] * p.inv_M));
-        loss = 0.5 * (double)v[8];
+        cons = (v[4] - v[0] * v[0] * p.inv_M) + (v[5] - v[1] * v[1] * p.inv_M) + (v[6] - v[2] * v[2] * p.inv_M) +
+               (v[7] - v[3] * v[3] * p.inv_M);
+        loss = v[8];
       }
       for (int off = 16; off > 0; off >>= 1) {
         cons += __shfl_down_sync(0xffffffffu, cons, off);
@@ -896,12 +928,12 @@ __global__ void __launch_bounds__(512) resident_rounds_kernel(const ResidentPara
       if (tid == 0) {
         double a = 0.0, b = 0.0;
         for (int w = 0; w < nwarps; ++w) {
-          a += red[w];
-          b += red[32 + w];
+          a += (double)red[w];
+          b += (double)red[32 + w];
         }
         double* out = p.partials + ((size_t)k * p.n_tiles + tile) * 2;
         out[0] = a;
-        out[1] = b;
+        out[1] = 0.5 * b;
       }
     }
 
