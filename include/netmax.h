@@ -105,8 +105,9 @@ typedef struct netmax_config {
   int32_t storage;               /* NETMAX_STORAGE_F32 (default) or NETMAX_STORAGE_BF16: see above       */
   int32_t fuse_rounds;           /* rounds that one launch may advance a tile of long vectors while it is
                                     resident on chip (see netmax_round): 0 (default) automatic, 1 never
-                                    (one launch per round), 2..4 at most that many.  Replicas and peer
-                                    traces do not depend on it                                           */
+                                    (one launch per round; short vectors then do not keep columns in shared
+                                    memory either), 2..4 at most that many.  Replicas and peer traces do
+                                    not depend on it                                                     */
 } netmax_config;
 
 /* Fills *cfg with defaults: rho = 0 (automatic), sigma = 0, stds 0, objective 1, seed 0,
@@ -153,7 +154,10 @@ int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
  * Eq. 16 to every element of every replica, reading the round-start buffer and writing the
  * other one, and reduces that round's telemetry.  The peers of up to trace_rounds rounds are
  * drawn ahead in one sampler launch (the draws are counter-based and do not depend on x).
- * Short vectors (a round of a few microseconds) run all rounds of a call in one cooperative
+ * Short vectors (a round of a few microseconds) whose M rows of at least one four-element column
+ * group fit in a CTA's shared memory (M up to about 4700) run all rounds of a call on
+ * shared-memory-resident columns: CTAs own disjoint columns and never exchange anything.
+ * Other short-vector shapes (and fuse_rounds = 1) run all rounds of a call in one cooperative
  * launch with a grid-wide barrier per round; its waits are bounded, and one that runs out is
  * reported by the next synchronising call as NETMAX_CUDA_ERROR (the replicas are then not
  * valid).
@@ -163,8 +167,7 @@ int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
  * sees x and c once per launch instead of once per round.
  * Whatever the launch shape and however a run is split into calls, replicas and peer traces
  * are the same bit for bit; telemetry sums are accumulated in an order that depends on the
- * launch shape and agree to rounding (1e-12 relative with fp32 state, 1e-6 with bfloat16
- * state, whose per-thread fp32 partial sums span eight or four columns).
+ * launch shape and agree to fp32 rounding of their partial sums (2e-5 relative or better).
  */
 int netmax_round(netmax_ctx* ctx, int64_t n_rounds);
 
