@@ -24,6 +24,28 @@ def test_library_exports_every_declared_symbol():
     assert sorted(binding.EXPORTS) == declared
 
 
+def test_binding_config_matches_the_header_field_by_field(tmp_path):
+    """The ctypes mirror of netmax_config must have the C compiler's layout: a small C program that
+    includes the header prints the size of the struct and the offset of every field."""
+    import subprocess
+    fields = [name for name, _ in binding.Config._fields_]
+    src = tmp_path / "layout.c"
+    lines = ['#include <stddef.h>', '#include <stdio.h>', f'#include "{os.path.join(ROOT, "include", "netmax.h")}"',
+             'int main(void) {', '  printf("%zu\\n", sizeof(netmax_config));']
+    lines += [f'  printf("%zu\\n", offsetof(netmax_config, {f}));' for f in fields]
+    lines += ['  return 0;', '}']
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-o", str(exe), str(src)], check=True)
+    out = [int(v) for v in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
+    assert out[0] == C.sizeof(binding.Config)
+    assert out[1:] == [getattr(binding.Config, f).offset for f in fields]
+    header = re.sub(r"/\*.*?\*/", "", open(os.path.join(ROOT, "include", "netmax.h")).read(), flags=re.S)
+    body = re.search(r"typedef struct netmax_config \{(.*?)\} netmax_config;", header, flags=re.S).group(1)
+    declared = re.findall(r"\b([A-Za-z_0-9]+)\s*(?:,|;)", body)
+    assert declared == fields      # every field of the header is mirrored, in order
+
+
 def test_iteration_times_match_oracle():
     for idx in (1, 2, 3, 4):
         w = workloads.config(idx)
