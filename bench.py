@@ -241,7 +241,7 @@ def run_ours(args, w):
         raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
 
     base = None
-    if rank == 0 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
         base = cpu_baseline(w, storage=args.storage)          # before the first CUDA call
 
     if not torch.cuda.is_available():
