@@ -34,7 +34,9 @@
 //
 // Parity pins (see tests/): Philox against cuRAND's host generator; normals against
 // the normal law; sampler against exact threshold sweeps and chi-square; the update
-// against the M=2 closed form, D^k products, contraction and fixed points.
+// against the M=2 closed form, D^k products, contraction and fixed points; the initial
+// state (fill_normal) value by value against the composition of the two pinned primitives
+// written out in numpy, against the normal law, and for the independence of its streams.
 // Telemetry (consensus distance, mean loss) is not defined by the paper: parity unpinned
 // by the paper; it is pinned against a direct numpy evaluation of its definition.
 
