@@ -198,6 +198,8 @@ struct Sim {
   std::vector<double> t_iter;          // [M][M] iteration times, t_ii = compute-only
   std::vector<int64_t> local_n;        // [M] local iteration index n of the pending iteration
   std::vector<int32_t> pending_peer;   // [M] peer drawn for the pending iteration
+  std::vector<float> pending_w;        // [M] its pull weight, from the policy in force when it started
+  std::vector<double> pending_t;       // [M] its duration t_im, from the times in force when it started
   std::vector<double> finish;          // [M] simulated time at which the pending iteration ends
   std::vector<double> ema;             // [M][M] EMA of measured iteration times (Algorithm 2)
   std::vector<int64_t> ema_count;      // [M][M] samples folded into the EMA
@@ -349,14 +351,19 @@ void sim_round(Sim* s, int threads) {
 // ---------------------------------------------------------------- asynchronous timeline
 // Worker i's iteration n: peer m drawn from P[i,:] with the PEER stream at counter (0, i, n),
 // duration t_im (Section II-B: t_im = max{C_i, N_im}); the next iteration starts when this
-// one ends.  A policy or time-matrix change affects iterations that START afterwards.
+// one ends.  Algorithm 2 takes a new policy (P[i], rho) at the top of an iteration, before the
+// peer is selected, and its UpdateTimeVector records how long the iteration took: so the pull
+// weight alpha rho gamma_im and the duration t_im of an iteration are those in force when it
+// STARTS, whatever changes while it is in flight.
 void async_start_iteration(Sim* s, int i, double start) {
   uint32_t ctr[4], r[4];
   make_ctr(0, (uint32_t)i, (uint64_t)s->local_n[i], TAG_PEER, ctr);
   philox4x32_10(ctr, s->key, r);
   const int m = sample_row(s->T.data() + (size_t)i * s->M, s->M, s->last_nz[i], r[0]);
   s->pending_peer[i] = m;
-  s->finish[i] = start + s->t_iter[(size_t)i * s->M + m];
+  s->pending_w[i] = (m != i) ? s->w[(size_t)i * s->M + m] : 0.0f;
+  s->pending_t[i] = s->t_iter[(size_t)i * s->M + m];
+  s->finish[i] = start + s->pending_t[i];
 }
 
 // One global step (Eq. 17): the worker whose iteration finishes first (ties: lowest index)
@@ -370,7 +377,8 @@ void async_step(Sim* s) {
     if (s->finish[j] < s->finish[i]) i = j;
   const int m = s->pending_peer[i];
   const int64_t nloc = s->local_n[i];
-  const double w = (double)s->w[(size_t)i * M + m];
+  const float wf = s->pending_w[i];  // fixed when the iteration started (0 on a self-draw)
+  const double w = (double)wf;
   const int64_t n = s->ncols;
   float* xi = s->x.data() + (size_t)i * n;
   const float* xm = s->x.data() + (size_t)m * n;
@@ -378,7 +386,6 @@ void async_step(Sim* s) {
   for (int64_t k = 0; k < n; ++k) {
     const int64_t e = s->cols[k];
     if (s->storage == 1) {  // bfloat16 state: the same fp32 evaluation as in a round, rounded once
-      const float wf = (m != i) ? s->w[(size_t)i * M + m] : 0.0f;
       const float xnew = update_fp32(s, i, (uint64_t)nloc, e, xi[k], ci[k], xm[k], (float)s->alpha, (float)s->sigma, wf);
       s->pre[(size_t)i * n + k] = xnew;
       xi[k] = bf16_round(xnew);
@@ -405,7 +412,7 @@ void async_step(Sim* s) {
   s->ev_n.push_back(nloc);
   s->ev_time.push_back(s->now);
   const size_t at = (size_t)i * M + m;
-  s->ema[at] = s->beta * s->ema[at] + (1.0 - s->beta) * s->t_iter[at];
+  s->ema[at] = s->beta * s->ema[at] + (1.0 - s->beta) * s->pending_t[i];  // the time this iteration took
   s->ema_count[at] += 1;
   s->local_n[i] = nloc + 1;
   async_start_iteration(s, i, s->now);
@@ -555,6 +562,8 @@ void nmo_async_begin(void* h, const double* t_iter, double beta) {
   s->t_iter.assign(t_iter, t_iter + (size_t)M * M);
   s->local_n.assign(M, 0);
   s->pending_peer.assign(M, 0);
+  s->pending_w.assign(M, 0.0f);
+  s->pending_t.assign(M, 0.0);
   s->finish.assign(M, 0.0);
   s->ema.assign((size_t)M * M, 0.0);
   s->ema_count.assign((size_t)M * M, 0);

@@ -211,3 +211,44 @@ def test_policy_change_applies_to_iterations_started_afterwards():
     worker, peer, local_iter, _ = sim.async_trace()
     assert (peer[:6] == (worker[:6] + 1) % M).all()
     assert (peer[6:] == (worker[6:] + 2) % M).all()
+
+
+def test_an_iteration_in_flight_keeps_the_weight_and_time_it_started_with():
+    """Algorithm 2 reads P[i] and rho at the top of an iteration, before it draws the peer, and
+    UpdateTimeVector folds in the time the iteration took.  An iteration that is in flight when
+    the policy or the iteration times change therefore pulls with the OLD alpha rho / (2 p_im) and
+    records the OLD t_im -- also when the new policy gives that peer probability zero."""
+    M, d, alpha, beta = 3, 5, 0.1, 0.5
+    P1 = np.array([[0, 1.0, 0], [0, 0, 1.0], [1.0, 0, 0]])          # i pulls from i + 1
+    P2 = np.array([[0, 0, 1.0], [1.0, 0, 0], [0, 1.0, 0]])          # i pulls from i + 2: p_{i,i+1} becomes 0
+    rho1, rho2 = 0.8, 2.4
+    t1 = np.array([[0.1, 1.0, 1.0], [1.0, 0.1, 1.0], [1.0, 1.0, 0.1]])
+    t2 = 3.0 * t1
+    x0 = np.random.default_rng(12).standard_normal((M, d)).astype(np.float32)
+    sim = oracle.Sim(M, d, P1, full_adj(M), alpha=alpha, rho=rho1, sigma=0.0, objective=0, seed=13)
+    sim.set_x(x0)
+    sim.async_begin(t1, beta=beta)
+    # all three first iterations are in flight (peers drawn under P1, finishing at t = 1)
+    sim.set_policy(P2, full_adj(M), rho2)
+    sim.async_set_times(t2)
+    a32 = float(np.float32(alpha))
+    w_old = float(np.float32(a32 * rho1 * 2.0 / (2.0 * 1.0)))
+    w_new = float(np.float32(a32 * rho2 * 2.0 / (2.0 * 1.0)))
+    x = x0.astype(np.float64)
+    for k in range(6):
+        sim.async_steps(1)
+        worker, peer, local_iter, time = sim.async_trace(k, 1)
+        i, m, n = int(worker[0]), int(peer[0]), int(local_iter[0])
+        w = w_old if n == 0 else w_new                             # iteration 0 started before the change
+        assert m == ((i + 1) % M if n == 0 else (i + 2) % M)
+        assert time[0] == pytest.approx(1.0 if n == 0 else 4.0)    # 1 s under t1, then 3 s under t2
+        x[i] = np.float32(x[i] - w * (x[i] - x[m]))
+        np.testing.assert_allclose(sim.x(), x, atol=1e-6)
+        assert np.abs(sim.x()[i].astype(np.float64) - x0[i]).max() > 1e-3 or n > 0   # the old-policy pull happened
+    ema, count = sim.async_ema()
+    want = np.zeros((M, M))
+    for i in range(M):
+        want[i, (i + 1) % M] = (1 - beta) * 1.0                    # the iteration in flight took t1 = 1 s
+        want[i, (i + 2) % M] = (1 - beta) * 3.0                    # the next one t2 = 3 s
+    np.testing.assert_allclose(ema, want, rtol=1e-12)
+    assert (count == (want > 0)).all()
