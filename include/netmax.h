@@ -81,7 +81,10 @@ typedef struct netmax_config {
   double lr;                     /* alpha > 0; the update uses its fp32 rounding                       */
   double rho;                    /* rho; <= 0: with prob given, the largest rho meeting Eq. 11 with a
                                     1e-6 margin, min_{p_im>0} p_im / (alpha (d_im+d_mi)); with prob
-                                    NULL, the rho Algorithm 3 selects                                  */
+                                    NULL, the rho Algorithm 3 selects.  A rho > 0 that breaks Eq. 11
+                                    (alpha rho (d_im+d_mi) > p_im on a link with p_im > 0, i.e. a pull
+                                    weight above 1/2) is rejected with NETMAX_INVALID_ARG unless
+                                    pull_weight replaces Eq. 16's weight                               */
   double pull_weight;            /* 0 (default): Eq. 16's weight alpha rho (d_im+d_mi)/(2 p_im).  In (0, 1):
                                     every pull uses this constant instead -- the update rule of gossip /
                                     AD-PSGD style averaging (1/2), which the paper's section on extending

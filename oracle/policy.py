@@ -6,7 +6,7 @@ iteration time t_bar, the row-wise linear programme (Eq. 14: minimise sum_i p_ii
 to Eq. 10-13), the matrix Y_P = E[D^T D] (Eq. 22) and its second largest eigenvalue, and
 the selection of the grid point with the smallest t_bar * ln(eps) / ln(lambda_2).
 
-Where the paper is silent or garbled the readings are (each is listed in the design doc):
+Where the paper is silent or garbled the readings are:
   * rho_k = k * U_rho / K and t_bar_r = L + r * (U - L) / R   (the printed loop bodies do
     not depend on the loop index);
   * U_rho = min(0.5/alpha, (1-1e-6) / (alpha * max_i sum_{m!=i} (d_im + d_mi))): beyond it

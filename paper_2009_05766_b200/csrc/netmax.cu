@@ -143,6 +143,8 @@ struct netmax_ctx {
   int64_t steps = 0;
   std::vector<int64_t> local_n;
   std::vector<int32_t> pending_peer;
+  std::vector<float> pending_weight;    // Eq. 16's weight for the pending iteration, under the policy it started with
+  std::vector<double> pending_duration; // t_im of the pending iteration, under the times it started with
   std::vector<double> finish;
   // pending iterations ordered by (finish time, worker): exactly one entry per worker
   std::priority_queue<std::pair<double, int>, std::vector<std::pair<double, int>>, std::greater<std::pair<double, int>>> queue;
@@ -251,6 +253,25 @@ double default_rho(int32_t M, const double* P, const std::vector<uint8_t>& adj, 
   return std::isfinite(best) ? (1.0 - 1e-6) * best : 0.0;
 }
 
+// A caller's rho must keep Eq. 11, p_im >= alpha rho (d_im + d_mi) on every link in use (taken
+// closed, as Algorithm 3's rows may sit on the floor): otherwise the pull weight of Eq. 16
+// exceeds 1/2, entries of Y_P (Eq. 22) can turn negative and Theorem 3's lambda_2 < 1 is lost.
+// With a fixed pull weight rho is unused and nothing is checked.
+int check_rho(netmax_ctx* ctx, int32_t M, const double* P, const std::vector<uint8_t>& adj, double alpha, double rho,
+              double pull_weight) {
+  if (pull_weight > 0.0) return NETMAX_OK;
+  for (int i = 0; i < M; ++i)
+    for (int m = 0; m < M; ++m) {
+      const double p = P[(size_t)i * M + m];
+      if (i == m || !(p > 0.0)) continue;
+      const double floor_im = alpha * rho * ((double)adj[(size_t)i * M + m] + (double)adj[(size_t)m * M + i]);
+      if (floor_im > p * (1.0 + 1e-9))
+        return fail(ctx, NETMAX_INVALID_ARG, "rho = %g breaks Eq. 11 on link (%d,%d): alpha rho (d_im + d_mi) = %g > p_im = %g",
+                    rho, i, m, floor_im, p);
+    }
+  return NETMAX_OK;
+}
+
 // T_j = floor(cum_j 2^32 + 1/2) over the left-to-right double prefix sums of the row,
 // non-decreasing, saturated, and pinned to the top from the last positive entry on.
 void build_tables(int32_t M, const double* P, const std::vector<uint8_t>& adj, double alpha32, double rho,
@@ -322,6 +343,10 @@ int resolve_policy(netmax_ctx* ctx, const double* speed, const double* prob, dou
   if (prob) {
     int rc = validate_policy(ctx, M, prob, ctx->adj);
     if (rc) return rc;
+    if (rho > 0.0) {
+      rc = check_rho(ctx, M, prob, ctx->adj, ctx->alpha, rho, ctx->pull_weight);
+      if (rc) return rc;
+    }
     ctx->P.assign(prob, prob + (size_t)M * M);
     ctx->rho = rho > 0.0 ? rho : default_rho(M, prob, ctx->adj, ctx->alpha);
     return NETMAX_OK;
@@ -337,6 +362,10 @@ int resolve_policy(netmax_ctx* ctx, const double* speed, const double* prob, dou
                      : netmax_policy_generate_ex(M, ctx->t_iter.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K,
                                                  ctx->policy_R, ctx->policy_rho_upper, ctx->P.data(), &rho_sel, nullptr);
   if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
+  if (rho > 0.0) {  // the caller's rho with Algorithm 3's P: it must still respect that P
+    rc = check_rho(ctx, M, ctx->P.data(), ctx->adj, ctx->alpha, rho, ctx->pull_weight);
+    if (rc) return rc;
+  }
   ctx->rho = rho > 0.0 ? rho : rho_sel;
   return NETMAX_OK;
 }
@@ -1140,7 +1169,7 @@ int netmax_read_columns(netmax_ctx* ctx, const int64_t* host_cols, int64_t n_col
   if (e != cudaSuccess) rc = fail(ctx, NETMAX_CUDA_ERROR, "read_columns: %s", cudaGetErrorString(e));
   cudaFree(d_cols);
   cudaFree(d_out);
-  return rc;
+  return rc ? rc : check_device_error(ctx);
 }
 
 // ---- sampled read-back that allocates nothing -------------------------------------------
@@ -1194,10 +1223,13 @@ int netmax_read_columns_static(netmax_ctx* ctx, const int64_t* host_cols, int64_
   NM_CUDA(ctx, cudaMemcpyAsync(scratch->cols, host_cols, (size_t)n_cols * sizeof(int64_t), cudaMemcpyHostToDevice, ctx->stream));
   gather_columns_kernel<<<grid, kThreads, 0, ctx->stream>>>(ctx->x[ctx->cur], ctx->storage == NETMAX_STORAGE_BF16, ctx->L.ld, ctx->M, scratch->cols, n_cols, scratch->values);
   ctx->launches += 1;
-  NM_CUDA(ctx, cudaGetLastError());
-  NM_CUDA(ctx, cudaMemcpyAsync(host_out, scratch->values, (size_t)total * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
-  NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-  return NETMAX_OK;
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaMemcpyAsync(host_out, scratch->values, (size_t)total * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream);
+  // whatever happened, leave the shared array idle: the next call, perhaps on another stream, reuses it
+  const cudaError_t es = cudaStreamSynchronize(ctx->stream);
+  if (e == cudaSuccess) e = es;
+  if (e != cudaSuccess) return fail(ctx, NETMAX_CUDA_ERROR, "read_columns_static: %s", cudaGetErrorString(e));
+  return check_device_error(ctx);
 }
 
 static int ring_range(netmax_ctx* ctx, int64_t first, int64_t n) {
@@ -1323,14 +1355,20 @@ static uint32_t host_peer_word(const PhiloxKeys& keys, uint32_t worker, uint64_t
 }
 
 // Draws the peer of worker i's next local iteration (Algorithm 2) and sets when it will finish.
+// The policy is read at the top of an iteration and the moving average records the time the
+// iteration took, so the pull weight and the duration are latched here: a policy or time
+// matrix that arrives while the iteration is in flight does not touch them.
 static void async_start_iteration(netmax_ctx* ctx, int i, double start) {
   const int32_t M = ctx->M;
   const uint32_t u = host_peer_word(ctx->keys, (uint32_t)i, (uint64_t)ctx->local_n[i]);
   const uint32_t* row = ctx->h_thr.data() + (size_t)i * M;
   const int32_t count = (int32_t)(std::upper_bound(row, row + M, u) - row);  // #{j : T[j] <= u}
   const int32_t m = std::min(count, ctx->h_last[i]);
+  const size_t link = (size_t)i * M + m;
   ctx->pending_peer[i] = m;
-  ctx->finish[i] = start + ctx->t_iter[(size_t)i * M + m];
+  ctx->pending_weight[i] = (m == i) ? 0.0f : ctx->h_w[link];
+  ctx->pending_duration[i] = ctx->t_iter[link];
+  ctx->finish[i] = start + ctx->pending_duration[i];
 }
 
 int netmax_async_begin(netmax_ctx* ctx, const double* t_iter, double beta) {
@@ -1353,6 +1391,8 @@ int netmax_async_begin(netmax_ctx* ctx, const double* t_iter, double beta) {
   ctx->steps = 0;
   ctx->local_n.assign(M, 0);
   ctx->pending_peer.assign(M, 0);
+  ctx->pending_weight.assign(M, 0.0f);
+  ctx->pending_duration.assign(M, 0.0);
   ctx->finish.assign(M, 0.0);
   ctx->ema.assign((size_t)M * M, 0.0);
   ctx->ema_count.assign((size_t)M * M, 0);
@@ -1475,7 +1515,7 @@ int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps) {
     e.peer = m;
     e.iter_lo = (uint32_t)n;
     e.ctr3 = philox_ctr3(kTagNoise, n);
-    e.w = (m == i) ? 0.0f : ctx->h_w[(size_t)i * M + m];
+    e.w = ctx->pending_weight[i];
     writes[i] = 1;
     reads[i] = 1;
     reads[m] = 1;
@@ -1487,7 +1527,7 @@ int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps) {
     ctx->ev_n[slot] = (int64_t)n;
     ctx->ev_time[slot] = ctx->now;
     const size_t at = (size_t)i * M + m;
-    ctx->ema[at] = ctx->beta * ctx->ema[at] + (1.0 - ctx->beta) * ctx->t_iter[at];
+    ctx->ema[at] = ctx->beta * ctx->ema[at] + (1.0 - ctx->beta) * ctx->pending_duration[i];
     ctx->ema_count[at] += 1;
     ctx->local_n[i] += 1;
     ctx->steps += 1;

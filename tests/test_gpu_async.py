@@ -99,6 +99,44 @@ def test_async_policy_and_time_changes_apply_to_later_iterations(nm):
     for a, b in zip(g.async_trace(), o.async_trace()):
         assert (a == b).all()
     close(g.read_replicas(), o.x())
+    for a, b in zip(g.async_ema(), o.async_ema()):
+        assert (a == b).all()
+    g.close()
+
+
+def test_iterations_in_flight_keep_their_weight_and_duration(nm):
+    """Algorithm 2 reads the policy at the top of an iteration and records the time the iteration
+    took: with every first iteration in flight, a new policy that gives the drawn peers probability
+    zero and a slower time matrix must leave those iterations' pulls (old alpha rho / (2 p_im)) and
+    moving averages (old t_im) untouched.  Closed form, no oracle."""
+    M, d, alpha, beta = 3, 1027, 0.1, 0.5
+    P1 = np.array([[0, 1.0, 0], [0, 0, 1.0], [1.0, 0, 0]])
+    P2 = np.array([[0, 0, 1.0], [1.0, 0, 0], [0, 1.0, 0]])
+    rho1, rho2 = 0.8, 2.4
+    t1 = np.array([[0.1, 1.0, 1.0], [1.0, 0.1, 1.0], [1.0, 1.0, 0.1]])
+    x0 = np.random.default_rng(12).standard_normal((M, d)).astype(np.float32)
+    g = nm.Netmax(M=M, d=d, lr=alpha, prob=P1, rho=rho1, objective=0, seed=13)
+    g.set_replicas(x0)
+    g.async_begin(t1, beta)
+    g.set_policy(prob=P2, rho=rho2)
+    g.async_set_times(3.0 * t1)
+    a32 = float(np.float32(alpha))
+    w_old, w_new = float(np.float32(a32 * rho1)), float(np.float32(a32 * rho2))
+    g.async_steps(6)
+    worker, peer, local_iter, time = g.async_trace()
+    x = x0.astype(np.float64)
+    for i, m, n, tt in zip(worker, peer, local_iter, time):
+        assert m == ((i + 1) % M if n == 0 else (i + 2) % M)
+        assert tt == pytest.approx(1.0 if n == 0 else 4.0)
+        x[i] = np.float32(x[i] - (w_old if n == 0 else w_new) * (x[i] - x[m]))
+    close(g.read_replicas(), x.astype(np.float32))
+    ema, count = g.async_ema()
+    want = np.zeros((M, M))
+    for i in range(M):
+        want[i, (i + 1) % M] = (1 - beta) * 1.0
+        want[i, (i + 2) % M] = (1 - beta) * 3.0
+    np.testing.assert_allclose(ema, want, rtol=1e-12)
+    assert (count == (want > 0)).all()
     g.close()
 
 

@@ -117,6 +117,7 @@ def test_create_validates_before_touching_the_gpu():
         (dict(M=M, d=8, lr=0.1, prob=good, sigma=-1.0), -1),
         (dict(M=M, d=8, lr=0.1, prob=good, objective=2), -1),
         (dict(M=M, d=8, lr=0.1, prob=good, trace_rounds=0), -1),
+        (dict(M=M, d=8, lr=0.1, prob=good, rho=2.6), -1),        # Eq. 11: alpha rho (d_im + d_mi) = 0.52 > p_im = 0.5
         (dict(M=M, d=8, lr=0.1, prob=good * 0.9), -2),
         (dict(M=M, d=8, lr=0.1, prob=np.array([[0, 1.5, -.5], [.5, 0, .5], [.5, .5, 0]])), -2),
         (dict(M=M, d=8, lr=0.1, prob=good, link_speed_gbps=np.array([[0, 1, 0], [1, 0, 1], [0, 1, 0.]])), -2),
@@ -126,6 +127,20 @@ def test_create_validates_before_touching_the_gpu():
         with pytest.raises(binding.NetmaxError) as e:
             binding.Netmax(**kw)
         assert e.value.code == code, (kw, str(e.value))
+
+
+def test_rho_beyond_eq_11_is_named_and_a_fixed_weight_or_the_floor_itself_passes(gpu_available):
+    good = np.array([[0, .5, .5], [.5, 0, .5], [.5, .5, 0]])
+    with pytest.raises(binding.NetmaxError) as e:
+        binding.Netmax(M=3, d=8, lr=0.1, prob=good, rho=2.6)
+    assert e.value.code == -1 and "Eq. 11" in str(e.value) and "(0,1)" in str(e.value)
+    # on the floor (w = 1/2, Eq. 11 taken closed) and with a fixed pull weight (rho unused) validation
+    # passes: without a GPU the call then fails later, at the device
+    for kw in (dict(rho=2.5), dict(rho=50.0, pull_weight=0.5)):
+        try:
+            binding.Netmax(M=3, d=8, lr=0.1, prob=good, **kw).close()
+        except binding.NetmaxError as err:
+            assert not gpu_available and err.code == -4, str(err)
 
 
 def test_null_context_calls_return_errors_not_crashes():
@@ -161,3 +176,15 @@ def test_explicit_rho_grid_matches_oracle_and_is_more_adaptive():
     assert rho < rhod
     fast, slow = P[0, 1], P[0, 5]
     assert fast / slow > Pd[0, 1] / Pd[0, 5] > 1.0
+
+
+def test_the_allocation_free_entry_point_names_no_allocating_call():
+    """netmax_read_columns_static promises to call no cudaMalloc / cudaFree: its body and the
+    helper that looks up the static array's address must not name one."""
+    src = open(os.path.join(ROOT, "paper_2009_05766_b200", "csrc", "netmax.cu")).read()
+    for start in ("int netmax_read_columns_static(", "static int gather_scratch_address("):
+        at = src.index(start)
+        body = src[at:src.index("\n}\n", at)]
+        assert "cudaGetSymbolAddress" in body or "gather_scratch_address" in body
+        for banned in ("cudaMalloc", "cudaFree", "cudaHostAlloc", "cudaMallocAsync", "new ", "std::vector"):
+            assert banned not in body, (start, banned)

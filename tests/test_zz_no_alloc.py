@@ -72,3 +72,35 @@ def test_static_read_back_is_shared_by_contexts_and_checks_its_limits(nm):
     assert b.read_columns_static(np.zeros(0, dtype=np.int64)).shape == (3, 0)
     a.close()
     b.close()
+
+
+def test_static_read_back_on_a_caller_owned_bfloat16_workspace_leaves_free_memory_alone(nm):
+    """The case the entry point exists for: every device buffer of the context lives in memory the
+    caller handed over (here a torch tensor, as a pool allocator would), the state is bfloat16 (the
+    gather widens it), and across a call the device's free memory does not move."""
+    import torch
+    M, d, ring = 5, 30011, 64
+    size = nm.Netmax.workspace_size(M, d, ring, storage="bf16")
+    ws = torch.empty(size + 256, dtype=torch.uint8, device="cuda")
+    ptr = (ws.data_ptr() + 255) // 256 * 256
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=_policy(M, 7), sigma=0.1, x0_std=1.0, c_std=1.0, seed=77, storage="bf16",
+                  trace_rounds=ring, workspace=ptr, workspace_bytes=size)
+    g.round(5)
+    cols = workloads.sample_columns(d, 2000, 3)
+    first = g.read_columns_static(cols)          # the first call on a device looks the array's address up
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    second = g.read_columns_static(cols)
+    third = g.read_columns_static(cols[::-1].copy())
+    free_after = torch.cuda.mem_get_info()[0]
+    assert free_after == free_before
+    want = g.read_replicas()[:, cols]            # (a bfloat16 context stages this through its own spare buffer)
+    assert (first == want).all() and (second == want).all() and (third == want[:, ::-1]).all()
+    assert (want == nm_bf16_exact(want)).all()   # the values are bfloat16 codes, widened exactly
+    g.close()
+    del ws
+
+
+def nm_bf16_exact(a):
+    """fp32 values with the low 16 bits cleared: what an exactly widened bfloat16 looks like."""
+    return (a.view(np.uint32) & np.uint32(0xFFFF0000)).view(np.float32)
