@@ -19,7 +19,7 @@
  *     the context's device.  Inputs are borrowed for the duration of the call and copied;
  *     outputs are caller-allocated and caller-owned.
  *   - Matrices are row-major M x M; replica arrays are dense row-major M x d (no padding).
- *   - Rounds are numbered from 0 over the life of a context.  All random numbers are
+ *   - Rounds are numbered from netmax_config.first_round (default 0) over the life of a context.  All random numbers are
  *     Philox4x32-10 blocks addressed by (seed, stream, worker, round, element), so splitting
  *     netmax_round(a + b) into netmax_round(a); netmax_round(b) changes no bit.
  *   - Work is enqueued on the context's stream.  Calls that return data to the host
@@ -111,11 +111,15 @@ typedef struct netmax_config {
                                     (one launch per round; short vectors then do not keep columns in shared
                                     memory either), 2..4 at most that many.  Replicas and peer traces do
                                     not depend on it                                                     */
+  int64_t first_round;           /* number of the context's first round, 0 <= first_round < 2^56 (default 0).  Rounds are
+                                    numbered from here; the round number is a word of every Philox counter, so a run
+                                    that is resumed from saved replicas at round r (netmax_set_replicas) with
+                                    first_round = r continues the streams of the run it was saved from               */
 } netmax_config;
 
 /* Fills *cfg with defaults: rho = 0 (automatic), sigma = 0, stds 0, objective 1, seed 0,
  * device 0, stream NULL, trace_rounds 1024, policy grid 20 x 20, no workspace, offset 0,
- * fp32 storage. */
+ * fp32 storage, first round 0. */
 int netmax_config_init(netmax_config* cfg);
 
 /* Device bytes a context with this M, d, trace_rounds and storage needs (only those fields are read). */
@@ -178,7 +182,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds);
  * round, 2..4 at most that many rounds per launch). */
 int netmax_set_fuse_rounds(netmax_ctx* ctx, int32_t fuse_rounds);
 
-/* Number of rounds enqueued so far. */
+/* Number of the next round: netmax_config.first_round plus the rounds enqueued so far. */
 int64_t netmax_rounds_done(const netmax_ctx* ctx);
 
 /* Synchronises, then copies the current replicas to host_out (M*d floats, dense; bfloat16
@@ -227,8 +231,8 @@ int netmax_read_columns_static(netmax_ctx* ctx, const int64_t* host_cols, int64_
 
 /*
  * Peers drawn in rounds [first_round, first_round + n): host_out[(r - first_round) * M + i]
- * is the peer of worker i in round r.  Only the last trace_rounds rounds are kept;
- * NETMAX_TRACE_RANGE otherwise.  Synchronises.
+ * is the peer of worker i in round r (an absolute round number, >= netmax_config.first_round).
+ * Only the last trace_rounds rounds are kept; NETMAX_TRACE_RANGE otherwise.  Synchronises.
  */
 int netmax_peer_trace(netmax_ctx* ctx, int64_t first_round, int64_t n, int32_t* host_out);
 

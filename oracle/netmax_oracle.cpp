@@ -185,7 +185,8 @@ struct Sim {
   int storage = 0;                       // 0: fp32 state, double arithmetic; 1: bfloat16 state, fp32 arithmetic
   std::vector<float> pre;                // storage 1: fp32 values of the last round before the bfloat16 rounding
   uint32_t key[2] = {0, 0};
-  uint64_t round = 0;
+  uint64_t round = 0;   // number of the next round: a word of every counter
+  uint64_t round0 = 0;  // number of the first round (the trace and telemetry vectors start there)
   std::vector<uint32_t> T;
   std::vector<int32_t> last_nz;
   std::vector<float> w;
@@ -536,7 +537,10 @@ void nmo_sim_round(void* h, int64_t n_rounds, int32_t threads) {
   for (int64_t r = 0; r < n_rounds; ++r) sim_round((Sim*)h, threads);
 }
 
-int64_t nmo_sim_rounds_done(void* h) { return (int64_t)((Sim*)h)->round; }
+// Rounds run since creation (the trace holds that many).
+int64_t nmo_sim_rounds_done(void* h) { return (int64_t)(((Sim*)h)->round - ((Sim*)h)->round0); }
+// Before any round: number the rounds from `first` on (the round number enters every counter).
+void nmo_sim_set_first_round(void* h, uint64_t first) { ((Sim*)h)->round = ((Sim*)h)->round0 = first; }
 
 void nmo_sim_get_trace(void* h, int64_t first, int64_t n, int32_t* out) {
   Sim* s = (Sim*)h;

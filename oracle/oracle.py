@@ -63,6 +63,7 @@ def lib():
         L.nmo_sim_round.argtypes = [vp, i64, i32]
         L.nmo_sim_rounds_done.argtypes = [vp]
         L.nmo_sim_rounds_done.restype = i64
+        L.nmo_sim_set_first_round.argtypes = [vp, u64]
         L.nmo_sim_get_trace.argtypes = [vp, i64, i64, vp]
         L.nmo_sim_get_telemetry.argtypes = [vp, i64, i64, vp, vp]
         L.nmo_sim_telemetry_now.argtypes = [vp, vp, vp]
@@ -154,7 +155,8 @@ def peer_draws(P: np.ndarray, seed: int, first_round: int, n_rounds: int) -> np.
 class Sim:
     """The round simulator: all M replicas (or a sample of their columns) on the CPU."""
 
-    def __init__(self, M, d, P, adj, alpha, rho, sigma, objective, seed, cols=None, pull_weight=0.0, storage="f32"):
+    def __init__(self, M, d, P, adj, alpha, rho, sigma, objective, seed, cols=None, pull_weight=0.0, storage="f32",
+                 first_round=0):
         self.M, self.d = int(M), int(d)
         self._P = np.ascontiguousarray(P, dtype=np.float64)
         self._adj = np.ascontiguousarray(adj, dtype=np.uint8)
@@ -173,6 +175,8 @@ class Sim:
         self.storage = storage
         if storage == "bf16":      # bfloat16 state, fp32 arithmetic, one rounding per stored value
             lib().nmo_sim_set_storage(self._h, 1)
+        if first_round:            # rounds numbered from here (trace and telemetry indices stay relative)
+            lib().nmo_sim_set_first_round(self._h, int(first_round))
 
     def close(self):
         if self._h:

@@ -43,7 +43,7 @@ class Config(C.Structure):
         ("c_std", C.c_double), ("objective", C.c_int32), ("seed", C.c_uint64), ("device", C.c_int32),
         ("stream", C.c_void_p), ("trace_rounds", C.c_int64), ("policy_K", C.c_int32), ("policy_R", C.c_int32), ("policy_rho_upper", C.c_double),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("storage", C.c_int32),
-        ("fuse_rounds", C.c_int32),
+        ("fuse_rounds", C.c_int32), ("first_round", C.c_int64),
     ]
 
 STORAGE = {"f32": 0, "bf16": 1}
@@ -171,7 +171,7 @@ class Netmax:
                  device: int = 0, stream: Optional[int] = None, trace_rounds: int = 1024, policy_K: int = 20,
                  policy_R: int = 20, workspace: Optional[int] = None, workspace_bytes: int = 0,
                  element_offset: int = 0, pull_weight: float = 0.0, policy_rho_upper: float = 0.0,
-                 storage: str = "f32", fuse_rounds: int = 0):
+                 storage: str = "f32", fuse_rounds: int = 0, first_round: int = 0):
         L = lib()
         cfg = Config()
         _check(L.netmax_config_init(C.byref(cfg)))
@@ -191,6 +191,8 @@ class Netmax:
         cfg.workspace, cfg.workspace_bytes = workspace, int(workspace_bytes)
         cfg.storage = STORAGE[storage]
         cfg.fuse_rounds = int(fuse_rounds)
+        cfg.first_round = int(first_round)
+        self.first_round = int(first_round)
         self.storage = storage
         self.M, self.d = int(M), int(d)
         self._h = C.c_void_p()
@@ -287,13 +289,15 @@ class Netmax:
         _check(lib().netmax_read_columns_static(self._h, _p(cols), cols.shape[0], _p(out)), self._h)
         return out
 
-    def peer_trace(self, first_round: int = 0, n: Optional[int] = None):
+    def peer_trace(self, first_round: Optional[int] = None, n: Optional[int] = None):
+        first_round = self.first_round if first_round is None else first_round
         n = self.rounds_done - first_round if n is None else n
         out = np.empty((n, self.M), dtype=np.int32)
         _check(lib().netmax_peer_trace(self._h, int(first_round), int(n), _p(out)), self._h)
         return out
 
-    def telemetry(self, first_round: int = 0, n: Optional[int] = None):
+    def telemetry(self, first_round: Optional[int] = None, n: Optional[int] = None):
+        first_round = self.first_round if first_round is None else first_round
         n = self.rounds_done - first_round if n is None else n
         cons = np.empty(n, dtype=np.float64)
         loss = np.empty(n, dtype=np.float64)

@@ -158,7 +158,8 @@ struct netmax_ctx {
   std::vector<double> ev_time;
   unsigned int* coltick = nullptr;
   int cur = 0;  // index of the buffer holding the current replicas
-  int64_t rounds = 0;
+  int64_t rounds = 0;  // number of the next round (absolute)
+  int64_t round0 = 0;  // number of the context's first round
   int64_t trace_rounds = 0;
   double alpha = 0, rho = 0, sigma = 0;
   double pull_weight = 0;  // > 0: fixed weight of every pull
@@ -687,6 +688,8 @@ static int check_sizes(const netmax_config* cfg) {
   if (cfg->trace_rounds < 1) return fail(nullptr, NETMAX_INVALID_ARG, "trace_rounds = %lld < 1", (long long)cfg->trace_rounds);
   if (cfg->fuse_rounds < 0 || cfg->fuse_rounds > kFusedMaxRounds)
     return fail(nullptr, NETMAX_INVALID_ARG, "fuse_rounds = %d outside [0, %d]", cfg->fuse_rounds, kFusedMaxRounds);
+  if (cfg->first_round < 0 || cfg->first_round >= ((int64_t)1 << 56))
+    return fail(nullptr, NETMAX_INVALID_ARG, "first_round = %lld outside [0, 2^56)", (long long)cfg->first_round);
   return NETMAX_OK;
 }
 
@@ -737,6 +740,7 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   ctx->keys = make_philox_keys(cfg->seed);
   ctx->storage = cfg->storage;
   ctx->fuse_rounds = cfg->fuse_rounds;
+  ctx->round0 = ctx->rounds = cfg->first_round;
   ctx->L = make_layout(cfg->M, cfg->d, cfg->trace_rounds, cfg->storage);
 
   rc = build_adjacency(ctx, cfg->M, cfg->link_speed_gbps, ctx->adj);
@@ -1233,7 +1237,7 @@ int netmax_read_columns_static(netmax_ctx* ctx, const int64_t* host_cols, int64_
 }
 
 static int ring_range(netmax_ctx* ctx, int64_t first, int64_t n) {
-  if (first < 0 || n < 0 || first + n > ctx->rounds || first < ctx->rounds - ctx->trace_rounds)
+  if (first < ctx->round0 || n < 0 || first + n > ctx->rounds || first < ctx->rounds - ctx->trace_rounds)
     return fail(ctx, NETMAX_TRACE_RANGE, "rounds [%lld, %lld) are not in the ring (rounds done %lld, capacity %lld)",
                 (long long)first, (long long)(first + n), (long long)ctx->rounds, (long long)ctx->trace_rounds);
   return NETMAX_OK;
@@ -1373,7 +1377,7 @@ static void async_start_iteration(netmax_ctx* ctx, int i, double start) {
 
 int netmax_async_begin(netmax_ctx* ctx, const double* t_iter, double beta) {
   if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
-  if (ctx->rounds != 0) return fail(ctx, NETMAX_INVALID_ARG, "netmax_async_begin must precede any netmax_round");
+  if (ctx->rounds != ctx->round0) return fail(ctx, NETMAX_INVALID_ARG, "netmax_async_begin must precede any netmax_round");
   if (!(beta >= 0.0 && beta < 1.0)) return fail(ctx, NETMAX_INVALID_ARG, "beta = %g outside [0, 1)", beta);
   const int32_t M = ctx->M;
   if (t_iter) {

@@ -65,7 +65,7 @@ def test_full_size_configs_on_sampled_columns(nm, idx):
     for epoch in range(w.n_epochs):
         s = w.link_speeds(epoch)
         t, adj = opolicy.iteration_times(s, w.d)
-        P, rho, _ = opolicy.generate_policy(t, adj, w.lr, w.K if idx != 4 else 4, w.R if idx != 4 else 4)
+        P, rho, _ = opolicy.generate_policy(t, adj, w.lr, w.K, w.R)
         if g is None:
             g = nm.Netmax(M=w.M, d=w.d, lr=w.lr, link_speed_gbps=s, prob=P, rho=rho, sigma=w.sigma,
                           x0_std=w.x0_std, c_std=w.c_std, objective=1, seed=w.seed, trace_rounds=w.rounds + 1)
@@ -95,7 +95,7 @@ def test_full_size_configs_on_sampled_columns(nm, idx):
 
 def test_full_size_sampling_stress_config(nm):
     w = workloads.config(5)
-    rounds = int(os.environ.get("NETMAX_CFG5_ROUNDS", "1000"))
+    rounds = int(os.environ.get("NETMAX_CFG5_ROUNDS", str(w.rounds)))     # all 10,000 rounds (about 200 s of oracle time)
     s = w.link_speeds(0)
     P = s / s.sum(axis=1, keepdims=True)      # dense heterogeneous rows: an input, not Algorithm 3
     cols = workloads.sample_columns(w.d, 40, w.seed)

@@ -335,3 +335,47 @@ def test_fixed_weight_ignores_rho_and_probabilities():
                 D[i, m] += 0.25
         x = (D @ x).astype(np.float32).astype(np.float64)
     np.testing.assert_allclose(sims[0].x(), x, atol=1e-6)
+
+
+def test_rounds_numbered_from_a_later_start_use_that_rounds_counters():
+    """A simulator that starts at round r0 draws the peers and the noise of rounds r0, r0 + 1, ...:
+    checked against the two pinned stream functions across the 2^32 boundary of the round word,
+    and against an uninterrupted run resumed half way."""
+    M, d, alpha, sigma, seed = 4, 12, 0.1, 0.3, 77
+    r0 = (1 << 32) - 3
+    P = random_policy(M, np.random.default_rng(3), self_prob=True)
+    rho = max_rho(P, alpha)
+    sim = oracle.Sim(M, d, P, full_adj(M), alpha=alpha, rho=rho, sigma=sigma, objective=1, seed=seed, first_round=r0)
+    sim.init(1.0, 1.0)
+    x0, c = sim.x().astype(np.float64), sim.c().astype(np.float64)
+    sim.round(6)
+    assert sim.rounds_done == 6
+    trace = sim.trace()
+    assert (trace == oracle.peer_draws(P, seed, r0, 6)).all()
+    assert not (trace == oracle.peer_draws(P, seed, 0, 6)).all()
+    # first round by hand: Eq. 15 with the noise of round r0, then Eq. 16 against the snapshot
+    a32, s32 = float(np.float32(alpha)), float(np.float32(sigma))
+    w = oracle.build_weights(P, full_adj(M), a32, rho).astype(np.float64)
+    one = oracle.Sim(M, d, P, full_adj(M), alpha=alpha, rho=rho, sigma=sigma, objective=1, seed=seed, first_round=r0)
+    one.init(1.0, 1.0)
+    one.round(1)
+    want = np.empty_like(x0)
+    for i in range(M):
+        z = oracle.noise(seed, i, r0, 0, d)
+        h = x0[i] - a32 * ((x0[i] - c[i]) + s32 * z)
+        m = int(trace[0, i])
+        want[i] = h if m == i else h - w[i, m] * (h - x0[m])
+    np.testing.assert_array_equal(one.x(), want.astype(np.float32))
+    # the initial state does not depend on where the rounds start
+    base = oracle.Sim(M, d, P, full_adj(M), alpha=alpha, rho=rho, sigma=sigma, objective=1, seed=seed)
+    base.init(1.0, 1.0)
+    np.testing.assert_array_equal(base.x(), x0.astype(np.float32))
+    # resume: 10 rounds from 0 == 4 rounds from 0, state handed over, 6 rounds numbered from 4
+    base.round(4)
+    rest = oracle.Sim(M, d, P, full_adj(M), alpha=alpha, rho=rho, sigma=sigma, objective=1, seed=seed, first_round=4)
+    rest.set_x(base.x())
+    rest.set_c(base.c())
+    base.round(6)
+    rest.round(6)
+    np.testing.assert_array_equal(rest.x(), base.x())
+    assert (rest.trace() == base.trace(4, 6)).all()
