@@ -40,24 +40,29 @@ import numpy as np  # noqa: E402
 
 from paper_2009_05766_b200 import workloads  # noqa: E402
 
-BYTES_PER_ELEMENT = 16          # x_i, x_peer, c_i read + x_i' written, fp32
+BYTES_PER_ELEMENT = 16          # x_i, x_peer, c_i read + x_i' written, fp32: the replica GB/s metric counts these
 BYTES_PER_ELEMENT_BF16 = 8      # the same four accesses with bfloat16 storage
+UNIQUE_FRACTION = 0.75          # x_peer is a row the same tile reads anyway (a cache hit by design): 12 of the 16
+                                # bytes (6 of 8) have to cross the DRAM pins, and the HBM roofline is taken against those
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
 KERNEL_SOURCES = ("netmax_kernels.cuh", "netmax_rng.cuh")
-# dram__bytes_read.sum + dram__bytes_write.sum of one round-kernel launch, from an ncu capture
-# (see profiles/); only reported while the kernel sources still hash to the value captured.
-NCU_TRAFFIC = {
-    ("f410b991e772e080", "cfg2_M8_resnet18"): 1_041_924_000,              # round_kernel: 8 B/element read, 3.65 written
-    ("f410b991e772e080", "cfg2_M8_resnet18/fused"): 1_041_056_000,        # fused_rounds_kernel, four rounds per launch
-    ("f410b991e772e080", "cfg2_M8_resnet18/bf16"): 505_763_000,
-    ("f410b991e772e080", "cfg2_M8_resnet18/bf16/fused"): 505_109_000,
-    ("f410b991e772e080", "cfg3_M16_vgg19scale/fused"): 3_806_318_000,
-}
-# smsp__inst_executed.sum of one launch / (elements x rounds of the launch), from the same captures
-NCU_WARP_INST_PER_ELEMENT_ROUND = {
-    ("f410b991e772e080", "cfg2_M8_resnet18/fused"): 346_883_835 / (89_391_696 * 4),
-    ("f410b991e772e080", "cfg2_M8_resnet18/bf16/fused"): 383_985_067 / (89_391_696 * 4),
-    ("f410b991e772e080", "cfg3_M16_vgg19scale/fused"): 1_183_131_797 / (320_000_000 * 4),
+# Counters of one launch, from ncu captures of this file's own commands (see profiles/): DRAM bytes
+# (dram__bytes_read.sum + dram__bytes_write.sum) per element of the launch and warp instructions
+# (smsp__inst_executed.sum) per element and round.  Captured on the workload itself where that is small
+# enough to profile, else on the same M and tile shape with a shorter vector (`captured_on`); bytes and
+# instructions per element are what carries over.  Only reported while the kernel sources still hash to
+# the value the capture was taken at.
+NCU_HASH = "f410b991e772e080"
+NCU_COUNTERS = {
+    # (workload tag, kernel): dram bytes per element-launch, warp instructions per element-round, captured on
+    ("cfg2_M8_resnet18", "round_kernel"): (1_041_924_000 / 89_391_696, None, "cfg2"),
+    ("cfg2_M8_resnet18", "fused_rounds_kernel"): (1_041_056_000 / 89_391_696, 346_883_835 / (89_391_696 * 4), "cfg2"),
+    ("cfg2_M8_resnet18/bf16", "round_kernel"): (505_763_000 / 89_391_696, None, "cfg2"),
+    ("cfg2_M8_resnet18/bf16", "fused_rounds_kernel"): (505_109_000 / 89_391_696, 383_985_067 / (89_391_696 * 4), "cfg2"),
+    ("cfg3_M16_vgg19scale", "fused_rounds_kernel"): (3_806_318_000 / 320_000_000, 1_183_131_797 / (320_000_000 * 4), "cfg3"),
+    ("cfg3_M16_vgg19scale", "round_kernel"): (1_543_900_928 / (16 * 8_000_002), 105_887_357 / (16 * 8_000_002), "cfg3 at d = 8,000,002"),
+    ("cfg4_M64_resnet18", "round_kernel"): (1_532_370_688 / (64 * 2_000_002), 108_627_174 / (64 * 2_000_002), "cfg4 at d = 2,000,002"),
 }
 SM_COUNT, SCHEDULERS_PER_SM = 148, 4     # one warp instruction per scheduler and clock at most
 
@@ -229,6 +234,125 @@ def shard_plan(d: int, world: int, rank: int, align: int = 4):
     return {"element_offset": rank * d4, "d": d, "global_d": world * d4}
 
 
+def counters_for(tag: str, kernel: str):
+    """(dram bytes per element-launch, warp instructions per element-round, captured_on) or Nones."""
+    if kernel_source_hash() != NCU_HASH:
+        return None, None, None
+    return NCU_COUNTERS.get((tag, kernel), (None, None, None))
+
+
+def hbm_roofline(tag, kernel, ms_per_round, elements, bpe, peak, peak_kind):
+    """HBM-bound launch (one round per launch): achieved = the bytes that must cross the DRAM pins
+    (12 of the 16 per element: the peer read is a cache hit by design) / time, against the measured
+    copy peak; the DRAM bytes ncu counted for the same launch and the 16-byte metric ride along."""
+    sec = ms_per_round / 1e3
+    unique = UNIQUE_FRACTION * bpe * elements
+    per_el, _, captured_on = counters_for(tag, kernel)
+    traffic = None if per_el is None else per_el * elements
+    out = {"bound": "hbm", "achieved": unique / sec / 1e9, "peak": peak, "unit": "GB/s",
+           "frac": unique / sec / 1e9 / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": kernel,
+           "bytes_per_launch": unique, "algorithmic_bytes_per_element": UNIQUE_FRACTION * bpe,
+           "replica_GBs": bpe * elements / sec / 1e9}
+    if traffic is not None:
+        out.update({"dram_GBs": traffic / sec / 1e9, "dram_frac_of_measured": traffic / sec / 1e9 / peak,
+                    "dram_frac_of_8TBs": traffic / sec / 1e9 / NOMINAL_HBM_GBS, "traffic_captured_on": captured_on})
+    return out
+
+
+def issue_roofline(tag, kernel, ms_per_round, elements, bpe, rounds_per_launch, sm_max_mhz, peak, peak_kind):
+    """Launches that keep a tile on chip for several rounds are bound by instruction issue:
+    achieved = warp instructions per second (ncu count per element and round x elements / time)
+    against 148 SMs x 4 schedulers x 1 warp instruction per clock at clocks.max.sm."""
+    sec = ms_per_round / 1e3
+    per_el, ipe, captured_on = counters_for(tag, kernel)
+    alu_peak = SM_COUNT * SCHEDULERS_PER_SM * (sm_max_mhz or 1965) / 1e3           # G warp instructions / s
+    achieved = None if ipe is None else ipe * elements / sec / 1e9
+    traffic = None if per_el is None else per_el * elements                         # per launch of rounds_per_launch rounds
+    out = {"bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "Gwarp-inst/s",
+           "frac": None if achieved is None else achieved / alu_peak, "traffic": traffic,
+           "peak_kind": "148 SMs x 4 schedulers x 1 warp instruction per clock x clocks.max.sm", "kernel": kernel,
+           "rounds_per_launch": rounds_per_launch, "warp_inst_per_element_round": ipe,
+           "bytes_per_launch": UNIQUE_FRACTION * bpe * elements,
+           "replica_GBs": bpe * elements / sec / 1e9, "hbm_peak": peak, "hbm_peak_kind": f"of {peak_kind}"}
+    if traffic is not None:
+        dram = traffic / (sec * rounds_per_launch) / 1e9
+        out.update({"dram_GBs": dram, "dram_frac_of_measured": dram / peak, "dram_frac_of_8TBs": dram / NOMINAL_HBM_GBS,
+                    "traffic_captured_on": captured_on})
+    return out
+
+
+class Timer:
+    """CUDA-event timing of netmax_round on the context's stream."""
+
+    def __init__(self, torch, stream, barrier):
+        self.torch, self.stream, self.barrier = torch, stream, barrier
+        self.start = torch.cuda.Event(enable_timing=True)
+        self.stop = torch.cuda.Event(enable_timing=True)
+
+    def rounds(self, g, n):
+        self.barrier()
+        with self.torch.cuda.stream(self.stream):
+            self.start.record()
+        g.round(n)
+        with self.torch.cuda.stream(self.stream):
+            self.stop.record()
+        self.stop.synchronize()
+        return self.start.elapsed_time(self.stop)
+
+    def repeats(self, g, n, reps=5):
+        return [self.rounds(g, n) / n for _ in range(reps)]
+
+
+def launch_shape(g, rounds, ring):
+    """Names the launch shape netmax_round chose, from the number of launches `rounds` rounds took."""
+    before = g.kernel_launches
+    g.round(rounds)
+    per = rounds / max(1, g.kernel_launches - before - (rounds + ring - 1) // ring)      # sampler launches excluded
+    if per > 4.5:
+        return "all rounds of a call on shared-memory-resident columns", "resident_rounds_kernel", per
+    if per > 1.5:
+        return "%d rounds per launch over resident tiles" % round(per), "fused_rounds_kernel", per
+    return "one launch per round", "round_kernel", per
+
+
+def measure_config(torch, binding, wk, args, local, timer, peak, peak_kind, sm_max_mhz):
+    """One entry of the line's `configs`: the workload in the launch shape the library picks (and, where
+    that fuses rounds, one launch per round as well), timed over at least 200 rounds per repeat."""
+    speeds = wk.link_speeds(0)
+    t_iter, adj = binding.netmax_iteration_times(speeds, wk.d)
+    generate = binding.netmax_policy_generate_device if wk.M >= 512 else binding.netmax_policy_generate
+    P, rho, _ = generate(t_iter, adj, wk.lr, wk.K, wk.R)
+    bf16 = args.storage == "bf16"
+    bpe = BYTES_PER_ELEMENT_BF16 if bf16 else BYTES_PER_ELEMENT
+    ring = 1024
+    g = binding.Netmax(M=wk.M, d=wk.d, lr=wk.lr, link_speed_gbps=speeds, prob=P, rho=rho, sigma=wk.sigma,
+                       x0_std=wk.x0_std, c_std=wk.c_std, objective=1, seed=wk.seed, device=local,
+                       stream=timer.stream.cuda_stream, trace_rounds=ring, storage=args.storage)
+    elements = wk.M * wk.d
+    tag = wk.name + ("/bf16" if bf16 else "")
+    rounds = 200 if elements > 1 << 22 else 2000
+    shape, kernel, per = launch_shape(g, 20, ring)
+    g.round(20)
+    ms = timer.repeats(g, rounds, 3)
+    best = min(ms)
+    entry = {"M": wk.M, "d": wk.d, "launch_shape": shape, "rounds_timed": rounds, "ms_per_round": best,
+             "ms_per_round_median": statistics.median(ms), "rounds_per_s": 1e3 / best,
+             "replica_GBs": bpe * elements / (best / 1e3) / 1e9, "peer_draws_per_s": wk.M * 1e3 / best}
+    if kernel == "round_kernel":
+        entry["roofline"] = hbm_roofline(tag, kernel, best, elements, bpe, peak, peak_kind)
+    else:
+        entry["roofline"] = issue_roofline(tag, kernel, best, elements, bpe, per, sm_max_mhz, peak, peak_kind)
+    if kernel == "fused_rounds_kernel":
+        g.set_fuse_rounds(1)
+        g.round(20)
+        one = min(timer.repeats(g, rounds, 3))
+        entry["one_launch_per_round"] = {"ms_per_round": one,
+                                         "roofline": hbm_roofline(tag, "round_kernel", one, elements, bpe, peak, peak_kind)}
+    g.close()
+    torch.cuda.empty_cache()
+    return entry
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -277,21 +401,19 @@ def run_ours(args, w):
         torch.cuda.synchronize()
 
     elements = w.M * w.d
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    timer = Timer(torch, stream, barrier)
+    start, stop = timer.start, timer.stop
 
     g.round(args.warmup)
     barrier()
     launches0 = g.kernel_launches
     with ClockSampler(local) as clocks:
-        with torch.cuda.stream(stream):
-            start.record()
-        g.round(args.steps)
-        with torch.cuda.stream(stream):
-            stop.record()
-        stop.synchronize()
-    barrier()
-    launches = g.kernel_launches - launches0
-    ms = start.elapsed_time(stop)
+        ms = timer.rounds(g, args.steps)                      # the contract's timed region: exactly K steps
+        launches = g.kernel_launches - launches0
+        barrier()
+        # repeats of a run long enough to time well (at least 200 rounds each): best and median per round
+        rep_rounds = max(200, min(args.steps, 2000)) if elements > 1 << 22 else max(2000, args.steps)
+        rep_ms = timer.repeats(g, rep_rounds)
     if world > 1:
         tmax = torch.tensor([ms], device="cuda", dtype=torch.float64)
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
@@ -299,30 +421,14 @@ def run_ours(args, w):
     sec = ms / 1e3
     value = bytes_per_element * elements * world * args.steps / sec / 1e9
 
-    # five more untimed-by-the-contract repeats of a shorter run: best and median per round
-    rep_rounds = max(1, min(args.steps, 200))
-
-    def repeats():
-        out = []
-        for _ in range(5):
-            barrier()
-            with torch.cuda.stream(stream):
-                start.record()
-            g.round(rep_rounds)
-            with torch.cuda.stream(stream):
-                stop.record()
-            stop.synchronize()
-            out.append(start.elapsed_time(stop) / rep_rounds)
-        return out
-
-    rep_ms = repeats()
     rounds_per_launch = args.steps / max(1, launches - (args.steps + ring - 1) // ring)   # sampler launches excluded
-    fused = 1.5 < rounds_per_launch <= 4.5      # (short vectors run thousands of rounds per cooperative launch)
+    fused = 1.5 < rounds_per_launch <= 4.5
+    resident = rounds_per_launch > 4.5      # short vectors: all rounds of a call on resident columns
     single_ms = None
     if fused:                       # the same rounds, one launch each: the HBM-bound kernel
         g.set_fuse_rounds(1)
         g.round(args.warmup)
-        single_ms = repeats()
+        single_ms = timer.repeats(g, rep_rounds)
         g.set_fuse_rounds(args.fuse_rounds)
 
     # end to end through the C ABI with host buffers: upload x and c, one round, download x'
@@ -358,6 +464,7 @@ def run_ours(args, w):
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         e2e_ms = float(tmax.item())
     e2e_value = bytes_per_element * elements * world * e2e_steps / (e2e_ms / 1e3) / 1e9
+    del hx, hc, ho
 
     # the sampler alone: one batched launch of 1024 rounds x M draws (Algorithm 2's peer selection)
     batch = 1024
@@ -376,36 +483,25 @@ def run_ours(args, w):
 
     cons, loss = g.telemetry(g.rounds_done - 1, 1)
     peak, peak_kind = measured_peak()
-    per_launch_ms = ms / args.steps
-    achieved = bytes_per_element * elements / (per_launch_ms / 1e3) / 1e9
+    per_round_ms = ms / args.steps
     tag = w.name + ("/bf16" if bf16 else "")
-    khash = kernel_source_hash()
-    if fused:
-        # several rounds per launch over a resident tile: bound by instruction issue
-        ipe = NCU_WARP_INST_PER_ELEMENT_ROUND.get((khash, tag + "/fused"))
-        sm_max_ghz = (clocks.summary()["sm_max_mhz"] or 1965) / 1e3
-        alu_peak = SM_COUNT * SCHEDULERS_PER_SM * sm_max_ghz           # G warp instructions / s
-        alu_achieved = None if ipe is None else ipe * elements / (per_launch_ms / 1e3) / 1e9
-        roofline = {"bound": "alu", "achieved": alu_achieved, "peak": alu_peak, "unit": "Gwarp-inst/s",
-                    "frac": None if alu_achieved is None else alu_achieved / alu_peak,
-                    "traffic": NCU_TRAFFIC.get((khash, tag + "/fused")),
-                    "peak_kind": "148 SMs x 4 schedulers x 1 warp instruction per clock x clocks.max.sm",
-                    "kernel": "fused_rounds_kernel", "rounds_per_launch": rounds_per_launch,
-                    "warp_inst_per_element_round": ipe,
-                    "bytes_per_launch": bytes_per_element * elements * rounds_per_launch,
-                    "replica_GBs_over_hbm_peak": achieved / peak, "hbm_peak": peak, "hbm_peak_kind": f"of {peak_kind}"}
+    sm_max_mhz = clocks.summary()["sm_max_mhz"]
+    if fused or resident:
+        kernel = "fused_rounds_kernel" if fused else ("multi_round_kernel" if args.fuse_rounds == 1 else "resident_rounds_kernel")
+        roofline = issue_roofline(tag, kernel, per_round_ms, elements, bytes_per_element, rounds_per_launch, sm_max_mhz,
+                                  peak, peak_kind)
     else:
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "traffic": NCU_TRAFFIC.get((khash, tag)), "peak_kind": f"of {peak_kind}", "kernel": "round_kernel",
-                    "bytes_per_launch": bytes_per_element * elements, "frac_of_nominal_8TBs": achieved / 8000.0}
+        roofline = hbm_roofline(tag, "round_kernel", per_round_ms, elements, bytes_per_element, peak, peak_kind)
     line = {
         "metric": "replica GB/s", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": per_launch_ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "warmup": args.warmup, "ms_per_step": per_round_ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 storage, f32 arithmetic" if bf16 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "M": w.M, "d_per_gpu": w.d, "global_d": plan["global_d"], "lr": w.lr,
                    "sigma": w.sigma, "policy": f"Algorithm 3, K={w.K}, R={w.R}, rho={rho:.6g}",
                    "sharding": "columns, no exchange" if world > 1 else "none", "storage": args.storage,
                    "l2": "inputs larger than L2: each of x, x', c is %.0f MB" % (elements * bytes_per_element / 4 / 1e6)},
+        "metric_definition": "replica GB/s = 16 bytes (x_i, x_peer, c_i read; x_i' written) x M x d x rounds / time; "
+                             "`roofline` holds the fraction of the bound that applies and the DRAM rate from ncu's counters",
         "repeats": {"rounds_each": rep_rounds, "ms_per_step_best": min(rep_ms),
                     "ms_per_step_median": statistics.median(rep_ms)},
         "hbm_footprint_bytes": int(size),
@@ -422,16 +518,39 @@ def run_ours(args, w):
                          "(ResNet18, 8x RTX 2080 Ti, throttled 1 GbE); not comparable to this metric",
     }
     if single_ms is not None:
-        one = bytes_per_element * elements / (min(single_ms) / 1e3) / 1e9
         line["one_launch_per_round"] = {
             "ms_per_step_best": min(single_ms), "ms_per_step_median": statistics.median(single_ms),
-            "roofline": {"bound": "hbm", "achieved": one, "peak": peak, "unit": "GB/s", "frac": one / peak,
-                         "traffic": NCU_TRAFFIC.get((khash, tag)), "peak_kind": f"of {peak_kind}",
-                         "kernel": "round_kernel", "bytes_per_launch": bytes_per_element * elements,
-                         "frac_of_nominal_8TBs": one / 8000.0}}
+            "roofline": hbm_roofline(tag, "round_kernel", min(single_ms), elements, bytes_per_element, peak, peak_kind)}
     if base is not None:
         line["cpu_baseline"] = base
     g.close()
+    del ws
+    torch.cuda.empty_cache()
+    if world == 1 and args.configs != "none" and args.d == 0:
+        # every config of the benchmark description in the same process (the headline's own numbers are reused)
+        which = [1, 2, 3, 4, 5] if args.configs == "all" else [int(c) for c in args.configs.split(",")]
+        configs = {}
+        for idx in which:
+            wk = workloads.config(idx)
+            if wk.name == w.name:
+                entry = {"M": w.M, "d": w.d, "launch_shape": "headline (see the top-level keys)",
+                         "rounds_timed": rep_rounds, "ms_per_round": min(rep_ms),
+                         "ms_per_round_median": statistics.median(rep_ms), "rounds_per_s": 1e3 / min(rep_ms),
+                         "replica_GBs": bytes_per_element * elements / (min(rep_ms) / 1e3) / 1e9,
+                         "peer_draws_per_s": w.M * 1e3 / min(rep_ms)}
+                entry["roofline"] = (issue_roofline(tag, kernel, min(rep_ms), elements, bytes_per_element, rounds_per_launch,
+                                                    sm_max_mhz, peak, peak_kind) if (fused or resident) else
+                                     hbm_roofline(tag, "round_kernel", min(rep_ms), elements, bytes_per_element, peak, peak_kind))
+                if single_ms is not None:
+                    entry["one_launch_per_round"] = {"ms_per_round": min(single_ms),
+                                                     "roofline": line["one_launch_per_round"]["roofline"]}
+                configs["cfg%d" % idx] = entry
+                continue
+            with ClockSampler(local) as ck:
+                entry = measure_config(torch, binding, wk, args, local, timer, peak, peak_kind, sm_max_mhz)
+            entry["clocks"] = ck.summary()
+            configs["cfg%d" % idx] = entry
+        line["configs"] = configs
     if world > 1:
         dist.destroy_process_group()
     if rank == 0:
@@ -503,6 +622,8 @@ def main():
     ap.add_argument("--d", type=int, default=0, help="override the workload's vector length (profiling on a smaller case)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--configs", default="all",
+                    help="one GPU: which of cfg1..cfg5 to time into the line's `configs` (all, none, or e.g. 3,4)")
     ap.add_argument("--fuse-rounds", type=int, default=0,
                     help="rounds per launch over a resident tile: 0 automatic, 1 one launch per round, 2..4")
     ap.add_argument("--storage", choices=["f32", "bf16"], default="f32",

@@ -343,6 +343,32 @@ int netmax_policy_generate_ex(int32_t M, const double* t_iter, const uint8_t* ad
                               double rho_upper, double* prob_out, double* rho_out, double* info_out);
 
 /*
+ * Algorithm 3 for a pull rule with a CONSTANT weight w (netmax_config.pull_weight): the paper's
+ * section on extending existing decentralised PSGD approaches (gossip / AD-PSGD style averaging,
+ * x_i <- (1 - w)(x_i - alpha g_i) + w x_m) asks for two steps.  First, Eq. 11 is replaced by the
+ * condition that every entry y_im of E[D^T D] on a link is positive; with a constant weight
+ * y_im = (w - w^2)(p_i p_im + p_m p_mi), so the condition is p_im + p_mi > 0, taken here as a floor
+ * phi on both directions of every link.  Second, the optimisation problem (Eq. 8-13) is solved
+ * again: phi takes rho's place in the outer loop (phi_k = k floor_upper / K; floor_upper <= 0: the
+ * value at which the floors alone fill a row), t_bar is searched in the inner loop (the midpoints of R
+ * cells between the least and the largest mean time the floors allow), and the grid
+ * point minimising t_bar ln(eps) / ln(lambda_2) is kept.  Y_P is doubly stochastic only if, besides
+ * Eq. 10, the columns of P sum to 1, which couples the rows; among the feasible P with p_ii = 0 the
+ * one of maximum entropy above the floors is returned (rows, columns and mean iteration times are
+ * met to 1e-9).  The link graph must be symmetric.  Host arrays; info_out as in
+ * netmax_policy_generate; *floor_out receives the selected phi.
+ */
+int netmax_policy_generate_fixed_weight(int32_t M, const double* t_iter, const uint8_t* adj, double pull_weight, int32_t K,
+                                        int32_t R, double floor_upper, double* prob_out, double* floor_out,
+                                        double* info_out /* 5 doubles or NULL */);
+
+/* One grid point of the search above: the maximum-entropy P with p_im >= floor on every link, zero
+ * diagonal, rows and columns summing to 1 and a mean iteration time of M t_bar in every row (Eq. 10);
+ * NETMAX_INFEASIBLE if there is none.  Host arrays; prob_out is M*M. */
+int netmax_policy_fixed_weight_at(int32_t M, const double* t_iter, const uint8_t* adj, double floor, double t_bar,
+                                  double* prob_out);
+
+/*
  * Algorithm 3 on the GPU, for large M (thousands of workers, links redrawn often): the same
  * grids, the same row-wise LP optimum and the same selection as netmax_policy_generate, with
  * one CTA per row of P, Y_P (Eq. 22) kept in device memory and lambda_2 by Lanczos on the

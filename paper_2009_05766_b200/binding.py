@@ -26,7 +26,7 @@ EXPORTS = [
     "netmax_peer_trace", "netmax_telemetry", "netmax_replicas_device", "netmax_sample_peers",
     "netmax_measure", "netmax_async_begin", "netmax_async_set_times", "netmax_async_steps", "netmax_async_time",
     "netmax_async_trace", "netmax_async_ema", "netmax_async_monitor", "netmax_async_monitor_refreshes",
-    "netmax_iteration_times", "netmax_policy_generate", "netmax_policy_generate_ex", "netmax_policy_generate_device", "netmax_debug_absent_ctas", "netmax_kernel_launches", "netmax_last_error",
+    "netmax_iteration_times", "netmax_policy_generate", "netmax_policy_generate_ex", "netmax_policy_generate_device", "netmax_policy_generate_fixed_weight", "netmax_policy_fixed_weight_at", "netmax_debug_absent_ctas", "netmax_kernel_launches", "netmax_last_error",
 ]
 
 
@@ -99,6 +99,8 @@ def lib():
             "netmax_policy_generate": ([i32, vp, vp, dbl, i32, i32, vp, vp, vp], C.c_int),
             "netmax_policy_generate_ex": ([i32, vp, vp, dbl, i32, i32, dbl, vp, vp, vp], C.c_int),
             "netmax_policy_generate_device": ([i32, vp, vp, dbl, i32, i32, dbl, i32, vp, vp, vp, vp], C.c_int),
+            "netmax_policy_generate_fixed_weight": ([i32, vp, vp, dbl, i32, i32, dbl, vp, vp, vp], C.c_int),
+            "netmax_policy_fixed_weight_at": ([i32, vp, vp, dbl, dbl, vp], C.c_int),
             "netmax_debug_absent_ctas": ([vp, i32], C.c_int),
             "netmax_kernel_launches": ([vp], i64),
             "netmax_last_error": ([vp], C.c_char_p),
@@ -148,6 +150,27 @@ def netmax_policy_generate(t_iter, adj, lr: float, K: int, R: int, rho_upper: fl
     _check(lib().netmax_policy_generate_ex(M, _p(t), _p(adj), float(lr), int(K), int(R), float(rho_upper), _p(P),
                                            C.byref(rho), _p(info)))
     return P, rho.value, dict(lam2=info[0], tbar=info[1], t_conv=info[2], k=int(info[3]), r=int(info[4]))
+
+
+def netmax_policy_generate_fixed_weight(t_iter, adj, pull_weight: float, K: int, R: int, floor_upper: float = 0.0):
+    t = _f64(t_iter)
+    M = t.shape[0]
+    adj = np.ascontiguousarray(adj, dtype=np.uint8)
+    P = np.empty((M, M), dtype=np.float64)
+    floor = C.c_double()
+    info = np.empty(5, dtype=np.float64)
+    _check(lib().netmax_policy_generate_fixed_weight(M, _p(t), _p(adj), float(pull_weight), int(K), int(R), float(floor_upper),
+                                                     _p(P), C.byref(floor), _p(info)))
+    return P, floor.value, dict(lam2=info[0], tbar=info[1], t_conv=info[2], k=int(info[3]), r=int(info[4]))
+
+
+def netmax_policy_fixed_weight_at(t_iter, adj, floor: float, t_bar: float):
+    t = _f64(t_iter)
+    M = t.shape[0]
+    adj = np.ascontiguousarray(adj, dtype=np.uint8)
+    P = np.empty((M, M), dtype=np.float64)
+    _check(lib().netmax_policy_fixed_weight_at(M, _p(t), _p(adj), float(floor), float(t_bar), _p(P)))
+    return P
 
 
 def netmax_policy_generate_device(t_iter, adj, lr: float, K: int, R: int, device: int = 0, stream=None,

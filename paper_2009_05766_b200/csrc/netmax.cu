@@ -471,6 +471,11 @@ ResidentKernel pick_resident_kernel(int objective, int halves) {
   return objective == 1 ? resident_rounds_kernel<1, true, false> : resident_rounds_kernel<0, true, false>;
 }
 
+// The kernels' noise scale: sigma (at its fp32 rounding, the value the update is defined with)
+// times the constant factor sqrt(2 ln 2) of the Box-Muller radius, which the fast normal generator
+// leaves out, rounded once to fp32.
+float noise_scale(const netmax_ctx* ctx) { return (float)((double)(float)ctx->sigma * kNormalScale); }
+
 int floor_pow2(int64_t v) {
   int r = 1;
   while ((int64_t)r * 2 <= v) r *= 2;
@@ -614,7 +619,7 @@ int plan_fused_uncached(netmax_ctx* ctx, const RoundPlan& plan, FusedPlan& f) {
   f = FusedPlan();
   if (ctx->fuse_rounds == 1 || plan.short_vectors) return NETMAX_OK;
   const int64_t M = ctx->M;
-  const size_t head = align_up((size_t)kFusedMaxRounds * M * 8, 128);
+  const size_t head = align_up((size_t)kFusedMaxRounds * M * 16, 128);
   const size_t fixed = head + 64 * sizeof(double);
   // 256 or 128 threads per CTA (a multiple of four warps keeps the SM's four schedulers evenly
   // loaded: 3 x 96 threads measured 587 us per cfg3 round against 508 for 2 x 128), whichever
@@ -989,7 +994,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   p.colpart = ctx->colpart;
   p.coltick = ctx->coltick;
   p.alpha = (float)ctx->alpha;
-  p.sigma = (float)ctx->sigma;
+  p.sigma = noise_scale(ctx);
   p.inv_M = 1.0f / (float)ctx->M;
   p.q_offset = ctx->q_offset;
   p.keys = ctx->keys;
@@ -1475,7 +1480,7 @@ int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps) {
   p.row_bytes = (uint32_t)(ctx->L.ld * ctx->L.elem);
   p.tail = (int32_t)(ctx->d % (4 * ctx->L.halves));
   p.alpha = (float)ctx->alpha;
-  p.sigma = (float)ctx->sigma;
+  p.sigma = noise_scale(ctx);
   p.q_offset = ctx->q_offset;
   p.n_events = 0;
   p.keys = ctx->keys;

@@ -15,6 +15,7 @@
 // rounded once, to the nearest bfloat16 (ties to even), at the store.
 #pragma once
 #include <cstdint>
+#include <type_traits>
 #include <cuda_runtime.h>
 
 #include "netmax_rng.cuh"
@@ -79,7 +80,7 @@ struct RoundParams {
   int32_t rows_per_group;  // ceil(M / rg)
   float4* colpart;       // rg > 1: per tile, per column group, per half: (sum, sum of squares) partials
   unsigned int* coltick; // rg > 1: arrivals per column tile (0 between launches)
-  float alpha, sigma;
+  float alpha, sigma;    // sigma: the noise scale sigma sqrt(2 ln 2) (see update_core_rnd)
   float inv_M;
   uint32_t round_lo, ctr3;
   uint32_t q_offset;     // Philox block index (element / 4) of the context's first element in the global vector
@@ -123,15 +124,73 @@ __device__ __forceinline__ int live_lanes(bool ragged, int tail, int h) {
   return ragged ? min(4, max(0, tail - 4 * h)) : 4;
 }
 
+// Per-lane noise scale of one column group (fused_rounds_kernel): sigma_s on real elements, 0 on the padding lanes of a
+// row's last, ragged group.  Padding lanes hold x = c = 0 in every row; with no noise Eq. 15-16
+// keep them at exactly +0 (every product and sum below is +0 or -0 + +0), so nothing has to be
+// masked after the update.
+struct NoiseLanes {
+  pair_t a, b;
+};
+__device__ __forceinline__ NoiseLanes noise_lanes(float sigma_s, int live) {
+  NoiseLanes n;
+  n.a = pack2(live > 0 ? sigma_s : 0.0f, live > 1 ? sigma_s : 0.0f);
+  n.b = pack2(live > 2 ? sigma_s : 0.0f, live > 3 ? sigma_s : 0.0f);
+  return n;
+}
+
 // Eq. 15 and Eq. 16 on one column group of one worker, on packed fp32 pairs:
 //   g = (x - c) + sigma z,  h = x - alpha g                                       (Eq. 15)
 //   x' = h - w (h - x_m),   w = alpha rho gamma_im  (w = 0 on a self-draw)          (Eq. 16)
-// q32 is the global index of the four elements' Philox block (first counter word), iter_lo /
-// ctr3 carry the round (or, on the asynchronous timeline, the worker's local iteration); `live`
-// is the number of real elements among the four (4 except in the last group of a row, whose
-// padding lanes must stay zero).  ta, tb return x - c for the caller's loss statistic.
+// rnd is the Philox block of the four elements (counter: global index of the block, worker,
+// round or -- on the asynchronous timeline -- the worker's local iteration); ns holds, per lane,
+// sigma sqrt(2 ln 2), the noise scale with the constant factor of the Box-Muller radius folded in
+// (fast path; the accurate path takes it out again), or 0 on padding lanes; nw2 is (-w, -w).
+// ta, tb return x - c for the caller's loss statistic.
 template <int kObjective, bool kFastNoise>
-__device__ __forceinline__ ulonglong2 update_core(float alpha, float sigma, const PhiloxKeys& keys,
+__device__ __forceinline__ ulonglong2 update_core_rnd(float alpha, const NoiseLanes& ns, uint4 rnd, ulonglong2 xv, ulonglong2 cv,
+                                                      ulonglong2 xm, pair_t nw2, pair_t& ta, pair_t& tb) {
+  const pair_t neg1 = pack2(-1.0f, -1.0f);
+  ta = fma2(cv.x, neg1, xv.x);  // x - c
+  tb = fma2(cv.y, neg1, xv.y);
+  pair_t ha = xv.x, hb = xv.y;
+  if (kObjective == 1) {
+    const pair_t nalpha2 = pack2(-alpha, -alpha);
+    pair_t za, zb, sa = ns.a, sb = ns.b;
+    if (kFastNoise) {
+      za = normal_pair_fast_unscaled(rnd.x, rnd.y);
+      zb = normal_pair_fast_unscaled(rnd.z, rnd.w);
+    } else {
+      const pair_t inv = pack2((float)(1.0 / kNormalScale), (float)(1.0 / kNormalScale));
+      sa = mul2(sa, inv);
+      sb = mul2(sb, inv);
+      const float4 z = normals4<false>(rnd);
+      za = pack2(z.x, z.y);
+      zb = pack2(z.z, z.w);
+    }
+    ha = fma2(nalpha2, fma2(sa, za, ta), xv.x);
+    hb = fma2(nalpha2, fma2(sb, zb, tb), xv.y);
+  }
+  const pair_t oa = fma2(nw2, fma2(xm.x, neg1, ha), ha);
+  const pair_t ob = fma2(nw2, fma2(xm.y, neg1, hb), hb);
+  return make_ulonglong2(oa, ob);
+}
+
+// The Philox block of the noise of one column group of one worker (only drawn when there is noise).
+template <int kObjective>
+__device__ __forceinline__ uint4 noise_block(const PhiloxKeys& keys, uint32_t iter_lo, uint32_t ctr3, uint32_t q32, uint32_t worker) {
+  if (kObjective != 1) return make_uint4(0u, 0u, 0u, 0u);
+  return philox4x32_10(q32, worker, iter_lo, ctr3, keys);
+}
+
+// The same update with the Philox block drawn inside, for the kernels that stream rows through
+// registers (round_kernel, step_kernel) or walk them one at a time (resident_rounds_kernel).  One
+// noise scale serves all four lanes and the padding lanes of a ragged group (`live` < 4 real
+// elements) are cleared after the update: the streaming kernel runs at its register limit, and
+// this form -- one scale pair instead of NoiseLanes' two, the masking behind a branch that is
+// almost never taken -- measured 191 us per round against 223 on 8 x 11.2 M elements.  Real lanes
+// see exactly the arithmetic of update_core_rnd, so all kernels agree bit for bit.
+template <int kObjective, bool kFastNoise>
+__device__ __forceinline__ ulonglong2 update_core(float alpha, float sigma_s, const PhiloxKeys& keys,
                                                   uint32_t iter_lo, uint32_t ctr3, uint32_t q32, uint32_t worker,
                                                   ulonglong2 xv, ulonglong2 cv, ulonglong2 xm, float w, int live,
                                                   pair_t& ta, pair_t& tb) {
@@ -141,14 +200,15 @@ __device__ __forceinline__ ulonglong2 update_core(float alpha, float sigma, cons
   tb = fma2(cv.y, neg1, xv.y);
   pair_t ha = xv.x, hb = xv.y;
   if (kObjective == 1) {
-    const pair_t sig2 = pack2(sigma, sigma);
+    pair_t sig2 = pack2(sigma_s, sigma_s);
     const pair_t nalpha2 = pack2(-alpha, -alpha);
     const uint4 rnd = philox4x32_10(q32, worker, iter_lo, ctr3, keys);
     pair_t za, zb;
     if (kFastNoise) {
-      za = normal_pair_fast_packed(rnd.x, rnd.y);
-      zb = normal_pair_fast_packed(rnd.z, rnd.w);
+      za = normal_pair_fast_unscaled(rnd.x, rnd.y);
+      zb = normal_pair_fast_unscaled(rnd.z, rnd.w);
     } else {
+      sig2 = mul2(sig2, pack2((float)(1.0 / kNormalScale), (float)(1.0 / kNormalScale)));
       const float4 z = normals4<false>(rnd);
       za = pack2(z.x, z.y);
       zb = pack2(z.z, z.w);
@@ -173,7 +233,29 @@ __device__ __forceinline__ ulonglong2 update_core(float alpha, float sigma, cons
 
 // update_core plus the telemetry sums of the round-start values.  kObjective == 2 measures only.
 template <int kObjective, bool kFastNoise>
-__device__ __forceinline__ ulonglong2 row_update(float alpha, float sigma, const PhiloxKeys& keys, uint32_t round_lo,
+__device__ __forceinline__ ulonglong2 row_update_rnd(float alpha, const NoiseLanes& ns, uint4 rnd, ulonglong2 xv, ulonglong2 cv,
+                                                     ulonglong2 xm, ulonglong2 pivot, pair_t nw2, ColAcc& acc, LossAcc& lacc) {
+  const pair_t neg1 = pack2(-1.0f, -1.0f);
+  pair_t ta, tb;
+  ulonglong2 o = xv;
+  if (kObjective == 2) {
+    ta = fma2(cv.x, neg1, xv.x);
+    tb = fma2(cv.y, neg1, xv.y);
+  } else {
+    o = update_core_rnd<kObjective, kFastNoise>(alpha, ns, rnd, xv, cv, xm, nw2, ta, tb);
+  }
+  const pair_t da = fma2(pivot.x, neg1, xv.x), db = fma2(pivot.y, neg1, xv.y);  // x - pivot
+  acc.s1a = add2(acc.s1a, da);
+  acc.s1b = add2(acc.s1b, db);
+  acc.s2a = fma2(da, da, acc.s2a);
+  acc.s2b = fma2(db, db, acc.s2b);
+  lacc.la = fma2(ta, ta, lacc.la);
+  lacc.lb = fma2(tb, tb, lacc.lb);
+  return o;
+}
+
+template <int kObjective, bool kFastNoise>
+__device__ __forceinline__ ulonglong2 row_update(float alpha, float sigma_s, const PhiloxKeys& keys, uint32_t round_lo,
                                                  uint32_t ctr3, uint32_t q32, uint32_t worker, ulonglong2 xv, ulonglong2 cv,
                                                  ulonglong2 xm, ulonglong2 pivot, float w, int live, ColAcc& acc,
                                                  LossAcc& lacc) {
@@ -184,7 +266,7 @@ __device__ __forceinline__ ulonglong2 row_update(float alpha, float sigma, const
     ta = fma2(cv.x, neg1, xv.x);
     tb = fma2(cv.y, neg1, xv.y);
   } else {
-    o = update_core<kObjective, kFastNoise>(alpha, sigma, keys, round_lo, ctr3, q32, worker, xv, cv, xm, w, live, ta, tb);
+    o = update_core<kObjective, kFastNoise>(alpha, sigma_s, keys, round_lo, ctr3, q32, worker, xv, cv, xm, w, live, ta, tb);
   }
   const pair_t da = fma2(pivot.x, neg1, xv.x), db = fma2(pivot.y, neg1, xv.y);  // x - pivot
   acc.s1a = add2(acc.s1a, da);
@@ -297,6 +379,14 @@ __device__ __forceinline__ void load_draws(const RoundParams& p, const int32_t* 
     s_pw[i] = make_int2(m, __float_as_int((m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * p.M + m)));
   }
 }
+
+// 16 bytes from global to shared memory without passing through registers or L1 (data that no other
+// thread of the SM will ask for); completion is awaited by the same thread with cp_async_wait_all.
+__device__ __forceinline__ void cp_async_16_stream(void* smem_dst, const void* gmem_src) {
+  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 // Loads of replica data.  Inside one launch per round the round-start buffer is read-only
 // (non-coherent path); a launch that runs several rounds reads what other SMs wrote a round
@@ -578,6 +668,9 @@ __global__ void __launch_bounds__(256, 2) multi_round_kernel(const MultiRoundPar
 #ifndef NETMAX_FUSED_UNROLL
 #define NETMAX_FUSED_UNROLL 2
 #endif
+#ifndef NETMAX_FUSED_PREFETCH
+#define NETMAX_FUSED_PREFETCH 1  // fetch the next tile under the last round of the current one (fp32 state)
+#endif
 constexpr int kFusedMaxRounds = NETMAX_FUSED_MAX_ROUNDS;
 constexpr int kFusedUnroll = NETMAX_FUSED_UNROLL;  // rows of a round in flight per thread
 
@@ -601,7 +694,7 @@ struct FusedParams {
   PhiloxKeys keys;
 };
 
-// Dynamic shared memory: (peer row offset, weight) int2[kFusedMaxRounds][M], then the slabs
+// Dynamic shared memory: (peer row offset, -, -weight, -weight) int4[kFusedMaxRounds][M], then the slabs
 // float4[3][M][blockDim] (replicas of even rounds, of odd rounds, centres), then 64 doubles.
 // Any block size that is a multiple of 32 up to 256 works.
 template <int kObjective, bool kFastNoise, bool kBf16>
@@ -609,8 +702,8 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
   constexpr uint32_t kGroupBytes = kBf16 ? 8u : 16u;  // four elements in global memory
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int tid = threadIdx.x, T = blockDim.x, M = p.M;
-  int2* s_pw = reinterpret_cast<int2*>(smem_raw);  // (byte offset of the peer's row in a slab, weight bits)
-  const uint32_t head = ((uint32_t)(kFusedMaxRounds * M * 8) + 127u) & ~127u;
+  int4* s_pw = reinterpret_cast<int4*>(smem_raw);  // (byte offset of the peer's row in a slab, unused, -w, -w)
+  const uint32_t head = ((uint32_t)(kFusedMaxRounds * M * 16) + 127u) & ~127u;
   const uint32_t stride = (uint32_t)T * 16u;     // bytes between consecutive rows of a slab
   const uint32_t plane = (uint32_t)M * stride;   // bytes of one [M][T] slab
   unsigned char* slab = smem_raw + head + (uint32_t)tid * 16u;  // this thread's column: slabs 0, 1 (replicas), 2 (centres)
@@ -620,7 +713,8 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
     const int32_t* peers = p.trace + ((p.slot0 + k) % p.ring) * M;
     for (int i = tid; i < M; i += T) {
       const int32_t m = __ldg(peers + i);
-      s_pw[k * M + i] = make_int2((int)((uint32_t)m * stride), __float_as_int((m == i) ? 0.0f : __ldg(p.wtab + (size_t)i * M + m)));
+      const int nw = __float_as_int((m == i) ? -0.0f : -__ldg(p.wtab + (size_t)i * M + m));
+      s_pw[k * M + i] = make_int4((int)((uint32_t)m * stride), 0, nw, nw);
     }
   }
   __syncthreads();
@@ -629,15 +723,29 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
 #pragma unroll
   for (int k = 0; k < kFusedMaxRounds; ++k) acc_cons[k] = acc_loss[k] = 0.0;
 
+  // Slab `base` (0 or 1) holds the tile's values at the start of the first round; round k reads
+  // slab (base + k) & 1 and writes the other one.  The LAST round of a tile writes its results
+  // straight to global memory, which leaves its would-be output slab idle for that whole round:
+  // the next tile's replicas are fetched into it (cp.async, fp32 state), and the next tile's centre
+  // of a row replaces the current one as soon as that row has been updated for the last time.  The
+  // global loads of a tile thus run under the last round of its predecessor.  Every slab slot is
+  // read and written by its own thread only, so cp.async.wait_all is all the synchronisation needed.
+  constexpr bool kPrefetch = !kBf16 && NETMAX_FUSED_PREFETCH != 0;
+  uint32_t base = 0;
+  bool fetched = false;  // has this tile been fetched by the previous one?
   for (int64_t tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x) {
     const int64_t q = tile * T + tid;
-    if (q >= p.nq) continue;  // no barrier below: threads are independent
-    const int live_lo = live_lanes((p.tail != 0) && (q == p.nq - 1), p.tail, 0);
+    if (q >= p.nq) continue;  // no barrier below: threads are independent (and later tiles only have larger q)
+    const NoiseLanes ns = noise_lanes(p.sigma, live_lanes((p.tail != 0) && (q == p.nq - 1), p.tail, 0));
     const uint32_t q32 = (uint32_t)q + p.q_offset;
-    {  // all rows of this column group into the thread's slabs
+    const int64_t q_next = q + (int64_t)gridDim.x * T;
+    const bool have_next = kPrefetch && tile + gridDim.x < p.n_tiles && q_next < p.nq;
+    if (fetched) {
+      cp_async_wait_all();
+    } else {  // all rows of this column group into the thread's slabs
       const char* xq = reinterpret_cast<const char*>(p.x_cur) + (uint64_t)q * kGroupBytes;
       const char* cq = reinterpret_cast<const char*>(p.c) + (uint64_t)q * kGroupBytes;
-      unsigned char* sx = slab;
+      unsigned char* sx = slab + base * plane;
       unsigned char* sc = slab + 2u * plane;
 #pragma unroll 4
       for (int i = 0; i < M; ++i) {
@@ -654,54 +762,83 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
         sc += stride;
       }
     }
-#pragma unroll
-    for (int k = 0; k < kFusedMaxRounds; ++k) {
-      if (k < p.n_rounds) {
-        const uint64_t round = p.first_round + (uint64_t)k;
-        const uint32_t round_lo = (uint32_t)round, ctr3 = philox_ctr3(kTagNoise, round);
-        const unsigned char* cur = slab + (uint32_t)(k & 1) * plane;
-        unsigned char* nxt = slab + (uint32_t)((k & 1) ^ 1) * plane;
-        const unsigned char* cen = slab + 2u * plane;
-        const int2* pw = s_pw + k * M;
-        const ulonglong2 pivot = *reinterpret_cast<const ulonglong2*>(cur);
-        ColAcc acc;
-        LossAcc lacc;
-        uint32_t off = 0;
-#pragma unroll kFusedUnroll
-        for (int i = 0; i < M; ++i) {
-          const int2 d = pw[i];
-          const ulonglong2 o = row_update<kObjective, kFastNoise>(
-              p.alpha, p.sigma, p.keys, round_lo, ctr3, q32, (uint32_t)i, *reinterpret_cast<const ulonglong2*>(cur + off),
-              *reinterpret_cast<const ulonglong2*>(cen + off), *reinterpret_cast<const ulonglong2*>(cur + (uint32_t)d.x), pivot,
-              __int_as_float(d.y), live_lo, acc, lacc);
-          *reinterpret_cast<ulonglong2*>(nxt + off) = kBf16 ? widen_bf16x4(narrow_bf16x4(o)) : o;
-          off += stride;
-        }
-        float4 s1, s2;
-        unpack2(acc.s1a, s1.x, s1.y);
-        unpack2(acc.s1b, s1.z, s1.w);
-        unpack2(acc.s2a, s2.x, s2.y);
-        unpack2(acc.s2b, s2.z, s2.w);
-        float l0, l1, l2, l3;
-        unpack2(lacc.la, l0, l1);
-        unpack2(lacc.lb, l2, l3);
-        const float cons = (s2.x - s1.x * s1.x * p.inv_M) + (s2.y - s1.y * s1.y * p.inv_M) +
-                           (s2.z - s1.z * s1.z * p.inv_M) + (s2.w - s1.w * s1.w * p.inv_M);
-        acc_cons[k] += (double)cons;
-        acc_loss[k] += (double)((l0 + l1) + (l2 + l3));
-      }
-    }
-    {
-      const unsigned char* fin = slab + (uint32_t)(p.n_rounds & 1) * plane;
-      char* oq = reinterpret_cast<char*>(p.x_nxt) + (uint64_t)q * kGroupBytes;
+    unsigned char* const cen = slab + 2u * plane;
+    char* const oq = reinterpret_cast<char*>(p.x_nxt) + (uint64_t)q * kGroupBytes;
+    const char* const cq_next = reinterpret_cast<const char*>(p.c) + (uint64_t)q_next * kGroupBytes;
+
+    // one round over the thread's column group; kLast: the tile's last round (see above)
+    auto run_round = [&](int k, auto last_tag) {
+      constexpr bool kLast = decltype(last_tag)::value;
+      const uint64_t round = p.first_round + (uint64_t)k;
+      const uint32_t round_lo = (uint32_t)round, ctr3 = philox_ctr3(kTagNoise, round);
+      const unsigned char* cur = slab + ((base + (uint32_t)k) & 1u) * plane;
+      unsigned char* nxt = slab + ((base + (uint32_t)k + 1u) & 1u) * plane;
+      if (kLast && have_next) {
+        const char* xq = reinterpret_cast<const char*>(p.x_cur) + (uint64_t)q_next * kGroupBytes;
+        unsigned char* sx = nxt;
 #pragma unroll 4
-      for (int i = 0; i < M; ++i) {
-        if (kBf16) *reinterpret_cast<unsigned long long*>(oq) = narrow_bf16x4(*reinterpret_cast<const ulonglong2*>(fin));
-        else *reinterpret_cast<ulonglong2*>(oq) = *reinterpret_cast<const ulonglong2*>(fin);
-        oq += p.row_bytes;
-        fin += stride;
+        for (int i = 0; i < M; ++i) {
+          cp_async_16_stream(sx, xq);
+          xq += p.row_bytes;
+          sx += stride;
+        }
       }
-    }
+      const int4* pw = s_pw + k * M;
+      const ulonglong2 pivot = *reinterpret_cast<const ulonglong2*>(cur);
+      ColAcc acc;
+      LossAcc lacc;
+      uint32_t off = 0;
+      uint64_t goff = 0;
+      auto do_row = [&](int i, uint4 rnd) {
+        const int4 d = pw[i];
+        const pair_t nw2 = ((pair_t)(uint32_t)d.w << 32) | (uint32_t)d.z;
+        const ulonglong2 o = row_update_rnd<kObjective, kFastNoise>(
+            p.alpha, ns, rnd, *reinterpret_cast<const ulonglong2*>(cur + off),
+            *reinterpret_cast<const ulonglong2*>(cen + off), *reinterpret_cast<const ulonglong2*>(cur + (uint32_t)d.x), pivot,
+            nw2, acc, lacc);
+        if (kLast) {
+          if (kBf16) *reinterpret_cast<unsigned long long*>(oq + goff) = narrow_bf16x4(o);
+          else *reinterpret_cast<ulonglong2*>(oq + goff) = o;
+          if (have_next) cp_async_16_stream(cen + off, cq_next + goff);  // this row's centre is not read again in this tile
+          goff += p.row_bytes;
+        } else {
+          *reinterpret_cast<ulonglong2*>(nxt + off) = kBf16 ? widen_bf16x4(narrow_bf16x4(o)) : o;
+        }
+        off += stride;
+      };
+      // the Philox block of row i + 1 is drawn while row i goes through Box-Muller and Eq. 15-16:
+      // the two are independent, so the integer multiplies of the one fill the latencies of the other
+      uint4 rnd = noise_block<kObjective>(p.keys, round_lo, ctr3, q32, 0u);
+#pragma unroll kFusedUnroll
+      for (int i = 0; i + 1 < M; ++i) {
+        const uint4 rnd_next = noise_block<kObjective>(p.keys, round_lo, ctr3, q32, (uint32_t)(i + 1));
+        do_row(i, rnd);
+        rnd = rnd_next;
+      }
+      do_row(M - 1, rnd);
+      float4 s1, s2;
+      unpack2(acc.s1a, s1.x, s1.y);
+      unpack2(acc.s1b, s1.z, s1.w);
+      unpack2(acc.s2a, s2.x, s2.y);
+      unpack2(acc.s2b, s2.z, s2.w);
+      float l0, l1, l2, l3;
+      unpack2(lacc.la, l0, l1);
+      unpack2(lacc.lb, l2, l3);
+      const double cons = (double)((s2.x - s1.x * s1.x * p.inv_M) + (s2.y - s1.y * s1.y * p.inv_M) +
+                                   (s2.z - s1.z * s1.z * p.inv_M) + (s2.w - s1.w * s1.w * p.inv_M));
+      const double loss = (double)((l0 + l1) + (l2 + l3));
+#pragma unroll
+      for (int kk = 0; kk < kFusedMaxRounds; ++kk) {  // acc[k] with k known only at run time: predicated adds keep it in registers
+        if (kk == k) {
+          acc_cons[kk] += cons;
+          acc_loss[kk] += loss;
+        }
+      }
+    };
+    for (int k = 0; k + 1 < p.n_rounds; ++k) run_round(k, std::false_type());
+    run_round(p.n_rounds - 1, std::true_type());
+    base = (base + (uint32_t)p.n_rounds) & 1u;
+    fetched = have_next;
   }
 
   // telemetry: per round, CTA partials; the last CTA to finish sums them in index order

@@ -13,6 +13,20 @@
 //     value that meets the time constraint and the remainder goes to the fastest peer(s);
 //   * with every row meeting Eq. 10, p_i = 1/M (Lemma 1), which Y_P uses directly;
 //   * eps = 1e-3; infeasible grid points are skipped; ties keep the earlier grid point.
+//
+// The same search for pull rules with a constant weight w (the section on extending existing
+// decentralised PSGD approaches), netmax_policy_generate_fixed_weight:
+//   * E[D^T D] for D = I + w e_i (e_m - e_i)^T has y_im = (w - w^2)(p_i p_im + p_m p_mi), so the
+//     replacement of Eq. 11 ("every y_im on a link is positive") reads p_im + p_mi > 0; it is taken
+//     closed with a floor phi on both directions of every link, and phi takes rho's place in the
+//     outer loop (phi_k = k U_phi / K, U_phi where the floors alone fill a row);
+//   * Y_P is doubly stochastic only if, besides Eq. 10 (p_i = 1/M), the columns of P sum to 1
+//     (row sums of Y_P are 1 + w (sum_m p_m p_mi - p_i sum_m p_im)): an added constraint that couples
+//     the rows of the LP;
+//   * the optimum is again not unique; the reading is p_ii = 0 and the maximum-entropy P above the
+//     floors, p_im = phi + A_i B_m exp(-eta_i t_im), found by alternating scalings: rows (A_i and
+//     eta_i from the row's sum and mean time), then columns (B_m from the column sums); the inner
+//     grid takes the midpoints of R cells of [L, U].
 #include "../../include/netmax.h"
 
 #include <algorithm>
@@ -373,6 +387,229 @@ int netmax_policy_generate_ex(int32_t M, const double* t, const uint8_t* adj, do
   if (bestP.empty()) return fail(NETMAX_INFEASIBLE, "policy_generate: no feasible (rho, t_bar) grid point");
   std::copy(bestP.begin(), bestP.end(), prob_out);
   *rho_out = best_rho;
+  if (info_out) {
+    info_out[0] = best_lam;
+    info_out[1] = best_tbar;
+    info_out[2] = best_tconv;
+    info_out[3] = best_k;
+    info_out[4] = best_r;
+  }
+  return NETMAX_OK;
+}
+
+}  // extern "C"
+
+
+// ---- constant pull weight -----------------------------------------------------------------------
+namespace {
+
+// The maximum-entropy P above the floor phi with zero diagonal, rows and columns summing to 1 and
+// sum_m t_im p_im = T in every row.  Residual r = p - phi on links: r_im = A_i B_m exp(-eta_i s_im)
+// with s the iteration times mapped to [0, 1].  Rows first (eta_i by a bracketed Newton iteration
+// on the row's mean time, then A_i from its sum), then columns (B_m); repeated until every
+// constraint holds to 1e-12.  Returns false when the constraints cannot be met.
+bool solve_fixed_weight(int M, const double* t, const uint8_t* adj, double phi, double T, std::vector<double>& P) {
+  std::vector<std::vector<int>> nb(M);
+  std::vector<double> rows(M), cols(M, 1.0), tau(M);
+  double tmin = INFINITY, tmax = 0.0;
+  for (int i = 0; i < M; ++i)
+    for (int m = 0; m < M; ++m)
+      if (m != i && adj[(size_t)i * M + m]) {
+        nb[i].push_back(m);
+        tmin = std::min(tmin, t[(size_t)i * M + m]);
+        tmax = std::max(tmax, t[(size_t)i * M + m]);
+        cols[m] -= phi;
+      }
+  const bool homogeneous = tmax - tmin <= kTie * tmax;  // all links equally fast: the time constraint only says T = t
+  if (homogeneous && std::fabs(T - tmin) > 1e-9 * tmax) return false;
+  const double scale = homogeneous ? INFINITY : tmax - tmin;  // (t - tmin) / scale = 0 on every link then
+  bool floors_fill = true;
+  for (int i = 0; i < M; ++i) {
+    rows[i] = 1.0 - phi * (double)nb[i].size();
+    if (rows[i] < -1e-15) return false;
+    double floor_time = 0.0;
+    for (int m : nb[i]) floor_time += t[(size_t)i * M + m];
+    tau[i] = homogeneous ? 0.0 : (T - phi * floor_time - tmin * rows[i]) / scale;  // target of sum_m s_im r_im
+    if (rows[i] > 1e-15) floors_fill = false;
+  }
+  P.assign((size_t)M * M, 0.0);
+  auto finish = [&](const std::vector<double>& r) {
+    double worst = 0.0;
+    std::vector<double> colsum(M, 0.0);
+    for (int i = 0; i < M; ++i) {
+      double sum = 0.0, time = 0.0;
+      for (int m : nb[i]) {
+        const double p = phi + r[(size_t)i * M + m];
+        P[(size_t)i * M + m] = p;
+        sum += p;
+        time += p * t[(size_t)i * M + m];
+        colsum[m] += p;
+      }
+      worst = std::max(worst, std::max(std::fabs(sum - 1.0), std::fabs(time - T) / tmax));
+    }
+    for (int m = 0; m < M; ++m) worst = std::max(worst, std::fabs(colsum[m] - 1.0));
+    return worst <= 1e-9;
+  };
+  std::vector<double> r((size_t)M * M, 0.0);
+  if (floors_fill) return finish(r);
+  for (int i = 0; i < M; ++i)
+    if (tau[i] < -1e-12 || tau[i] > rows[i] * (1.0 + 1e-12)) return false;
+
+  std::vector<double> A(M, 1.0), B(M, 1.0), eta(M, 0.0), wgt(M);
+  for (int sweep = 0; sweep < 20000; ++sweep) {
+    // rows: weights B_m exp(-eta s_im); their mean s must equal tau_i / rows_i
+    double row_change = 0.0;
+    for (int i = 0; i < M; ++i) {
+      if (!(rows[i] > 1e-15)) { A[i] = 0.0; continue; }
+      const double sig = std::min(std::max(tau[i] / rows[i], 0.0), 1.0);
+      auto stats = [&](double e, double& z, double& mean, double& var) {
+        double a = 0.0, b = 0.0;
+        z = 0.0;
+        for (int m : nb[i]) {
+          const double sv = (t[(size_t)i * M + m] - tmin) / scale;
+          const double w = B[m] * std::exp(-e * sv);
+          z += w;
+          a += w * sv;
+          b += w * sv * sv;
+        }
+        mean = a / z;
+        var = b / z - mean * mean;
+      };
+      double lo = -kEtaCap, hi = kEtaCap, e = eta[i], z, mean, var;
+      stats(lo, z, mean, var);
+      if (sig >= mean) {
+        e = lo;
+      } else {
+        stats(hi, z, mean, var);
+        if (sig <= mean) {
+          e = hi;
+        } else {
+          stats(e, z, mean, var);
+          for (int it = 0; it < 200; ++it) {
+            const double gap = mean - sig;
+            if (std::fabs(gap) <= 1e-15) break;
+            if (gap > 0) lo = e; else hi = e;
+            double next = (var > 1e-300) ? e + gap / var : 0.5 * (lo + hi);
+            if (!(next > lo && next < hi)) next = 0.5 * (lo + hi);
+            if (next == e || hi - lo <= 1e-15 * (1.0 + std::fabs(e))) break;
+            e = next;
+            stats(e, z, mean, var);
+          }
+        }
+      }
+      stats(e, z, mean, var);
+      row_change = std::max(row_change, std::fabs(e - eta[i]));
+      eta[i] = e;
+      A[i] = rows[i] / z;
+    }
+    // columns: B_m from the column sums
+    double col_err = 0.0;
+    std::fill(wgt.begin(), wgt.end(), 0.0);
+    for (int i = 0; i < M; ++i)
+      for (int m : nb[i]) wgt[m] += A[i] * std::exp(-eta[i] * (t[(size_t)i * M + m] - tmin) / scale);
+    for (int m = 0; m < M; ++m) {
+      if (!(wgt[m] > 0.0)) continue;
+      const double next = std::max(cols[m], 0.0) / wgt[m];
+      col_err = std::max(col_err, std::fabs(next - B[m]) * wgt[m]);   // column sum before the rescaling, off by this much
+      B[m] = next;
+    }
+    if (col_err <= 1e-13 && row_change <= 1e-12) break;
+  }
+  for (int i = 0; i < M; ++i)
+    for (int m : nb[i]) r[(size_t)i * M + m] = A[i] * B[m] * std::exp(-eta[i] * (t[(size_t)i * M + m] - tmin) / scale);
+  return finish(r);
+}
+
+}  // namespace
+
+extern "C" {
+
+int netmax_policy_fixed_weight_at(int32_t M, const double* t, const uint8_t* adj, double floor, double t_bar, double* prob_out) {
+  if (M < 2 || !t || !adj || !prob_out || !(floor >= 0.0) || !(t_bar > 0.0) || !std::isfinite(floor) || !std::isfinite(t_bar))
+    return fail(NETMAX_INVALID_ARG, "policy_fixed_weight_at: bad argument");
+  std::vector<double> P;
+  if (!solve_fixed_weight(M, t, adj, floor, M * t_bar, P))
+    return fail(NETMAX_INFEASIBLE, "policy_fixed_weight_at: no P meets the floors, the row and column sums and the mean iteration time");
+  std::copy(P.begin(), P.end(), prob_out);
+  return NETMAX_OK;
+}
+
+int netmax_policy_generate_fixed_weight(int32_t M, const double* t, const uint8_t* adj, double pull_weight, int32_t K,
+                                        int32_t R, double floor_upper, double* prob_out, double* floor_out, double* info_out) {
+  if (M < 2 || !t || !adj || !prob_out || !floor_out || !(pull_weight > 0.0 && pull_weight < 1.0) || K < 1 || R < 1)
+    return fail(NETMAX_INVALID_ARG, "policy_generate_fixed_weight: bad argument");
+  int max_deg = 0;
+  for (int i = 0; i < M; ++i) {
+    int deg = 0;
+    for (int m = 0; m < M; ++m) {
+      if (m == i || !adj[(size_t)i * M + m]) continue;
+      if (!adj[(size_t)m * M + i]) return fail(NETMAX_INVALID_ARG, "policy_generate_fixed_weight: the link graph must be symmetric");
+      const double tm = t[(size_t)i * M + m];
+      if (!(tm > 0.0) || !std::isfinite(tm)) return fail(NETMAX_INVALID_ARG, "policy_generate_fixed_weight: iteration time on a link is not positive");
+      ++deg;
+    }
+    if (deg == 0) return fail(NETMAX_NOT_CONNECTED, "policy_generate_fixed_weight: a worker has no neighbour");
+    max_deg = std::max(max_deg, deg);
+  }
+  const double U_phi = floor_upper > 0.0 ? floor_upper : (1.0 - 1e-6) / max_deg;
+  const double w = pull_weight;
+  std::vector<double> P, Y((size_t)M * M), bestP;
+  double best_tconv = INFINITY, best_phi = 0, best_lam = 0, best_tbar = 0;
+  int best_k = 0, best_r = 0;
+  for (int k = 1; k <= K; ++k) {
+    const double phi = k * U_phi / K;
+    // range of the rows' mean time: floors plus all of the remainder on the fastest / slowest link
+    double L = 0.0, U = INFINITY;
+    bool rows_ok = true;
+    for (int i = 0; i < M; ++i) {
+      double sum_t = 0.0, tmin = INFINITY, tmax = 0.0;
+      int deg = 0;
+      for (int m = 0; m < M; ++m) {
+        if (m == i || !adj[(size_t)i * M + m]) continue;
+        const double tm = t[(size_t)i * M + m];
+        sum_t += tm;
+        tmin = std::min(tmin, tm);
+        tmax = std::max(tmax, tm);
+        ++deg;
+      }
+      const double rest = 1.0 - phi * deg;
+      if (rest < -1e-15) rows_ok = false;
+      L = std::max(L, (phi * sum_t + rest * tmin) / M);
+      U = std::min(U, (phi * sum_t + rest * tmax) / M);
+    }
+    if (!rows_ok || !(U >= L)) continue;
+    for (int r = 1; r <= R; ++r) {
+      const double tbar = L + (r - 0.5) * (U - L) / R;  // cell midpoints: the end points are degenerate vertices
+      if (!solve_fixed_weight(M, t, adj, phi, M * tbar, P)) continue;
+      // E[D^T D] with p_i = 1/M (Eq. 10 holds by construction)
+      for (int i = 0; i < M; ++i) {
+        double pulls = 0.0, pulled = 0.0;
+        for (int m = 0; m < M; ++m) {
+          if (m == i) continue;
+          const double pim = P[(size_t)i * M + m], pmi = P[(size_t)m * M + i];
+          Y[(size_t)i * M + m] = (w - w * w) * (pim + pmi) / M;
+          pulls += pim;
+          pulled += pmi;
+        }
+        Y[(size_t)i * M + i] = 1.0 - (2.0 * w - w * w) * pulls / M + w * w * pulled / M;
+      }
+      const double lam2 = second_eigenvalue(Y, M);
+      if (!(lam2 > 0.0 && lam2 < 1.0)) continue;
+      const double tconv = tbar * std::log(kEps) / std::log(lam2);
+      if (bestP.empty() || tconv < best_tconv * (1.0 - 1e-12)) {
+        bestP = P;
+        best_tconv = tconv;
+        best_phi = phi;
+        best_lam = lam2;
+        best_tbar = tbar;
+        best_k = k;
+        best_r = r;
+      }
+    }
+  }
+  if (bestP.empty()) return fail(NETMAX_INFEASIBLE, "policy_generate_fixed_weight: no feasible (floor, t_bar) grid point");
+  std::copy(bestP.begin(), bestP.end(), prob_out);
+  *floor_out = best_phi;
   if (info_out) {
     info_out[0] = best_lam;
     info_out[1] = best_tbar;

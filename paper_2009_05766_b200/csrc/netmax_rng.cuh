@@ -130,13 +130,18 @@ __device__ __forceinline__ pair_t add2(pair_t a, pair_t b) {
   return d;
 }
 
-// The two normals of one Box-Muller pair, packed (fast path; same arithmetic as normal_pair_fast).
-__device__ __forceinline__ pair_t normal_pair_fast_packed(uint32_t a, uint32_t b) {
+// The two normals of one Box-Muller pair, packed, fast path, WITHOUT the constant factor of the
+// radius: returns sqrt(-log2 u1) (cos 2 pi u2, sin 2 pi u2), i.e. the pair of normals divided by
+// kNormalScale = sqrt(2 ln 2); the caller folds that constant into its noise scale.
+// u1 < 1, so log2 u1 < 0; the hardware logarithm has an absolute error of about 2^-22 and may
+// return +0 or a tiny positive value for u1 next to 1, hence |.| (an operand modifier, not an
+// instruction) instead of a negation under the square root.
+constexpr double kNormalScale = 1.17741002251547469101;  // sqrt(2 ln 2)
+__device__ __forceinline__ pair_t normal_pair_fast_unscaled(uint32_t a, uint32_t b) {
   const float u1 = radius_uniform(a);
-  const float ang = (float)((int32_t)b >> 8) * 3.74507028e-07f;
-  const float r2 = fmaxf(-1.38629436111989f * log2_fast(u1), 0.0f);
+  const float ang = (float)((int32_t)b >> 8) * 3.74507028e-07f;  // 2 pi / 2^24
   float rad;
-  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(r2));
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(fabsf(log2_fast(u1))));
   float s, c;
   __sincosf(ang, &s, &c);
   return mul2(pack2(rad, rad), pack2(c, s));

@@ -24,7 +24,9 @@ def run_bench(*args):
 
 
 @pytest.mark.parametrize("args,bound", [
-    (["--workload", "cfg1", "--steps", "40", "--warmup", "3", "--e2e-steps", "2", "--no-cpu-baseline"], "hbm"),
+    (["--workload", "cfg1", "--steps", "40", "--warmup", "3", "--e2e-steps", "2", "--no-cpu-baseline", "--configs", "none"], "alu"),
+    (["--workload", "cfg1", "--steps", "40", "--warmup", "3", "--e2e-steps", "2", "--no-cpu-baseline", "--configs", "none",
+      "--fuse-rounds", "1"], "alu"),       # short vectors: one cooperative launch runs all 40 rounds
     (["--d", "400003", "--steps", "12", "--warmup", "3", "--e2e-steps", "2", "--no-cpu-baseline"], "alu"),
     (["--d", "400003", "--steps", "6", "--warmup", "3", "--e2e-steps", "2", "--no-cpu-baseline", "--fuse-rounds", "1"], "hbm"),
     (["--d", "800003", "--steps", "8", "--warmup", "3", "--e2e-steps", "1", "--no-cpu-baseline", "--storage", "bf16"], "alu"),
@@ -35,7 +37,8 @@ def test_bench_line_has_the_contract_keys(args, bound):
         assert key in line, key
     assert line["metric"] == "replica GB/s" and line["unit"] == "GB/s" and line["higher_is_better"] is True
     assert line["n_gpus"] == 1 and line["value"] > 0 and line["ms_per_step"] > 0 and line["gpu_launches"] > 0
-    assert line["dtype"] == "f32" and line["data"] == "synthetic" and line["vs_baseline"] is None
+    assert line["dtype"] == ("bf16 storage, f32 arithmetic" if "bf16" in args else "f32")
+    assert line["data"] == "synthetic" and line["vs_baseline"] is None
     assert "workload" in line["config"] and "model" not in line["config"]
     roof = line["roofline"]
     for key in ("bound", "achieved", "peak", "unit", "frac", "traffic"):
@@ -45,8 +48,20 @@ def test_bench_line_has_the_contract_keys(args, bound):
     assert e2e["value"] > 0 and e2e["h2d_bytes_per_step"] > 0 and e2e["d2h_bytes_per_step"] > 0
     assert e2e["value"] < line["value"]
     assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(line["clocks"])
-    if bound == "alu":
+    if bound == "alu" and roof["kernel"] == "fused_rounds_kernel":
         assert "one_launch_per_round" in line and line["one_launch_per_round"]["roofline"]["bound"] == "hbm"
+    if bound == "hbm":
+        assert roof["achieved"] == pytest.approx(0.75 * roof["replica_GBs"])       # 12 of the 16 bytes per element
+
+
+def test_bench_line_carries_the_other_configs():
+    line = run_bench("--workload", "cfg1", "--steps", "40", "--warmup", "3", "--e2e-steps", "1", "--no-cpu-baseline",
+                     "--configs", "1,5")
+    assert set(line["configs"]) == {"cfg1", "cfg5"}
+    for entry in line["configs"].values():
+        assert entry["ms_per_round"] > 0 and entry["replica_GBs"] > 0 and entry["launch_shape"]
+        assert {"bound", "achieved", "peak", "frac", "traffic"} <= set(entry["roofline"])
+    assert line["configs"]["cfg5"]["M"] == 4096 and "clocks" in line["configs"]["cfg5"]
 
 
 def test_async_bench_line():

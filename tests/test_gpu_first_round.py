@@ -25,6 +25,11 @@ def nm():
     return binding
 
 
+def bf16_ulp(v):
+    """Spacing of bfloat16 (8 significant bits) at magnitude v."""
+    return 2.0 ** (np.floor(np.log2(v)) - 7)
+
+
 def full_adj(M):
     return (1 - np.eye(M)).astype(np.uint8)
 
@@ -72,10 +77,10 @@ def test_rounds_across_the_32_bit_boundary_match_the_oracle(nm, M, d, fuse, stor
     got = g.read_replicas() if cols is None else g.read_columns(cols)
     want = o.x()
     if storage == "bf16":
-        # codes may differ by one bfloat16 step where the fast noise moves a value across a rounding boundary
-        step = np.abs(want.astype(np.float64)) * 2.0 ** -7 + 1e-30
-        assert (np.abs(got.astype(np.float64) - want) <= step).all()
-        assert (got != want).mean() < 5e-3
+        # a code may differ by a bfloat16 step where the fast noise moves a value across a rounding
+        # boundary, and such a step travels on with the pulls: a few steps of the state's scale at most
+        units = np.abs(got.astype(np.float64) - want) / bf16_ulp(np.maximum(np.abs(want), 0.25))
+        assert units.max() <= 2.0 and (units > 0).mean() < 2e-3, f"max {units.max():.2f} units, {(units > 0).mean():.2e} differ"
     else:
         assert (np.abs(got.astype(np.float64) - want) <= TOL * (1.0 + np.abs(want.astype(np.float64)))).all()
     gc, gl = g.telemetry()
