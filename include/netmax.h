@@ -77,7 +77,9 @@ typedef struct netmax_config {
   const double* link_speed_gbps; /* host, M*M, symmetric, diagonal ignored; speed <= 0 means "no link"
                                     (d_im = 0).  NULL means fully connected with equal speeds          */
   const double* prob;            /* host, M*M, row i = P[i,:].  NULL: run Algorithm 3 on the iteration
-                                    times derived from link_speed_gbps (policy_K x policy_R grid)      */
+                                    times derived from link_speed_gbps (policy_K x policy_R grid); with
+                                    pull_weight > 0 in the form for a constant weight
+                                    (netmax_policy_generate_fixed_weight)                              */
   double lr;                     /* alpha > 0; the update uses its fp32 rounding                       */
   double rho;                    /* rho; <= 0: with prob given, the largest rho meeting Eq. 11 with a
                                     1e-6 margin, min_{p_im>0} p_im / (alpha (d_im+d_mi)); with prob
@@ -99,7 +101,8 @@ typedef struct netmax_config {
   int64_t trace_rounds;          /* capacity of the peer-trace / telemetry ring, in rounds (>= 1)      */
   int32_t policy_K, policy_R;    /* Algorithm 3 grid sizes when prob is NULL (<= 0: 20 x 20)           */
   double policy_rho_upper;       /* upper end of Algorithm 3's rho grid (<= 0: default cap; see
-                                    netmax_policy_generate_ex)                                         */
+                                    netmax_policy_generate_ex); with pull_weight > 0 the upper end of
+                                    the floor grid of netmax_policy_generate_fixed_weight              */
   void* workspace;               /* device memory for ALL of the context's device buffers, 256-byte
                                     aligned, at least netmax_workspace_size() bytes, owned by the
                                     caller and kept alive until netmax_destroy.  NULL: the library
@@ -281,7 +284,9 @@ int netmax_async_steps(netmax_ctx* ctx, int64_t n_steps);
  * collected, Algorithm 3 runs on them (policy_K x policy_R grid) and the resulting P and rho are
  * installed for iterations that start afterwards.  An average with n samples is read as
  * T / (1 - beta^n) (Algorithm 2 starts T at 0); a link never sampled so far is taken at its
- * current iteration time; a grid with no feasible point leaves the policy unchanged.
+ * current iteration time; a grid with no feasible point leaves the policy unchanged.  A context
+ * with a constant pull weight runs netmax_policy_generate_fixed_weight instead ("AD-PSGD with a
+ * Network Monitor").
  * period_s = 0 switches the monitor off.  netmax_async_monitor_refreshes counts the policies
  * installed so far.
  */

@@ -290,10 +290,11 @@ def solve_fixed_weight(t: np.ndarray, adj: np.ndarray, phi: float, T: float, tol
     res = minimize(dual, z0, jac=True, hess=hess, method="trust-exact", options=dict(gtol=1e-14, maxiter=400))
     z = res.x
     for _ in range(50):     # the trust-region method stops where the dual's value no longer resolves: finish with Newton steps on the gradient
-        g = dual(z)[1]
-        if np.abs(g).max() <= 1e-14:
-            break
-        step = np.linalg.lstsq(hess(z), -g, rcond=None)[0]
+        with np.errstate(over="ignore", invalid="ignore"):
+            g, H = dual(z)[1], hess(z)
+        if not (np.isfinite(g).all() and np.isfinite(H).all()) or np.abs(g).max() <= 1e-14:
+            break                                  # (an infeasible target drives the multipliers to infinity)
+        step = np.linalg.lstsq(H, -g, rcond=None)[0]
         if not np.isfinite(step).all():
             break
         z = z + step

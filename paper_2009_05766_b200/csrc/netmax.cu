@@ -354,6 +354,16 @@ int resolve_policy(netmax_ctx* ctx, const double* speed, const double* prob, dou
   }
   ctx->P.assign((size_t)M * M, 0.0);
   double rho_sel = 0.0;
+  if (ctx->pull_weight > 0.0) {
+    // constant pull weight: Algorithm 3 in the form the paper's extension section prescribes (a floor
+    // on p_im in rho's place, balanced columns); rho plays no part in the update
+    double floor_sel = 0.0;
+    int rc = netmax_policy_generate_fixed_weight(M, ctx->t_iter.data(), ctx->adj.data(), ctx->pull_weight, ctx->policy_K,
+                                                 ctx->policy_R, ctx->policy_rho_upper, ctx->P.data(), &floor_sel, nullptr);
+    if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
+    ctx->rho = rho > 0.0 ? rho : 0.0;
+    return NETMAX_OK;
+  }
   // Algorithm 3: on the device from 512 workers up (where the host generator takes seconds)
   int ndev = 0;
   const bool on_device = M >= 512 && cudaGetDeviceCount(&ndev) == cudaSuccess && ctx->device < ndev;
@@ -1441,15 +1451,19 @@ static int monitor_refresh(netmax_ctx* ctx) {
   std::vector<double> P((size_t)M * M);
   double rho = 0.0;
   int ndev = 0;
-  const bool on_device = M >= 512 && cudaGetDeviceCount(&ndev) == cudaSuccess && ctx->device < ndev;
-  int rc = on_device ? netmax_policy_generate_device(M, t.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K, ctx->policy_R,
+  const bool fixed = ctx->pull_weight > 0.0;  // constant pull weight: the extension section's form of Algorithm 3
+  const bool on_device = !fixed && M >= 512 && cudaGetDeviceCount(&ndev) == cudaSuccess && ctx->device < ndev;
+  double floor_sel = 0.0;
+  int rc = fixed ? netmax_policy_generate_fixed_weight(M, t.data(), ctx->adj.data(), ctx->pull_weight, ctx->policy_K, ctx->policy_R,
+                                                       ctx->policy_rho_upper, P.data(), &floor_sel, nullptr)
+           : on_device ? netmax_policy_generate_device(M, t.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K, ctx->policy_R,
                                                      ctx->policy_rho_upper, ctx->device, ctx->stream, P.data(), &rho, nullptr)
                      : netmax_policy_generate_ex(M, t.data(), ctx->adj.data(), ctx->alpha, ctx->policy_K, ctx->policy_R,
                                                  ctx->policy_rho_upper, P.data(), &rho, nullptr);
   if (rc == NETMAX_INFEASIBLE) return NETMAX_OK;
   if (rc) return fail(ctx, rc, "%s", netmax_last_error(nullptr));
   ctx->P.swap(P);
-  ctx->rho = rho;
+  if (!fixed) ctx->rho = rho;
   ctx->monitor_refreshes += 1;
   NM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
   return upload_policy(ctx);

@@ -188,3 +188,55 @@ def test_the_allocation_free_entry_point_names_no_allocating_call():
         assert "cudaGetSymbolAddress" in body or "gather_scratch_address" in body
         for banned in ("cudaMalloc", "cudaFree", "cudaHostAlloc", "cudaMallocAsync", "new ", "std::vector"):
             assert banned not in body, (start, banned)
+
+
+# ---- constant pull weight (the paper's extension section)
+def _fixed_case(name):
+    if name.startswith("cfg"):
+        w = workloads.config(int(name[3]))
+        return opolicy.iteration_times(w.link_speeds(0), w.d)
+    rng = np.random.default_rng(5)
+    M = 7
+    s = np.triu(np.exp(rng.uniform(np.log(1.0), np.log(50.0), (M, M))), 1)
+    s[0, 4] = s[1, 5] = s[2, 6] = 0.0
+    return opolicy.iteration_times(s + s.T, 1_000_000)
+
+
+@pytest.mark.parametrize("name,floor_upper,K,R", [("cfg1", 0.0, 6, 6), ("cfg1", 0.1, 4, 4), ("cfg2", 0.0, 6, 6),
+                                                  ("cfg2", 0.3 / 7, 6, 6), ("cfg3", 0.0, 3, 4), ("cfg3", 0.02, 4, 4),
+                                                  ("sparse7", 0.0, 3, 3), ("sparse7", 0.05, 3, 3)])
+def test_fixed_weight_generator_matches_oracle(name, floor_upper, K, R):
+    t, adj = _fixed_case(name)
+    P, phi, info = binding.netmax_policy_generate_fixed_weight(t, adj, 0.5, K, R, floor_upper)
+    P0, phi0, info0 = opolicy.generate_policy_fixed_weight(t, adj, 0.5, K, R, floor_upper=floor_upper)
+    assert (info["k"], info["r"]) == (info0["k"], info0["r"]) and phi == pytest.approx(phi0, rel=1e-14)
+    np.testing.assert_allclose(P, P0, atol=1e-8)
+    assert info["lam2"] == pytest.approx(info0["lam2"], abs=1e-9)
+    assert info["t_conv"] == pytest.approx(info0["t_conv"], rel=1e-6)
+    np.testing.assert_allclose(P.sum(axis=1), 1.0, atol=1e-9)
+    np.testing.assert_allclose(P.sum(axis=0), 1.0, atol=1e-9)
+
+
+def test_fixed_weight_grid_points_match_oracle_and_report_infeasibility():
+    t, adj = _fixed_case("cfg2")
+    M = t.shape[0]
+    mean_time = float(t[0][adj[0] == 1].mean())
+    for phi, frac in ((0.02, 0.6), (0.05, 0.9), (0.1, 1.0), (1.0 / 7, 1.0)):
+        P = binding.netmax_policy_fixed_weight_at(t, adj, phi, frac * mean_time / M)
+        P0 = opolicy.solve_fixed_weight(t, adj, phi, frac * mean_time)
+        np.testing.assert_allclose(P, P0, atol=1e-8)
+    with pytest.raises(binding.NetmaxError) as e:           # faster than the intra-machine links allow
+        binding.netmax_policy_fixed_weight_at(t, adj, 0.02, 0.5 * float(t[0, 1]) / M)
+    assert e.value.code == -7
+    assert opolicy.solve_fixed_weight(t, adj, 0.02, 0.5 * float(t[0, 1])) is None
+    with pytest.raises(binding.NetmaxError) as e:           # floors beyond a row sum of one
+        binding.netmax_policy_fixed_weight_at(t, adj, 0.2, mean_time / M)
+    assert e.value.code == -7
+    with pytest.raises(binding.NetmaxError) as e:
+        binding.netmax_policy_generate_fixed_weight(t, adj, 1.0, 4, 4)
+    assert e.value.code == -1
+    one_way = adj.copy()
+    one_way[0, 1] = 0
+    with pytest.raises(binding.NetmaxError) as e:
+        binding.netmax_policy_generate_fixed_weight(t, one_way, 0.5, 4, 4)
+    assert e.value.code == -1
