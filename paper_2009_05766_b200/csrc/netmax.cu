@@ -59,6 +59,13 @@ struct FusedPlan {  // launch shape of fused_rounds_kernel
   int64_t n_tiles = 0;
 };
 
+struct ClusterPlan {  // launch shape of cluster_rounds_kernel
+  bool ok = false;
+  int threads = 0, grid = 0, C = 0, rpc = 0, max_rounds = 0;
+  size_t smem = 0;
+  int64_t n_tiles = 0;
+};
+
 struct Layout {
   int64_t ld = 0, ldq = 0, nq = 0;  // row stride in elements / in 16-byte column groups; column groups in use
   int elem = 4, halves = 1;         // bytes per stored element; Philox blocks (4 elements) per column group
@@ -172,6 +179,8 @@ struct netmax_ctx {
   FusedPlan fused;
   bool resident_planned = false;
   ResidentPlan resident;
+  bool cluster_planned = false;
+  ClusterPlan cluster;
   PhiloxKeys keys;
   std::vector<double> P;      // policy in force
   std::vector<uint8_t> adj;   // link graph in force
@@ -676,6 +685,83 @@ int plan_fused(netmax_ctx* ctx, const RoundPlan& plan, FusedPlan& f) {
   return rc;
 }
 
+using ClusterKernel = void (*)(const ClusterParams);
+
+ClusterKernel pick_cluster_kernel(int objective) {
+  return objective == 1 ? cluster_rounds_kernel<1, true> : cluster_rounds_kernel<0, true>;
+}
+
+#ifndef NETMAX_CLUSTER_SIZE
+#define NETMAX_CLUSTER_SIZE 8
+#endif
+#ifndef NETMAX_CLUSTER_THREADS
+#define NETMAX_CLUSTER_THREADS 0  // 0: the smallest of 64, 128, 256 threads per CTA whose slabs fit
+#endif
+
+size_t cluster_smem(int rpc, int threads) {
+  return align_up((size_t)kFusedMaxRounds * rpc * 16, 128) + (size_t)3 * rpc * threads * 16 + (size_t)2 * threads * 16 +
+         64 * sizeof(double);
+}
+
+// Long fp32 vectors with more workers than fused_rounds_kernel can hold per thread (M > 18): the rows
+// of a tile are split over the CTAs of a cluster (cluster_rounds_kernel), up to 18 rows per CTA.
+int plan_cluster_uncached(netmax_ctx* ctx, const RoundPlan& plan, const FusedPlan& fused, ClusterPlan& f) {
+  f = ClusterPlan();
+  if (ctx->fuse_rounds == 1 || plan.short_vectors || fused.ok || ctx->storage != NETMAX_STORAGE_F32) return NETMAX_OK;
+  const int C = NETMAX_CLUSTER_SIZE;
+  const int64_t M = ctx->M;
+  const int rpc = (int)((M + C - 1) / C);
+  if (rpc > 18) return NETMAX_OK;
+  ClusterKernel k = pick_cluster_kernel(ctx->objective);
+  NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
+  // Small CTAs, many per SM: a CTA that waits at the cluster barrier leaves its SM to the others.  Measured
+  // on 64 x 11.2 M elements, clusters of 8: 64 threads (8 CTAs per SM) 1.39 ms per round, 128 threads 1.43,
+  // 256 threads 1.69, 32 threads 2.08; clusters of 4 with 64 threads 1.54 (one launch per round: 1.62).
+  for (int cand : {64, 128, 256}) {
+    if (NETMAX_CLUSTER_THREADS != 0 && cand != NETMAX_CLUSTER_THREADS) continue;
+    const size_t smem = cluster_smem(rpc, cand);
+    if (smem > (size_t)113 * 1024) continue;  // at least two CTAs per SM
+    NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(C * ctx->sm_count));
+    cfg.blockDim = dim3((unsigned)cand);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = (unsigned)C;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, k, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
+    if (clusters < 1) continue;
+    f.threads = cand;
+    f.C = C;
+    f.rpc = rpc;
+    f.smem = smem;
+    f.n_tiles = ((ctx->d + 3) / 4 + cand - 1) / cand;
+    f.max_rounds = ctx->fuse_rounds >= 2 ? std::min(ctx->fuse_rounds, kFusedMaxRounds) : kFusedMaxRounds;
+    f.grid = (int)std::min<int64_t>(f.n_tiles, (int64_t)clusters) * C;
+    f.ok = true;
+    break;
+  }
+  return NETMAX_OK;
+}
+
+int plan_cluster(netmax_ctx* ctx, const RoundPlan& plan, const FusedPlan& fused, ClusterPlan& f) {
+  if (ctx->cluster_planned) {
+    f = ctx->cluster;
+    return NETMAX_OK;
+  }
+  int rc = plan_cluster_uncached(ctx, plan, fused, f);
+  if (rc == NETMAX_OK) {
+    ctx->cluster = f;
+    ctx->cluster_planned = true;
+  }
+  return rc;
+}
+
 }  // namespace
 
 extern "C" {
@@ -985,6 +1071,9 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   rc = plan_resident(ctx, plan, resident);
   if (rc) return rc;
   if (ctx->fuse_rounds == 1) resident.ok = false;  // one launch per round was asked for
+  ClusterPlan cluster;
+  rc = plan_cluster(ctx, plan, fused, cluster);
+  if (rc) return rc;
 
   RoundParams p;
   p.c = reinterpret_cast<const float4*>(ctx->c);
@@ -1096,8 +1185,8 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
       continue;
     }
     for (int64_t b = 0; b < batch;) {
-      if (fused.ok && batch - b >= 2) {  // the next rounds in one launch over resident tiles
-        const int chunk = (int)std::min<int64_t>(batch - b, fused.max_rounds);
+      if ((fused.ok || cluster.ok) && batch - b >= 2) {  // the next rounds in one launch over resident tiles
+        const int chunk = (int)std::min<int64_t>(batch - b, fused.ok ? fused.max_rounds : cluster.max_rounds);
         FusedParams fp;
         fp.x_cur = reinterpret_cast<const float4*>(ctx->x[ctx->cur]);
         fp.x_nxt = reinterpret_cast<float4*>(ctx->x[ctx->cur ^ 1]);
@@ -1112,7 +1201,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
         fp.first_round = (uint64_t)ctx->rounds;
         fp.n_rounds = chunk;
         fp.nq = (ctx->d + 3) / 4;
-        fp.n_tiles = fused.n_tiles;
+        fp.n_tiles = fused.ok ? fused.n_tiles : cluster.n_tiles;
         fp.row_bytes = p.row_bytes;
         fp.M = p.M;
         fp.tail = (int32_t)(ctx->d % 4);
@@ -1121,6 +1210,31 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
         fp.inv_M = p.inv_M;
         fp.q_offset = p.q_offset;
         fp.keys = p.keys;
+        if (!fused.ok) {  // rows split over the CTAs of a cluster
+          ClusterParams cpar;
+          cpar.f = fp;
+          cpar.rpc = cluster.rpc;
+          ClusterKernel ck = pick_cluster_kernel(ctx->objective);
+          NM_CUDA(ctx, cudaFuncSetAttribute(ck, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cluster.smem));
+          cudaLaunchConfig_t lc = {};
+          lc.gridDim = dim3((unsigned)cluster.grid);
+          lc.blockDim = dim3((unsigned)cluster.threads);
+          lc.dynamicSmemBytes = cluster.smem;
+          lc.stream = ctx->stream;
+          cudaLaunchAttribute attr;
+          attr.id = cudaLaunchAttributeClusterDimension;
+          attr.val.clusterDim.x = (unsigned)cluster.C;
+          attr.val.clusterDim.y = 1;
+          attr.val.clusterDim.z = 1;
+          lc.attrs = &attr;
+          lc.numAttrs = 1;
+          NM_CUDA(ctx, cudaLaunchKernelEx(&lc, ck, cpar));
+          ctx->launches += 1;
+          ctx->cur ^= 1;
+          ctx->rounds += chunk;
+          b += chunk;
+          continue;
+        }
         // (the attribute belongs to the kernel, not to this context: another context may have lowered it)
         FusedKernel fk = pick_fused_kernel(ctx->objective, ctx->L.halves);
         NM_CUDA(ctx, cudaFuncSetAttribute(fk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fused.smem));
@@ -1159,6 +1273,7 @@ int netmax_set_fuse_rounds(netmax_ctx* ctx, int32_t fuse_rounds) {
     return fail(ctx, NETMAX_INVALID_ARG, "fuse_rounds = %d outside [0, %d]", fuse_rounds, kFusedMaxRounds);
   ctx->fuse_rounds = fuse_rounds;
   ctx->fused_planned = false;
+  ctx->cluster_planned = false;
   return NETMAX_OK;
 }
 

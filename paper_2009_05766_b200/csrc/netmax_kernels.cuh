@@ -860,6 +860,244 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
   }
 }
 
+// ---- several rounds over a tile that is resident across a thread-block cluster ----------------
+// More workers than a thread's slab can hold (48 M bytes per column group: M = 64 would leave two
+// warps per SM): the rows of a tile are split over the CTAs of a cluster.  CTA `rank` keeps rows
+// [rank * rpc, rank * rpc + rpc) of T column groups in its shared memory exactly as
+// fused_rounds_kernel keeps all of them, a thread still owns one column group, and the peer's
+// value -- the same column group of a row that may live in another CTA of the cluster -- is read
+// through distributed shared memory (mapa + ld.shared::cluster: plain loads, no multicast).  All
+// CTAs of a cluster advance round by round: a cluster barrier (the hardware's
+// barrier.cluster, not a spin) ends every round, which orders this round's remote reads of a slab
+// before the next round's writes to it and keeps a CTA's shared memory alive while others read it.
+// The consensus statistic needs the column sums over ALL rows: every CTA measures its rows against
+// the common pivot (row 0 of the tile, read from rank 0), sum (x - a)^2 adds up CTA by CTA like
+// the loss does, and the per-column sums of (x - a) go to a small double-buffered exchange area
+// that rank 0 collects after the barrier.  Prefetch, direct store of the last round and the
+// arithmetic are fused_rounds_kernel's, so replicas agree with every other launch shape bit for bit.
+struct ClusterParams {
+  FusedParams f;       // n_tiles: tiles of blockDim column groups
+  int32_t rpc;         // rows per CTA = ceil(M / cluster size)
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+// All threads of all CTAs of the cluster; release / acquire order shared-memory accesses across it.
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// 16 bytes at the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ ulonglong2 ld_cluster_16(uint32_t smem_addr, uint32_t rank) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_addr), "r"(rank));
+  ulonglong2 v;
+  asm volatile("ld.shared::cluster.v2.u64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "r"(remote) : "memory");
+  return v;
+}
+
+// Dynamic shared memory: (peer's local row offset, peer's CTA, -weight, -weight) int4[kFusedMaxRounds][rpc],
+// then the slabs float4[3][rpc][blockDim], then the exchange area float4[2][blockDim], then 64 doubles.
+template <int kObjective, bool kFastNoise>
+__global__ void __launch_bounds__(256, 2) cluster_rounds_kernel(const ClusterParams cp) {
+  const FusedParams& p = cp.f;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int tid = threadIdx.x, T = blockDim.x, M = p.M, rpc = cp.rpc;
+  const uint32_t rank = cluster_ctarank(), C = cluster_nctarank();
+  const int r0 = min(M, (int)rank * rpc), rows = min(M, r0 + rpc) - r0;  // this CTA's rows [r0, r0 + rows)
+  int4* s_pw = reinterpret_cast<int4*>(smem_raw);
+  const uint32_t head = ((uint32_t)(kFusedMaxRounds * rpc * 16) + 127u) & ~127u;
+  const uint32_t stride = (uint32_t)T * 16u;
+  const uint32_t plane = (uint32_t)rpc * stride;
+  unsigned char* slab = smem_raw + head + (uint32_t)tid * 16u;
+  float4* s_xchg = reinterpret_cast<float4*>(smem_raw + head + 3u * plane);  // [2][T] column sums of (x - pivot) over this CTA's rows
+  double* s_red = reinterpret_cast<double*>(smem_raw + head + 3u * plane + 2u * stride);
+  const uint32_t slab_addr = (uint32_t)__cvta_generic_to_shared(slab);
+  const uint32_t xchg_addr = (uint32_t)__cvta_generic_to_shared(s_xchg + tid);
+
+  for (int k = 0; k < p.n_rounds; ++k) {
+    const int32_t* peers = p.trace + ((p.slot0 + k) % p.ring) * M;
+    for (int j = tid; j < rows; j += T) {
+      const int i = r0 + j;
+      const int32_t m = __ldg(peers + i);
+      const int nw = __float_as_int((m == i) ? -0.0f : -__ldg(p.wtab + (size_t)i * M + m));
+      const int pm = m / rpc;
+      s_pw[k * rpc + j] = make_int4((int)((uint32_t)(m - pm * rpc) * stride), pm, nw, nw);
+    }
+  }
+  __syncthreads();
+
+  double acc_cons[kFusedMaxRounds], acc_loss[kFusedMaxRounds];
+#pragma unroll
+  for (int k = 0; k < kFusedMaxRounds; ++k) acc_cons[k] = acc_loss[k] = 0.0;
+
+  const int64_t n_clusters = gridDim.x / C, cluster_id = blockIdx.x / C;
+  const uint64_t row0_bytes = (uint64_t)(uint32_t)r0 * p.row_bytes;
+  uint32_t base = 0;
+  bool fetched = false;
+  uint32_t epoch = 0;  // rounds done by this cluster: parity selects the exchange buffer
+  // every CTA of a cluster runs the same tiles and rounds, so all of them meet at every barrier
+  for (int64_t tile = cluster_id; tile < p.n_tiles; tile += n_clusters) {
+    const int64_t q = tile * T + tid;
+    const bool live = q < p.nq;
+    const NoiseLanes ns = noise_lanes(p.sigma, live_lanes((p.tail != 0) && (q == p.nq - 1), p.tail, 0));
+    const uint32_t q32 = (uint32_t)q + p.q_offset;
+    const int64_t q_next = q + n_clusters * T;
+    const bool tile_has_next = NETMAX_FUSED_PREFETCH != 0 && tile + n_clusters < p.n_tiles;  // the same in every CTA of the cluster
+    const bool have_next = tile_has_next && q_next < p.nq;
+    if (!fetched && live) {
+      const char* xq = reinterpret_cast<const char*>(p.x_cur) + row0_bytes + (uint64_t)q * 16u;
+      const char* cq = reinterpret_cast<const char*>(p.c) + row0_bytes + (uint64_t)q * 16u;
+      unsigned char* sx = slab + base * plane;
+      unsigned char* sc = slab + 2u * plane;
+#pragma unroll 4
+      for (int j = 0; j < rows; ++j) {
+        *reinterpret_cast<ulonglong2*>(sx) = __ldg(reinterpret_cast<const ulonglong2*>(xq));
+        *reinterpret_cast<ulonglong2*>(sc) = __ldg(reinterpret_cast<const ulonglong2*>(cq));
+        xq += p.row_bytes;
+        cq += p.row_bytes;
+        sx += stride;
+        sc += stride;
+      }
+    }
+    // every CTA's rows of the tile are in place before anyone pulls from them (a fetched tile was
+    // published by the barrier that ended its predecessor's last round)
+    if (!fetched) cluster_barrier();
+    unsigned char* const cen = slab + 2u * plane;
+    char* const oq = reinterpret_cast<char*>(p.x_nxt) + row0_bytes + (uint64_t)q * 16u;
+    const char* const cq_next = reinterpret_cast<const char*>(p.c) + row0_bytes + (uint64_t)q_next * 16u;
+
+    auto run_round = [&](int k, auto last_tag) {
+      constexpr bool kLast = decltype(last_tag)::value;
+      const uint64_t round = p.first_round + (uint64_t)k;
+      const uint32_t round_lo = (uint32_t)round, ctr3 = philox_ctr3(kTagNoise, round);
+      const uint32_t cur_off = ((base + (uint32_t)k) & 1u) * plane;
+      const unsigned char* cur = slab + cur_off;
+      unsigned char* nxt = slab + ((base + (uint32_t)k + 1u) & 1u) * plane;
+      if (kLast && have_next) {
+        const char* xq = reinterpret_cast<const char*>(p.x_cur) + row0_bytes + (uint64_t)q_next * 16u;
+        unsigned char* sx = nxt;
+#pragma unroll 4
+        for (int j = 0; j < rows; ++j) {
+          cp_async_16_stream(sx, xq);
+          xq += p.row_bytes;
+          sx += stride;
+        }
+      }
+      ColAcc acc;
+      LossAcc lacc;
+      if (live) {
+        const int4* pw = s_pw + k * rpc;
+        const ulonglong2 pivot = ld_cluster_16(slab_addr + cur_off, 0u);  // row 0 of the tile lives in CTA 0
+        uint32_t off = 0;
+        uint64_t goff = 0;
+        auto pull = [&](int j) {  // the peer's value for local row j, from whichever CTA holds that row
+          const int4 d = pw[j];
+          return ld_cluster_16(slab_addr + cur_off + (uint32_t)d.x, (uint32_t)d.y);
+        };
+        auto do_row = [&](int j, uint4 rnd, ulonglong2 xm) {
+          const int4 d = pw[j];
+          const pair_t nw2 = ((pair_t)(uint32_t)d.w << 32) | (uint32_t)d.z;
+          const ulonglong2 o = row_update_rnd<kObjective, kFastNoise>(p.alpha, ns, rnd, *reinterpret_cast<const ulonglong2*>(cur + off),
+                                                                      *reinterpret_cast<const ulonglong2*>(cen + off), xm, pivot, nw2, acc,
+                                                                      lacc);
+          if (kLast) {
+            *reinterpret_cast<ulonglong2*>(oq + goff) = o;
+            if (have_next) cp_async_16_stream(cen + off, cq_next + goff);
+            goff += p.row_bytes;
+          } else {
+            *reinterpret_cast<ulonglong2*>(nxt + off) = o;
+          }
+          off += stride;
+        };
+        if (rows > 0) {
+          // one row ahead: the next row's Philox block (integer work that fills this row's latencies) and
+          // its pull, whose trip through the cluster's shared-memory network takes several hundred cycles
+          // (two rows ahead measured slower: 1.43 against 1.39 ms per round of 64 x 11.2 M elements)
+          uint4 rnd = noise_block<kObjective>(p.keys, round_lo, ctr3, q32, (uint32_t)r0);
+          ulonglong2 xm = pull(0);
+#pragma unroll kFusedUnroll
+          for (int j = 0; j + 1 < rows; ++j) {
+            const ulonglong2 xm_next = pull(j + 1);
+            const uint4 rnd_next = noise_block<kObjective>(p.keys, round_lo, ctr3, q32, (uint32_t)(r0 + j + 1));
+            do_row(j, rnd, xm);
+            rnd = rnd_next;
+            xm = xm_next;
+          }
+          do_row(rows - 1, rnd, xm);
+        }
+      }
+      float4 s1, s2;
+      unpack2(acc.s1a, s1.x, s1.y);
+      unpack2(acc.s1b, s1.z, s1.w);
+      unpack2(acc.s2a, s2.x, s2.y);
+      unpack2(acc.s2b, s2.z, s2.w);
+      float l0, l1, l2, l3;
+      unpack2(lacc.la, l0, l1);
+      unpack2(lacc.lb, l2, l3);
+      const uint32_t buf = epoch & 1u;
+      s_xchg[buf * T + tid] = s1;
+      if (kLast) cp_async_wait_all();  // the next tile's rows have landed: the barrier below publishes them too
+      cluster_barrier();  // the round is complete everywhere; the column sums of all CTAs are published
+      ++epoch;
+      double cons = (double)((s2.x + s2.y) + (s2.z + s2.w));  // this CTA's share of sum (x - a)^2
+      if (rank == 0) {
+        // sum_i (x_i - xbar)^2 = sum_i (x_i - a)^2 - (sum_i (x_i - a))^2 / M per column: rank 0 subtracts the second term
+        float4 tot = s1;
+        for (uint32_t r = 1; r < C; ++r) {
+          const ulonglong2 v = ld_cluster_16(xchg_addr + buf * stride, r);
+          float a, b, c2, d2;
+          unpack2(v.x, a, b);
+          unpack2(v.y, c2, d2);
+          tot.x += a;
+          tot.y += b;
+          tot.z += c2;
+          tot.w += d2;
+        }
+        cons -= (double)((tot.x * tot.x + tot.y * tot.y + tot.z * tot.z + tot.w * tot.w) * p.inv_M);
+      }
+      const double loss = (double)((l0 + l1) + (l2 + l3));
+#pragma unroll
+      for (int kk = 0; kk < kFusedMaxRounds; ++kk) {
+        if (kk == k) {
+          acc_cons[kk] += cons;
+          acc_loss[kk] += loss;
+        }
+      }
+    };
+    for (int k = 0; k + 1 < p.n_rounds; ++k) run_round(k, std::false_type());
+    run_round(p.n_rounds - 1, std::true_type());
+    base = (base + (uint32_t)p.n_rounds) & 1u;
+    fetched = tile_has_next;
+  }
+  cluster_barrier();  // no CTA leaves while another may still read its exchange area
+
+#pragma unroll
+  for (int k = 0; k < kFusedMaxRounds; ++k)
+    if (k < p.n_rounds) block_partials(p.partials + (size_t)k * 2 * gridDim.x, acc_cons[k], acc_loss[k], s_red);
+  __shared__ bool s_last;
+  if (tid == 0) {
+    __threadfence();
+    const unsigned int t = atomicAdd(p.ticket, 1u);
+    s_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    for (int k = 0; k < p.n_rounds; ++k)
+      sum_partials(p.partials + (size_t)k * 2 * gridDim.x, (double)p.inv_M, p.tel + 2 * ((p.slot0 + k) % p.ring), s_red);
+    if (tid == 0) *p.ticket = 0u;
+  }
+}
+
 // ---- all rounds of a call over resident columns (short vectors) -------------------------------
 // The same independence of columns serves the opposite shape: when the whole problem is a few
 // megabytes, a round takes microseconds and what costs time is every launch and every grid-wide

@@ -79,6 +79,55 @@ def test_fused_rounds_change_no_bit(nm, M, d, fuse, storage, objective):
     many.close()
 
 
+# more workers than a thread's slab holds: the rows of a tile are split over the CTAs of a cluster
+@pytest.mark.parametrize("M,d,fuse", [(64, 80_003, 0), (20, 303_201, 0), (33, 152_002, 3), (100, 38_001, 0), (136, 40_001, 2),
+                                      (19, 310_000, 4)])
+@pytest.mark.parametrize("objective", [0, 1])
+def test_cluster_resident_rounds_change_no_bit(nm, M, d, fuse, objective):
+    rng = np.random.default_rng(M * 7 + d)
+    P = random_policy(M, rng, zeros=0.3)
+    kw = dict(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=objective, seed=d + M, trace_rounds=64)
+    one = nm.Netmax(fuse_rounds=1, **kw)
+    many = nm.Netmax(fuse_rounds=fuse, **kw)
+    rounds = 0
+    for n in (9, 1, 2, 4, 3):
+        launches = many.kernel_launches
+        one.round(n)
+        many.round(n)
+        rounds += n
+        if n >= 2:
+            assert many.kernel_launches - launches < n + 1, "rounds were not fused"
+    assert (one.read_replicas().view(np.uint32) == many.read_replicas().view(np.uint32)).all()
+    assert (one.peer_trace(0, rounds) == many.peer_trace(0, rounds)).all()
+    (ca, la), (cb, lb) = one.telemetry(0, rounds), many.telemetry(0, rounds)
+    np.testing.assert_allclose(cb, ca, rtol=2e-6)      # the column sums are added CTA by CTA here: fp32 rounding of partial sums
+    np.testing.assert_allclose(lb, la, rtol=1e-6)
+    one.close()
+    many.close()
+
+
+def test_cluster_resident_rounds_match_the_oracle(nm):
+    M, d = 64, 80_003
+    rng = np.random.default_rng(M + d)
+    P = random_policy(M, rng, zeros=0.2)
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=1, seed=7, trace_rounds=32)
+    o = oracle.Sim(M, d, P, full_adj(M), alpha=0.05, rho=g.get_policy()[1], sigma=0.1, objective=1, seed=7)
+    o.init(1.0, 1.0)
+    rounds = 10
+    launches = g.kernel_launches
+    g.round(rounds)
+    assert g.kernel_launches - launches <= 1 + (rounds + 3) // 4
+    o.round(rounds, threads=8)
+    assert (g.peer_trace() == o.trace()).all()
+    got, want = g.read_replicas().astype(np.float64), o.x().astype(np.float64)
+    assert (np.abs(got - want) <= TOL * (1.0 + np.abs(want))).all()
+    gc, gl = g.telemetry()
+    oc, ol = o.telemetry()
+    np.testing.assert_allclose(gc, oc, rtol=1e-4)
+    np.testing.assert_allclose(gl, ol, rtol=1e-4)
+    g.close()
+
+
 @pytest.mark.parametrize("M,d", [(3, 400_003), (8, 303_107)])
 def test_fused_rounds_match_the_oracle(nm, M, d):
     rng = np.random.default_rng(M + d)
