@@ -440,25 +440,31 @@ def run_ours(args, w):
     lib = binding.lib()
     assert lib.netmax_read_centres(g._h, hc.data_ptr()) == 0
 
-    def e2e_step():
+    def e2e_step():           # the public call for a step through host buffers: upload, one round, download, pipelined by columns
+        g.round_from_host(hx.data_ptr(), hc.data_ptr(), 1, ho.data_ptr(), args.e2e_chunks)
+
+    def e2e_step_serial():    # the same through the four separate calls, one after the other
         g.set_replicas(hx.data_ptr())
         g.set_centres(hc.data_ptr())
         g.round(1)
         g.read_replicas(ho.data_ptr())
 
-    for _ in range(2):
-        e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    with torch.cuda.stream(stream):
-        start.record()
-    for _ in range(e2e_steps):
-        e2e_step()
-    with torch.cuda.stream(stream):
-        stop.record()
-    stop.synchronize()
-    e2e_ms = start.elapsed_time(stop)
-    e2e_wall = time.perf_counter() - t0
+    def time_e2e(step):
+        for _ in range(2):
+            step()
+        barrier()
+        t0 = time.perf_counter()
+        with torch.cuda.stream(stream):
+            start.record()
+        for _ in range(e2e_steps):
+            step()
+        with torch.cuda.stream(stream):
+            stop.record()
+        stop.synchronize()
+        return start.elapsed_time(stop), time.perf_counter() - t0
+
+    e2e_serial_ms, _ = time_e2e(e2e_step_serial)
+    e2e_ms, e2e_wall = time_e2e(e2e_step)
     if world > 1:
         tmax = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
@@ -510,7 +516,8 @@ def run_ours(args, w):
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": 2 * elements * 4,
                 "d2h_bytes_per_step": elements * 4, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
-                "wall_ms_per_step": e2e_wall * 1e3 / e2e_steps},
+                "wall_ms_per_step": e2e_wall * 1e3 / e2e_steps, "call": "netmax_round_from_host (column chunks pipelined)",
+                "ms_per_step_four_separate_calls": e2e_serial_ms / e2e_steps},
         "gpu_launches": int(launches),
         "clocks": clocks.summary(),
         "telemetry_last_round": {"consensus": float(cons[0]), "loss": float(loss[0])},
@@ -621,6 +628,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", help="cfg1..cfg5 (default: the ResNet18-sized cfg2)")
     ap.add_argument("--d", type=int, default=0, help="override the workload's vector length (profiling on a smaller case)")
     ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--e2e-chunks", type=int, default=0, help="column chunks of the pipelined host round trip (0: automatic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--configs", default="all",
                     help="one GPU: which of cfg1..cfg5 to time into the line's `configs` (all, none, or e.g. 3,4)")

@@ -181,6 +181,21 @@ int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
  */
 int netmax_round(netmax_ctx* ctx, int64_t n_rounds);
 
+/*
+ * A whole step through host buffers in one call: replaces the replicas by host_x and the centres by
+ * host_c (either may be NULL: keep what the context holds), runs n_rounds rounds and copies the
+ * resulting replicas to host_out -- what netmax_set_replicas, netmax_set_centres, netmax_round and
+ * netmax_read_replicas do one after the other, with the same replicas, peer trace, telemetry and
+ * round counter bit for bit.  Given the draws, Eq. 15-16 act on every column separately, so the work
+ * is cut into n_chunks column ranges (0: automatic; at most 32) and pipelined: while the rounds of
+ * one range run on the context's stream, the next range is uploaded and the previous one downloaded
+ * on two streams of the library's own.  All arrays are dense M*d floats on the host; pinned memory
+ * lets the copies overlap.  Ranges are pipelined for fp32 state, long vectors and
+ * 1 <= n_rounds <= trace_rounds; otherwise the call runs the four steps in turn.  Synchronises.
+ */
+int netmax_round_from_host(netmax_ctx* ctx, const float* host_x, const float* host_c, int64_t n_rounds, float* host_out,
+                           int32_t n_chunks);
+
 /* Changes netmax_config.fuse_rounds for the rounds that follow (0 automatic, 1 one launch per
  * round, 2..4 at most that many rounds per launch). */
 int netmax_set_fuse_rounds(netmax_ctx* ctx, int32_t fuse_rounds);

@@ -21,6 +21,7 @@ STATUS = {0: "OK", -1: "INVALID_ARG", -2: "BAD_PROB_ROW", -3: "OOM", -4: "CUDA_E
 EXPORTS = [
     "netmax_config_init", "netmax_workspace_size", "netmax_create_ex", "netmax_create", "netmax_destroy",
     "netmax_set_policy", "netmax_get_policy", "netmax_set_replicas", "netmax_set_centres", "netmax_round",
+    "netmax_round_from_host",
     "netmax_rounds_done", "netmax_set_fuse_rounds", "netmax_read_replicas", "netmax_read_centres", "netmax_read_columns",
     "netmax_read_columns_static",
     "netmax_peer_trace", "netmax_telemetry", "netmax_replicas_device", "netmax_sample_peers",
@@ -76,6 +77,7 @@ def lib():
             "netmax_set_replicas": ([vp, vp], C.c_int),
             "netmax_set_centres": ([vp, vp], C.c_int),
             "netmax_round": ([vp, i64], C.c_int),
+            "netmax_round_from_host": ([vp, vp, vp, i64, vp, i32], C.c_int),
             "netmax_rounds_done": ([vp], i64),
             "netmax_set_fuse_rounds": ([vp, i32], C.c_int),
             "netmax_read_replicas": ([vp, vp], C.c_int),
@@ -277,6 +279,19 @@ class Netmax:
 
     def round(self, n_rounds: int = 1):
         _check(lib().netmax_round(self._h, int(n_rounds)), self._h)
+
+    def round_from_host(self, x, c, n_rounds: int, out, n_chunks: int = 0):
+        """netmax_round_from_host: x, c, out are numpy arrays (M, d) float32 or host pointers (int); x and c may be None."""
+        def ptr(a):
+            return None if a is None else self._host_plane(a)
+        keep = [ptr(x), ptr(c)]
+        if isinstance(out, int):
+            po = C.c_void_p(out)
+        else:
+            assert out.dtype == np.float32 and out.shape == (self.M, self.d) and out.flags.c_contiguous
+            po = _p(out)
+        _check(lib().netmax_round_from_host(self._h, keep[0], keep[1], int(n_rounds), po, int(n_chunks)), self._h)
+        return out
 
     def set_fuse_rounds(self, fuse_rounds: int):
         _check(lib().netmax_set_fuse_rounds(self._h, int(fuse_rounds)), self._h)

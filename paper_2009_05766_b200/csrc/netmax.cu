@@ -71,12 +71,13 @@ struct Layout {
   int elem = 4, halves = 1;         // bytes per stored element; Philox blocks (4 elements) per column group
   size_t plane = 0;                 // bytes of one [M][ld] array
   size_t off_x0 = 0, off_x1 = 0, off_c = 0, off_thr = 0, off_last = 0, off_w = 0, off_trace = 0, off_wring = 0, off_tel = 0,
-         off_partials = 0, off_ticket = 0, off_colpart = 0, off_coltick = 0, total = 0;
+         off_partials = 0, off_ticket = 0, off_colpart = 0, off_coltick = 0, off_pipe_tel = 0, total = 0;
 };
 
 constexpr int kMaxGrid = 148 * 16;  // upper bound on resident CTAs of the round kernel
 constexpr int64_t kMaxRoundsPerLaunch = 4096;  // rounds one cooperative launch runs at most
 constexpr size_t kColPartBytes = (size_t)8 << 20;  // column partials of the row-split (short vector) shape
+constexpr int kMaxChunks = 32;  // column chunks of a pipelined host round trip
 
 Layout make_layout(int64_t M, int64_t d, int64_t trace_rounds, int storage) {
   Layout L;
@@ -103,6 +104,7 @@ Layout make_layout(int64_t M, int64_t d, int64_t trace_rounds, int storage) {
   L.off_ticket = take(256);
   L.off_colpart = take(kColPartBytes);
   L.off_coltick = take((size_t)kMaxGrid * sizeof(unsigned int));
+  L.off_pipe_tel = take((size_t)kMaxChunks * trace_rounds * 2 * sizeof(double));  // per-chunk telemetry of a pipelined round trip
   L.total = o;
   return L;
 }
@@ -164,6 +166,8 @@ struct netmax_ctx {
   std::vector<int64_t> ev_n;
   std::vector<double> ev_time;
   unsigned int* coltick = nullptr;
+  double* pipe_tel = nullptr;                      // [kMaxChunks][trace_rounds][2]
+  cudaStream_t up_stream = nullptr, down_stream = nullptr;  // host round trips: uploads and downloads beside the context's stream
   int cur = 0;  // index of the buffer holding the current replicas
   int64_t rounds = 0;  // number of the next round (absolute)
   int64_t round0 = 0;  // number of the context's first round
@@ -762,6 +766,141 @@ int plan_cluster(netmax_ctx* ctx, const RoundPlan& plan, const FusedPlan& fused,
   return rc;
 }
 
+// What every launch of the round kernels shares: buffers, tile shape, step sizes, keys.
+RoundParams make_round_params(const netmax_ctx* ctx, const RoundPlan& plan) {
+  RoundParams p;
+  std::memset(&p, 0, sizeof p);
+  p.c = reinterpret_cast<const float4*>(ctx->c);
+  p.wtab = ctx->wtab;
+  p.partials = ctx->partials;
+  p.ticket = ctx->ticket;
+  p.ldq = ctx->L.ldq;
+  p.row_bytes = (uint32_t)(ctx->L.ld * ctx->L.elem);
+  p.nq = ctx->L.nq;
+  p.n_tiles = plan.n_tiles;
+  p.M = ctx->M;
+  p.tail = (int32_t)(ctx->d % (4 * ctx->L.halves));
+  p.cg = plan.cg;
+  p.rl = plan.rl;
+  p.rg = plan.rg;
+  p.rows_per_group = plan.rows_per_group;
+  p.colpart = ctx->colpart;
+  p.coltick = ctx->coltick;
+  p.alpha = (float)ctx->alpha;
+  p.sigma = noise_scale(ctx);
+  p.inv_M = 1.0f / (float)ctx->M;
+  p.q_offset = ctx->q_offset;
+  p.keys = ctx->keys;
+  return p;
+}
+
+// A range of column groups (four fp32 elements each) of every replica: the whole vector, or one
+// chunk of a pipelined host round trip.  Given the draws, columns evolve independently, so the
+// kernels run on a range exactly as on the whole: shifted base pointers, the range's group count,
+// and the Philox block offset moved along.
+struct ColumnRange {
+  int64_t q0 = 0, nq4 = 0;  // first group and number of groups (four elements each)
+  int32_t tail4 = 0;        // live elements of the range's last group (0: all four); non-zero only at the end of the rows
+  bool whole = true;        // the whole vector (the only form bfloat16 state takes)
+};
+
+// Enqueues rounds [first, first + n) -- their draws are in the trace ring -- for one column range on
+// `stream`: up to four rounds per launch where tiles stay resident (fused_rounds_kernel, or
+// cluster_rounds_kernel for more workers), else one launch per round.  `cur` is the buffer that holds
+// the range's values at round `first`; it is flipped launch by launch.  Telemetry of the range goes
+// to tel (ring-indexed like the context's).
+int launch_long_rounds(netmax_ctx* ctx, cudaStream_t stream, const RoundPlan& plan, const FusedPlan& fused,
+                       const ClusterPlan& cluster, RoundParams p, const ColumnRange& range, double* tel, uint64_t first,
+                       int64_t n, int& cur) {
+  RoundKernel kernel = pick_kernel(ctx->objective, plan.short_vectors, ctx->L.halves);
+  const size_t shift = range.whole ? 0 : (size_t)range.q0 * 16;  // bytes into every row (fp32 state when not whole)
+  const unsigned char* cbase = ctx->c + shift;
+  if (!range.whole) {
+    p.nq = range.nq4;
+    p.n_tiles = (range.nq4 + plan.cg - 1) / plan.cg * plan.rg;
+    p.tail = range.tail4;
+    p.q_offset = ctx->q_offset + (uint32_t)range.q0;
+    p.c = reinterpret_cast<const float4*>(cbase);
+  }
+  const int round_grid = (int)std::min<int64_t>(plan.grid, p.n_tiles);
+  uint64_t r = first;
+  for (int64_t b = 0; b < n;) {
+    const unsigned char* xin = ctx->x[cur] + shift;
+    unsigned char* xout = ctx->x[cur ^ 1] + shift;
+    if ((fused.ok || cluster.ok) && n - b >= 2) {  // the next rounds in one launch over resident tiles
+      const int chunk = (int)std::min<int64_t>(n - b, fused.ok ? fused.max_rounds : cluster.max_rounds);
+      const int threads = fused.ok ? fused.threads : cluster.threads;
+      FusedParams fp;
+      fp.x_cur = reinterpret_cast<const float4*>(xin);
+      fp.x_nxt = reinterpret_cast<float4*>(xout);
+      fp.c = reinterpret_cast<const float4*>(cbase);
+      fp.trace = ctx->trace;
+      fp.wtab = ctx->wtab;
+      fp.tel = tel;
+      fp.partials = ctx->partials;
+      fp.ticket = ctx->ticket;
+      fp.slot0 = (int64_t)(r % (uint64_t)ctx->trace_rounds);
+      fp.ring = ctx->trace_rounds;
+      fp.first_round = r;
+      fp.n_rounds = chunk;
+      fp.nq = range.nq4;
+      fp.n_tiles = (range.nq4 + threads - 1) / threads;
+      fp.row_bytes = p.row_bytes;
+      fp.M = p.M;
+      fp.tail = range.tail4;
+      fp.alpha = p.alpha;
+      fp.sigma = p.sigma;
+      fp.inv_M = p.inv_M;
+      fp.q_offset = ctx->q_offset + (uint32_t)range.q0;
+      fp.keys = p.keys;
+      if (!fused.ok) {  // rows split over the CTAs of a cluster
+        ClusterParams cpar;
+        cpar.f = fp;
+        cpar.rpc = cluster.rpc;
+        ClusterKernel ck = pick_cluster_kernel(ctx->objective);
+        NM_CUDA(ctx, cudaFuncSetAttribute(ck, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cluster.smem));
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3((unsigned)(std::min<int64_t>(cluster.grid / cluster.C, fp.n_tiles) * cluster.C));
+        lc.blockDim = dim3((unsigned)cluster.threads);
+        lc.dynamicSmemBytes = cluster.smem;
+        lc.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = (unsigned)cluster.C;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        lc.attrs = &attr;
+        lc.numAttrs = 1;
+        NM_CUDA(ctx, cudaLaunchKernelEx(&lc, ck, cpar));
+      } else {
+        // (the attribute belongs to the kernel, not to this context: another context may have lowered it)
+        FusedKernel fk = pick_fused_kernel(ctx->objective, ctx->L.halves);
+        NM_CUDA(ctx, cudaFuncSetAttribute(fk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fused.smem));
+        fk<<<(unsigned)std::min<int64_t>(fused.grid, fp.n_tiles), fused.threads, fused.smem, stream>>>(fp);
+      }
+      ctx->launches += 1;
+      cur ^= 1;
+      r += (uint64_t)chunk;
+      b += chunk;
+      continue;
+    }
+    const int64_t slot = (int64_t)(r % (uint64_t)ctx->trace_rounds);
+    p.x_cur = reinterpret_cast<const float4*>(xin);
+    p.x_nxt = reinterpret_cast<float4*>(xout);
+    p.peers = ctx->trace + slot * ctx->M;
+    p.tel_out = tel + 2 * slot;
+    p.round_lo = (uint32_t)r;
+    p.ctr3 = philox_ctr3(kTagNoise, r);
+    kernel<<<round_grid, kThreads, plan.smem, stream>>>(p);
+    ctx->launches += 1;
+    cur ^= 1;
+    r += 1;
+    b += 1;
+  }
+  NM_CUDA(ctx, cudaGetLastError());
+  return NETMAX_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -902,6 +1041,7 @@ int netmax_create_ex(const netmax_config* cfg, netmax_ctx** out) {
   ctx->dev_error = ctx->ticket + 32;
   ctx->measure_out = (double*)(ctx->ticket + 48);
   ctx->coltick = (unsigned int*)(ctx->base + L.off_coltick);
+  ctx->pipe_tel = (double*)(ctx->base + L.off_pipe_tel);
 
   auto step = [&](cudaError_t e, const char* what) {
     if (e == cudaSuccess) return true;
@@ -942,6 +1082,12 @@ int netmax_create(int32_t M, int64_t d, const double* link_speed_gbps, const dou
 
 void netmax_destroy(netmax_ctx* ctx) {
   if (!ctx) return;
+  if (ctx->up_stream || ctx->down_stream) {
+    DeviceGuard guard(ctx->device);
+    if (ctx->up_stream) cudaStreamDestroy(ctx->up_stream);
+    if (ctx->down_stream) cudaStreamDestroy(ctx->down_stream);
+    cudaGetLastError();
+  }
   if (ctx->own_memory && ctx->base) {
     DeviceGuard guard(ctx->device);
     cudaStreamSynchronize(ctx->stream);
@@ -1063,7 +1209,6 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   RoundPlan plan;
   int rc = plan_round(ctx, plan, ctx->objective);
   if (rc) return rc;
-  RoundKernel kernel = pick_kernel(ctx->objective, plan.short_vectors, ctx->L.halves);
   FusedPlan fused;
   rc = plan_fused(ctx, plan, fused);
   if (rc) return rc;
@@ -1075,28 +1220,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
   rc = plan_cluster(ctx, plan, fused, cluster);
   if (rc) return rc;
 
-  RoundParams p;
-  p.c = reinterpret_cast<const float4*>(ctx->c);
-  p.wtab = ctx->wtab;
-  p.partials = ctx->partials;
-  p.ticket = ctx->ticket;
-  p.ldq = ctx->L.ldq;
-  p.row_bytes = (uint32_t)(ctx->L.ld * ctx->L.elem);
-  p.nq = ctx->L.nq;
-  p.n_tiles = plan.n_tiles;
-  p.M = ctx->M;
-  p.tail = (int32_t)(ctx->d % (4 * ctx->L.halves));
-  p.cg = plan.cg;
-  p.rl = plan.rl;
-  p.rg = plan.rg;
-  p.rows_per_group = plan.rows_per_group;
-  p.colpart = ctx->colpart;
-  p.coltick = ctx->coltick;
-  p.alpha = (float)ctx->alpha;
-  p.sigma = noise_scale(ctx);
-  p.inv_M = 1.0f / (float)ctx->M;
-  p.q_offset = ctx->q_offset;
-  p.keys = ctx->keys;
+  RoundParams p = make_round_params(ctx, plan);
 
   int64_t done = 0;
   while (done < n_rounds) {
@@ -1184,80 +1308,17 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
       done += batch;
       continue;
     }
-    for (int64_t b = 0; b < batch;) {
-      if ((fused.ok || cluster.ok) && batch - b >= 2) {  // the next rounds in one launch over resident tiles
-        const int chunk = (int)std::min<int64_t>(batch - b, fused.ok ? fused.max_rounds : cluster.max_rounds);
-        FusedParams fp;
-        fp.x_cur = reinterpret_cast<const float4*>(ctx->x[ctx->cur]);
-        fp.x_nxt = reinterpret_cast<float4*>(ctx->x[ctx->cur ^ 1]);
-        fp.c = p.c;
-        fp.trace = ctx->trace;
-        fp.wtab = ctx->wtab;
-        fp.tel = ctx->tel;
-        fp.partials = ctx->partials;
-        fp.ticket = ctx->ticket;
-        fp.slot0 = ctx->rounds % ctx->trace_rounds;
-        fp.ring = ctx->trace_rounds;
-        fp.first_round = (uint64_t)ctx->rounds;
-        fp.n_rounds = chunk;
-        fp.nq = (ctx->d + 3) / 4;
-        fp.n_tiles = fused.ok ? fused.n_tiles : cluster.n_tiles;
-        fp.row_bytes = p.row_bytes;
-        fp.M = p.M;
-        fp.tail = (int32_t)(ctx->d % 4);
-        fp.alpha = p.alpha;
-        fp.sigma = p.sigma;
-        fp.inv_M = p.inv_M;
-        fp.q_offset = p.q_offset;
-        fp.keys = p.keys;
-        if (!fused.ok) {  // rows split over the CTAs of a cluster
-          ClusterParams cpar;
-          cpar.f = fp;
-          cpar.rpc = cluster.rpc;
-          ClusterKernel ck = pick_cluster_kernel(ctx->objective);
-          NM_CUDA(ctx, cudaFuncSetAttribute(ck, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cluster.smem));
-          cudaLaunchConfig_t lc = {};
-          lc.gridDim = dim3((unsigned)cluster.grid);
-          lc.blockDim = dim3((unsigned)cluster.threads);
-          lc.dynamicSmemBytes = cluster.smem;
-          lc.stream = ctx->stream;
-          cudaLaunchAttribute attr;
-          attr.id = cudaLaunchAttributeClusterDimension;
-          attr.val.clusterDim.x = (unsigned)cluster.C;
-          attr.val.clusterDim.y = 1;
-          attr.val.clusterDim.z = 1;
-          lc.attrs = &attr;
-          lc.numAttrs = 1;
-          NM_CUDA(ctx, cudaLaunchKernelEx(&lc, ck, cpar));
-          ctx->launches += 1;
-          ctx->cur ^= 1;
-          ctx->rounds += chunk;
-          b += chunk;
-          continue;
-        }
-        // (the attribute belongs to the kernel, not to this context: another context may have lowered it)
-        FusedKernel fk = pick_fused_kernel(ctx->objective, ctx->L.halves);
-        NM_CUDA(ctx, cudaFuncSetAttribute(fk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fused.smem));
-        fk<<<fused.grid, fused.threads, fused.smem, ctx->stream>>>(fp);
-        ctx->launches += 1;
-        ctx->cur ^= 1;
-        ctx->rounds += chunk;
-        b += chunk;
-        continue;
-      }
-      const uint64_t r = (uint64_t)ctx->rounds;
-      const int64_t slot = (int64_t)(r % (uint64_t)ctx->trace_rounds);
-      p.x_cur = reinterpret_cast<const float4*>(ctx->x[ctx->cur]);
-      p.x_nxt = reinterpret_cast<float4*>(ctx->x[ctx->cur ^ 1]);
-      p.peers = ctx->trace + slot * ctx->M;
-      p.tel_out = ctx->tel + 2 * slot;
-      p.round_lo = (uint32_t)r;
-      p.ctr3 = philox_ctr3(kTagNoise, r);
-      kernel<<<plan.grid, kThreads, plan.smem, ctx->stream>>>(p);
-      ctx->launches += 1;
-      ctx->cur ^= 1;
-      ctx->rounds += 1;
-      b += 1;
+    {  // long vectors: fused, cluster-resident or one launch per round, over all columns
+      ColumnRange all;
+      all.q0 = 0;
+      all.nq4 = (ctx->d + 3) / 4;
+      all.tail4 = (int32_t)(ctx->d % 4);
+      all.whole = true;
+      int cur = ctx->cur;
+      rc = launch_long_rounds(ctx, ctx->stream, plan, fused, cluster, p, all, ctx->tel, (uint64_t)ctx->rounds, batch, cur);
+      if (rc) return rc;
+      ctx->cur = cur;
+      ctx->rounds += batch;
     }
     NM_CUDA(ctx, cudaGetLastError());
     done += batch;
@@ -1266,6 +1327,115 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
 }
 
 int64_t netmax_rounds_done(const netmax_ctx* ctx) { return ctx ? ctx->rounds : -1; }
+
+// ---- host round trip, pipelined over column chunks ----------------------------------------------
+int netmax_round_from_host(netmax_ctx* ctx, const float* host_x, const float* host_c, int64_t n_rounds, float* host_out,
+                           int32_t n_chunks) {
+  if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");
+  if (n_rounds < 0) return fail(ctx, NETMAX_INVALID_ARG, "n_rounds = %lld < 0", (long long)n_rounds);
+  if (!host_out) return fail(ctx, NETMAX_INVALID_ARG, "host_out is NULL");
+  if (n_chunks < 0 || n_chunks > kMaxChunks) return fail(ctx, NETMAX_INVALID_ARG, "n_chunks = %d outside [0, %d]", n_chunks, kMaxChunks);
+  if (ctx->async_on) return fail(ctx, NETMAX_INVALID_ARG, "the context runs the asynchronous timeline; use netmax_async_steps");
+  DeviceGuard guard(ctx->device);
+  RoundPlan plan;
+  int rc = plan_round(ctx, plan, ctx->objective);
+  if (rc) return rc;
+  const int64_t nq4 = (ctx->d + 3) / 4;
+  const int64_t unit = 256;  // chunk boundaries on 4 KB of every row
+  int chunks = n_chunks > 0 ? n_chunks : 8;
+  chunks = (int)std::min<int64_t>(chunks, (nq4 + unit - 1) / unit);
+  const bool pipelined = ctx->storage == NETMAX_STORAGE_F32 && !plan.short_vectors && n_rounds >= 1 &&
+                         n_rounds <= ctx->trace_rounds && chunks >= 2 &&
+                         (uint64_t)(ctx->rounds + n_rounds) < ((uint64_t)1 << 56);
+  if (!pipelined) {  // the same three steps one after the other
+    if (host_x) { rc = netmax_set_replicas(ctx, host_x); if (rc) return rc; }
+    if (host_c) { rc = netmax_set_centres(ctx, host_c); if (rc) return rc; }
+    rc = netmax_round(ctx, n_rounds);
+    if (rc) return rc;
+    return netmax_read_replicas(ctx, host_out);
+  }
+  FusedPlan fused;
+  rc = plan_fused(ctx, plan, fused);
+  if (rc) return rc;
+  ClusterPlan cluster;
+  rc = plan_cluster(ctx, plan, fused, cluster);
+  if (rc) return rc;
+  if (!ctx->up_stream) NM_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->up_stream, cudaStreamNonBlocking));
+  if (!ctx->down_stream) NM_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->down_stream, cudaStreamNonBlocking));
+
+  const int64_t per_chunk = ((nq4 + chunks - 1) / chunks + unit - 1) / unit * unit;
+  chunks = (int)((nq4 + per_chunk - 1) / per_chunk);
+  std::vector<cudaEvent_t> events(2 * chunks + 1, nullptr);
+  auto cleanup = [&]() {
+    for (cudaEvent_t e : events)
+      if (e) cudaEventDestroy(e);
+  };
+  for (auto& e : events) {
+    cudaError_t ce = cudaEventCreateWithFlags(&e, cudaEventDisableTiming);
+    if (ce != cudaSuccess) { cleanup(); return fail(ctx, NETMAX_CUDA_ERROR, "cudaEventCreate: %s", cudaGetErrorString(ce)); }
+  }
+  // from here on a failure still has to wait for what is in flight before the events go away
+  auto bail = [&](int code) {
+    cudaStreamSynchronize(ctx->up_stream);
+    cudaStreamSynchronize(ctx->stream);
+    cudaStreamSynchronize(ctx->down_stream);
+    cleanup();
+    return code;
+  };
+#define NM_PIPE(call)                                                                                   \
+  do {                                                                                                  \
+    cudaError_t e_ = (call);                                                                            \
+    if (e_ != cudaSuccess) return bail(fail(ctx, NETMAX_CUDA_ERROR, "%s: %s", #call, cudaGetErrorString(e_))); \
+  } while (0)
+
+  const uint64_t first = (uint64_t)ctx->rounds;
+  rc = launch_sampler(ctx, first, n_rounds, ctx->trace, ctx->wring, ctx->rounds % ctx->trace_rounds, ctx->trace_rounds);
+  if (rc) return bail(rc);
+  // uploads must not overtake earlier work of the context that still reads the buffers
+  NM_PIPE(cudaEventRecord(events[2 * chunks], ctx->stream));
+  NM_PIPE(cudaStreamWaitEvent(ctx->up_stream, events[2 * chunks], 0));
+  const RoundParams p = make_round_params(ctx, plan);
+  const size_t dev_pitch = (size_t)ctx->L.ld * sizeof(float), host_pitch = (size_t)ctx->d * sizeof(float);
+  int cur_end = ctx->cur;
+  for (int k = 0; k < chunks; ++k) {
+    ColumnRange range;
+    range.q0 = (int64_t)k * per_chunk;
+    range.nq4 = std::min<int64_t>(per_chunk, nq4 - range.q0);
+    range.tail4 = (k == chunks - 1) ? (int32_t)(ctx->d % 4) : 0;
+    range.whole = false;
+    const int64_t e0 = range.q0 * 4, cols = std::min<int64_t>(range.nq4 * 4, ctx->d - e0);
+    const size_t width = (size_t)cols * sizeof(float), at = (size_t)e0 * sizeof(float);
+    if (host_x)
+      NM_PIPE(cudaMemcpy2DAsync(ctx->x[ctx->cur] + at, dev_pitch, host_x + e0, host_pitch, width, (size_t)ctx->M,
+                                cudaMemcpyHostToDevice, ctx->up_stream));
+    if (host_c)
+      NM_PIPE(cudaMemcpy2DAsync(ctx->c + at, dev_pitch, host_c + e0, host_pitch, width, (size_t)ctx->M, cudaMemcpyHostToDevice,
+                                ctx->up_stream));
+    NM_PIPE(cudaEventRecord(events[2 * k], ctx->up_stream));
+    NM_PIPE(cudaStreamWaitEvent(ctx->stream, events[2 * k], 0));
+    int cur = ctx->cur;
+    rc = launch_long_rounds(ctx, ctx->stream, plan, fused, cluster, p, range, ctx->pipe_tel + (size_t)k * ctx->trace_rounds * 2,
+                            first, n_rounds, cur);
+    if (rc) return bail(rc);
+    cur_end = cur;
+    NM_PIPE(cudaEventRecord(events[2 * k + 1], ctx->stream));
+    NM_PIPE(cudaStreamWaitEvent(ctx->down_stream, events[2 * k + 1], 0));
+    NM_PIPE(cudaMemcpy2DAsync(host_out + e0, host_pitch, ctx->x[cur_end] + at, dev_pitch, width, (size_t)ctx->M,
+                              cudaMemcpyDeviceToHost, ctx->down_stream));
+  }
+  // the rounds' telemetry: the chunks' shares added in chunk order
+  sum_chunk_telemetry_kernel<<<(unsigned)((n_rounds + kThreads - 1) / kThreads), kThreads, 0, ctx->stream>>>(
+      ctx->pipe_tel, chunks, ctx->trace_rounds, (int64_t)(first % (uint64_t)ctx->trace_rounds), n_rounds, ctx->tel);
+  ctx->launches += 1;
+  NM_PIPE(cudaGetLastError());
+  ctx->cur = cur_end;
+  ctx->rounds += n_rounds;
+  NM_PIPE(cudaStreamSynchronize(ctx->down_stream));
+  NM_PIPE(cudaStreamSynchronize(ctx->stream));
+#undef NM_PIPE
+  cleanup();
+  return check_device_error(ctx);
+}
 
 int netmax_set_fuse_rounds(netmax_ctx* ctx, int32_t fuse_rounds) {
   if (!ctx) return fail(nullptr, NETMAX_INVALID_ARG, "ctx is NULL");

@@ -1346,6 +1346,22 @@ __global__ void __launch_bounds__(256) sum_tile_partials_kernel(const double* pa
   }
 }
 
+// tel[slot of round k] = sum over chunks of chunk_tel[chunk][slot], chunks in order (a pipelined host
+// round trip runs the rounds chunk of columns by chunk; both statistics are sums over columns).
+__global__ void __launch_bounds__(256) sum_chunk_telemetry_kernel(const double* chunk_tel, int32_t n_chunks, int64_t ring,
+                                                                  int64_t slot0, int64_t n_rounds, double* tel) {
+  const int64_t k = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (k >= n_rounds) return;
+  const int64_t slot = (slot0 + k) % ring;
+  double a = 0.0, b = 0.0;
+  for (int c = 0; c < n_chunks; ++c) {
+    a += chunk_tel[((size_t)c * ring + slot) * 2];
+    b += chunk_tel[((size_t)c * ring + slot) * 2 + 1];
+  }
+  tel[2 * slot] = a;
+  tel[2 * slot + 1] = b;
+}
+
 // ------------------------------------------------------------------------- asynchronous steps
 // The paper's own process (Eq. 17): at a global step ONE worker i applies Eq. 15-16 to its
 // replica, in place, with the peer's current replica; every other replica is unchanged.  A
