@@ -386,6 +386,11 @@ __device__ __forceinline__ void cp_async_16_stream(void* smem_dst, const void* g
   const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
 }
+// The same for 8 bytes (four bfloat16 values; copies below 16 bytes go through L1).
+__device__ __forceinline__ void cp_async_8(void* smem_dst, const void* gmem_src) {
+  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 // Loads of replica data.  Inside one launch per round the round-start buffer is read-only
@@ -730,7 +735,9 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
   // of a row replaces the current one as soon as that row has been updated for the last time.  The
   // global loads of a tile thus run under the last round of its predecessor.  Every slab slot is
   // read and written by its own thread only, so cp.async.wait_all is all the synchronisation needed.
-  constexpr bool kPrefetch = !kBf16 && NETMAX_FUSED_PREFETCH != 0;
+  // bfloat16 state arrives as the 8 stored bytes in the low half of a 16-byte slot and is widened in
+  // place when the tile starts.
+  constexpr bool kPrefetch = NETMAX_FUSED_PREFETCH != 0;
   uint32_t base = 0;
   bool fetched = false;  // has this tile been fetched by the previous one?
   for (int64_t tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x) {
@@ -742,6 +749,17 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
     const bool have_next = kPrefetch && tile + gridDim.x < p.n_tiles && q_next < p.nq;
     if (fetched) {
       cp_async_wait_all();
+      if (kBf16) {
+        unsigned char* sx = slab + base * plane;
+        unsigned char* sc = slab + 2u * plane;
+#pragma unroll 4
+        for (int i = 0; i < M; ++i) {
+          *reinterpret_cast<ulonglong2*>(sx) = widen_bf16x4(*reinterpret_cast<const unsigned long long*>(sx));
+          *reinterpret_cast<ulonglong2*>(sc) = widen_bf16x4(*reinterpret_cast<const unsigned long long*>(sc));
+          sx += stride;
+          sc += stride;
+        }
+      }
     } else {  // all rows of this column group into the thread's slabs
       const char* xq = reinterpret_cast<const char*>(p.x_cur) + (uint64_t)q * kGroupBytes;
       const char* cq = reinterpret_cast<const char*>(p.c) + (uint64_t)q * kGroupBytes;
@@ -778,7 +796,8 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
         unsigned char* sx = nxt;
 #pragma unroll 4
         for (int i = 0; i < M; ++i) {
-          cp_async_16_stream(sx, xq);
+          if (kBf16) cp_async_8(sx, xq);
+          else cp_async_16_stream(sx, xq);
           xq += p.row_bytes;
           sx += stride;
         }
@@ -799,7 +818,10 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
         if (kLast) {
           if (kBf16) *reinterpret_cast<unsigned long long*>(oq + goff) = narrow_bf16x4(o);
           else *reinterpret_cast<ulonglong2*>(oq + goff) = o;
-          if (have_next) cp_async_16_stream(cen + off, cq_next + goff);  // this row's centre is not read again in this tile
+          if (have_next) {  // this row's centre is not read again in this tile
+            if (kBf16) cp_async_8(cen + off, cq_next + goff);
+            else cp_async_16_stream(cen + off, cq_next + goff);
+          }
           goff += p.row_bytes;
         } else {
           *reinterpret_cast<ulonglong2*>(nxt + off) = kBf16 ? widen_bf16x4(narrow_bf16x4(o)) : o;
