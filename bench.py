@@ -53,16 +53,29 @@ KERNEL_SOURCES = ("netmax_kernels.cuh", "netmax_rng.cuh")
 # enough to profile, else on the same M and tile shape with a shorter vector (`captured_on`); bytes and
 # instructions per element are what carries over.  Only reported while the kernel sources still hash to
 # the value the capture was taken at.
-NCU_HASH = "f410b991e772e080"
+NCU_HASH = "c9812615affa1170"
 NCU_COUNTERS = {
     # (workload tag, kernel): dram bytes per element-launch, warp instructions per element-round, captured on
-    ("cfg2_M8_resnet18", "round_kernel"): (1_041_924_000 / 89_391_696, None, "cfg2"),
-    ("cfg2_M8_resnet18", "fused_rounds_kernel"): (1_041_056_000 / 89_391_696, 346_883_835 / (89_391_696 * 4), "cfg2"),
-    ("cfg2_M8_resnet18/bf16", "round_kernel"): (505_763_000 / 89_391_696, None, "cfg2"),
-    ("cfg2_M8_resnet18/bf16", "fused_rounds_kernel"): (505_109_000 / 89_391_696, 383_985_067 / (89_391_696 * 4), "cfg2"),
-    ("cfg3_M16_vgg19scale", "fused_rounds_kernel"): (3_806_318_000 / 320_000_000, 1_183_131_797 / (320_000_000 * 4), "cfg3"),
-    ("cfg3_M16_vgg19scale", "round_kernel"): (1_543_900_928 / (16 * 8_000_002), 105_887_357 / (16 * 8_000_002), "cfg3 at d = 8,000,002"),
-    ("cfg4_M64_resnet18", "round_kernel"): (1_532_370_688 / (64 * 2_000_002), 108_627_174 / (64 * 2_000_002), "cfg4 at d = 2,000,002"),
+    ("cfg2_M8_resnet18", "round_kernel"): (1_041_923_000 / 89_391_696, 78_504_733 / 89_391_696, "cfg2"),
+    ("cfg2_M8_resnet18", "fused_rounds_kernel"): (1_040_247_000 / 89_391_696, 314_012_326 / (89_391_696 * 4), "cfg2"),
+    ("cfg2_M8_resnet18/bf16", "round_kernel"): (505_283_000 / 89_391_696, 85_164_099 / 89_391_696, "cfg2"),
+    ("cfg2_M8_resnet18/bf16", "fused_rounds_kernel"): (505_837_000 / 89_391_696, 345_321_682 / (89_391_696 * 4), "cfg2"),
+    ("cfg3_M16_vgg19scale", "fused_rounds_kernel"): (3_804_985_000 / 320_000_000, 1_031_374_061 / (320_000_000 * 4), "cfg3"),
+    ("cfg3_M16_vgg19scale", "round_kernel"): (1_544_190_000 / (16 * 8_000_002), 101_887_293 / (16 * 8_000_002), "cfg3 at d = 8,000,002"),
+    ("cfg4_M64_resnet18", "cluster_rounds_kernel"): (1_504_340_000 / (64 * 2_000_002), 524_126_023 / (64 * 2_000_002 * 4), "cfg4 at d = 2,000,002"),
+    ("cfg4_M64_resnet18", "round_kernel"): (1_545_685_000 / (64 * 2_000_002), 104_626_918 / (64 * 2_000_002), "cfg4 at d = 2,000,002"),
+    ("cfg1_M4_d4096", "resident_rounds_kernel"): (None, 52_552_832 / (16_384 * 1024), "cfg1"),
+    ("cfg5_M4096_sampling", "resident_rounds_kernel"): (None, 5_767_606_912 / (4_194_304 * 1024), "cfg5"),
+}
+# Busy fractions (of active SM cycles) of the issue slots and of the arithmetic pipes, from the same captures on
+# shorter vectors of the same M: which unit a launch that is bound by instruction issue leans on hardest.
+NCU_PIPES = {
+    ("cfg2_M8_resnet18", "fused_rounds_kernel"): {"issue": 0.598, "fmaheavy": 0.645, "fmalite": 0.280, "alu": 0.357,
+                                                   "captured_on": "cfg2 at d = 4,000,002"},
+    ("cfg3_M16_vgg19scale", "fused_rounds_kernel"): {"issue": 0.567, "fmaheavy": 0.647, "fmalite": 0.284, "alu": 0.336,
+                                                      "captured_on": "cfg3 at d = 8,000,002"},
+    ("cfg4_M64_resnet18", "cluster_rounds_kernel"): {"issue": 0.483, "fmaheavy": 0.496, "fmalite": 0.196, "alu": 0.337,
+                                                      "captured_on": "cfg4 at d = 2,000,002"},
 }
 SM_COUNT, SCHEDULERS_PER_SM = 148, 4     # one warp instruction per scheduler and clock at most
 
@@ -274,6 +287,8 @@ def issue_roofline(tag, kernel, ms_per_round, elements, bpe, rounds_per_launch, 
            "rounds_per_launch": rounds_per_launch, "warp_inst_per_element_round": ipe,
            "bytes_per_launch": UNIQUE_FRACTION * bpe * elements,
            "replica_GBs": bpe * elements / sec / 1e9, "hbm_peak": peak, "hbm_peak_kind": f"of {peak_kind}"}
+    if kernel_source_hash() == NCU_HASH and (tag, kernel) in NCU_PIPES:
+        out["pipes_busy"] = NCU_PIPES[(tag, kernel)]
     if traffic is not None:
         dram = traffic / (sec * rounds_per_launch) / 1e9
         out.update({"dram_GBs": dram, "dram_frac_of_measured": dram / peak, "dram_frac_of_8TBs": dram / NOMINAL_HBM_GBS,
@@ -311,6 +326,8 @@ def launch_shape(g, rounds, ring):
     if per > 4.5:
         return "all rounds of a call on shared-memory-resident columns", "resident_rounds_kernel", per
     if per > 1.5:
+        if g.M > 18:        # more rows than one CTA's slabs hold: the tile is resident across a cluster of CTAs
+            return "%d rounds per launch over tiles resident across a thread-block cluster" % round(per), "cluster_rounds_kernel", per
         return "%d rounds per launch over resident tiles" % round(per), "fused_rounds_kernel", per
     return "one launch per round", "round_kernel", per
 
@@ -342,7 +359,7 @@ def measure_config(torch, binding, wk, args, local, timer, peak, peak_kind, sm_m
         entry["roofline"] = hbm_roofline(tag, kernel, best, elements, bpe, peak, peak_kind)
     else:
         entry["roofline"] = issue_roofline(tag, kernel, best, elements, bpe, per, sm_max_mhz, peak, peak_kind)
-    if kernel == "fused_rounds_kernel":
+    if kernel in ("fused_rounds_kernel", "cluster_rounds_kernel"):
         g.set_fuse_rounds(1)
         g.round(20)
         one = min(timer.repeats(g, rounds, 3))
@@ -493,7 +510,8 @@ def run_ours(args, w):
     tag = w.name + ("/bf16" if bf16 else "")
     sm_max_mhz = clocks.summary()["sm_max_mhz"]
     if fused or resident:
-        kernel = "fused_rounds_kernel" if fused else ("multi_round_kernel" if args.fuse_rounds == 1 else "resident_rounds_kernel")
+        kernel = (("cluster_rounds_kernel" if w.M > 18 else "fused_rounds_kernel") if fused else
+                  ("multi_round_kernel" if args.fuse_rounds == 1 else "resident_rounds_kernel"))
         roofline = issue_roofline(tag, kernel, per_round_ms, elements, bytes_per_element, rounds_per_launch, sm_max_mhz,
                                   peak, peak_kind)
     else:
