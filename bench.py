@@ -53,7 +53,7 @@ KERNEL_SOURCES = ("netmax_kernels.cuh", "netmax_rng.cuh")
 # enough to profile, else on the same M and tile shape with a shorter vector (`captured_on`); bytes and
 # instructions per element are what carries over.  Only reported while the kernel sources still hash to
 # the value the capture was taken at.
-NCU_HASH = "c9812615affa1170"
+NCU_HASH = "e75efcc271203a22"
 NCU_COUNTERS = {
     # (workload tag, kernel): dram bytes per element-launch, warp instructions per element-round, captured on
     ("cfg2_M8_resnet18", "round_kernel"): (1_041_923_000 / 89_391_696, 78_504_733 / 89_391_696, "cfg2"),
@@ -359,6 +359,21 @@ def measure_config(torch, binding, wk, args, local, timer, peak, peak_kind, sm_m
         entry["roofline"] = hbm_roofline(tag, kernel, best, elements, bpe, peak, peak_kind)
     else:
         entry["roofline"] = issue_roofline(tag, kernel, best, elements, bpe, per, sm_max_mhz, peak, peak_kind)
+    # the sampler alone: batched launches of 1024 rounds x M draws (Algorithm 2's peer selection)
+    batch = 1024
+    draws = torch.empty((batch, wk.M), dtype=torch.int32, device="cuda")
+    for _ in range(3):
+        g.sample_peers(0, batch, draws.data_ptr())
+    timer.barrier()
+    with torch.cuda.stream(timer.stream):
+        timer.start.record()
+    for rep in range(10):
+        g.sample_peers(rep * batch, batch, draws.data_ptr())
+    with torch.cuda.stream(timer.stream):
+        timer.stop.record()
+    timer.stop.synchronize()
+    entry["sampler_only_draws_per_s"] = 10 * batch * wk.M / (timer.start.elapsed_time(timer.stop) / 1e3)
+    del draws
     if kernel in ("fused_rounds_kernel", "cluster_rounds_kernel"):
         g.set_fuse_rounds(1)
         g.round(20)

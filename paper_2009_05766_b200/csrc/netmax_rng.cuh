@@ -76,22 +76,6 @@ __device__ __forceinline__ float log2_fast(float v) {
 #endif
 }
 
-// Fast pair: hardware log2 / sin / cos / sqrt approximations.  The absolute error of each
-// normal is about 2e-7 for typical radii and is bounded by 6e-4 for radii below 1e-3
-// (probability 5e-7), far inside the replica tolerance after scaling by alpha*sigma.
-__device__ __forceinline__ void normal_pair_fast(uint32_t a, uint32_t b, float& z0, float& z1) {
-  const float u1 = radius_uniform(a);
-  // angle = 2 pi u2 with u2 = top24(b)/2^24 taken modulo 1 into [-1/2, 1/2)
-  const float ang = (float)((int32_t)b >> 8) * 3.74507028e-07f;  // 2 pi / 2^24
-  const float r2 = fmaxf(-1.38629436111989f * log2_fast(u1), 0.0f);  // -2 ln 2 * log2(u1)
-  float rad;
-  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(r2));
-  float s, c;
-  __sincosf(ang, &s, &c);
-  z0 = rad * c;
-  z1 = rad * s;
-}
-
 // Accurate pair (library logf / sincospif / sqrtf): used where speed does not matter.
 __device__ __forceinline__ void normal_pair_accurate(uint32_t a, uint32_t b, float& z0, float& z1) {
   const float u1 = radius_uniform(a);
@@ -150,9 +134,10 @@ __device__ __forceinline__ pair_t normal_pair_fast_unscaled(uint32_t a, uint32_t
 template <bool kFast>
 __device__ __forceinline__ float4 normals4(uint4 r) {
   float4 z;
-  if (kFast) {
-    normal_pair_fast(r.x, r.y, z.x, z.y);
-    normal_pair_fast(r.z, r.w, z.z, z.w);
+  if (kFast) {  // (the update kernels use normal_pair_fast_unscaled directly and fold the constant into their noise scale)
+    unpack2(normal_pair_fast_unscaled(r.x, r.y), z.x, z.y);
+    unpack2(normal_pair_fast_unscaled(r.z, r.w), z.z, z.w);
+    z.x *= (float)kNormalScale; z.y *= (float)kNormalScale; z.z *= (float)kNormalScale; z.w *= (float)kNormalScale;
   } else {
     normal_pair_accurate(r.x, r.y, z.x, z.y);
     normal_pair_accurate(r.z, r.w, z.z, z.w);
