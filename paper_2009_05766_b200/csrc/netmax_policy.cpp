@@ -456,6 +456,7 @@ bool solve_fixed_weight(int M, const double* t, const uint8_t* adj, double phi, 
     if (tau[i] < -1e-12 || tau[i] > rows[i] * (1.0 + 1e-12)) return false;
 
   std::vector<double> A(M, 1.0), B(M, 1.0), eta(M, 0.0), wgt(M);
+  double err_mark = INFINITY;
   for (int sweep = 0; sweep < 20000; ++sweep) {
     // rows: weights B_m exp(-eta s_im); their mean s must equal tau_i / rows_i
     double row_change = 0.0;
@@ -514,6 +515,12 @@ bool solve_fixed_weight(int M, const double* t, const uint8_t* adj, double phi, 
       B[m] = next;
     }
     if (col_err <= 1e-13 && row_change <= 1e-12) break;
+    // a target outside the reachable set never settles: give up when 500 sweeps did not halve the misfit
+    // (a grid point that converges more slowly than that counts as infeasible)
+    if (sweep % 500 == 0) {
+      if (sweep > 0 && col_err > 0.5 * err_mark) break;
+      err_mark = col_err;
+    }
   }
   for (int i = 0; i < M; ++i)
     for (int m : nb[i]) r[(size_t)i * M + m] = A[i] * B[m] * std::exp(-eta[i] * (t[(size_t)i * M + m] - tmin) / scale);
