@@ -1133,9 +1133,13 @@ __global__ void __launch_bounds__(256, 2) cluster_rounds_kernel(const ClusterPar
 // memory, fp32, double-buffered by round, together with their centres, and runs every round of
 // the call on them; CTAs never talk to each other.  Two thread mappings:
 //   G == blockDim  a thread owns a column group and walks all M rows (small M): no barrier is
-//                  needed for the data, only the per-round telemetry reduction synchronises;
+//                  needed for the data, only the per-round telemetry reduction synchronises
+//                  (and not even that in a CTA of a single warp);
 //   G <= 32        thread (g, r) owns the rows r, r + blockDim / G, ... of group g (large M):
-//                  a peer's row belongs to another thread, so rounds are separated by a barrier.
+//                  a peer's row belongs to another thread, so rounds are separated by ONE barrier
+//                  (a warp-level one in a single-warp CTA); the column sums of the round are
+//                  added over the lanes of each warp before it and over the warps after it, by
+//                  one warp that changes from round to round while the others carry on.
 // Per round every CTA writes its two telemetry sums to partials[round][tile]; a second small
 // kernel adds the tiles of each round in index order.  Arithmetic per element is row_update's,
 // so replicas are bit-identical to the other launch shapes.
@@ -1287,56 +1291,87 @@ __global__ void __launch_bounds__(512) resident_rounds_kernel(const ResidentPara
         unpack2(lacc.lb, l2, l3);
         v[8] = (l0 + l1) + (l2 + l3);
       }
-      float* scratch = s_scratch + (k & 1) * scratch_floats;
-      float* red = s_red + (k & 1) * 64;
-      bool owner = true;  // does this thread hold the complete sums of its column group?
+      double* out = p.partials + ((size_t)k * p.n_tiles + tile) * 2;
       if (RL > 1) {
+        // the rows of a column group are spread over row lanes: first over those of this warp ...
         for (int off = 16; off >= G; off >>= 1) {
 #pragma unroll
           for (int a = 0; a < 9; ++a) v[a] += __shfl_xor_sync(0xffffffffu, v[a], off);
         }
-        owner = lane < G;  // a single warp: its lanes 0 .. G-1 now hold the sums of their groups
-      }
-      if (RL > 1 && nwarps > 1) {
-        if (lane < G) {
+        if (nwarps > 1) {
+          float* scratch = s_scratch + (k & 1) * scratch_floats;
+          if (lane < G) {
 #pragma unroll
-          for (int a = 0; a < 9; ++a) scratch[(warp * G + lane) * 9 + a] = v[a];
+            for (int a = 0; a < 9; ++a) scratch[(warp * G + lane) * 9 + a] = v[a];
+          }
+          __syncthreads();  // the round's one barrier: every row is written before the next round reads it, every warp's sums are out
+          // ... then over the warps, by ONE warp (a different one every round) while the others go on with
+          // the next round: its buffer is not written again before the barrier after next.  (With a second
+          // barrier and one thread adding the warps' sums, a round of 4096 x 4 elements spent 2,900 of its
+          // 9,800 cycles here.)
+          if (warp == k % nwarps) {
+#pragma unroll
+            for (int a = 0; a < 9; ++a) v[a] = 0.f;
+            for (int e = lane; e < nwarps * G; e += 32) {  // entry e = (warp, group e % G); G divides 32
+#pragma unroll
+              for (int a = 0; a < 9; ++a) v[a] += scratch[e * 9 + a];
+            }
+            for (int off = 16; off >= G; off >>= 1) {
+#pragma unroll
+              for (int a = 0; a < 9; ++a) v[a] += __shfl_xor_sync(0xffffffffu, v[a], off);
+            }
+          }
+        } else {
+          __syncwarp();  // a single warp: its lanes are all the threads that exchange rows
         }
-        __syncthreads();
-        owner = tid < G;
-        if (owner) {
-#pragma unroll
-          for (int a = 0; a < 9; ++a) v[a] = 0.f;
-          for (int w = 0; w < nwarps; ++w) {  // (G <= 32: every warp holds rows of every group)
-#pragma unroll
-            for (int a = 0; a < 9; ++a) v[a] += scratch[(w * G + tid) * 9 + a];
+        if (nwarps == 1 || warp == k % nwarps) {  // lanes 0 .. G-1 hold the sums of their groups
+          float cons = 0.f, loss = 0.f;
+          if (lane < G) {
+            cons = (v[4] - v[0] * v[0] * p.inv_M) + (v[5] - v[1] * v[1] * p.inv_M) + (v[6] - v[2] * v[2] * p.inv_M) +
+                   (v[7] - v[3] * v[3] * p.inv_M);
+            loss = v[8];
+          }
+          for (int off = 16; off > 0; off >>= 1) {
+            cons += __shfl_down_sync(0xffffffffu, cons, off);
+            loss += __shfl_down_sync(0xffffffffu, loss, off);
+          }
+          if (lane == 0) {
+            out[0] = (double)cons;
+            out[1] = 0.5 * (double)loss;
           }
         }
-      }
-      float cons = 0.f, loss = 0.f;
-      if (owner) {
-        cons = (v[4] - v[0] * v[0] * p.inv_M) + (v[5] - v[1] * v[1] * p.inv_M) + (v[6] - v[2] * v[2] * p.inv_M) +
-               (v[7] - v[3] * v[3] * p.inv_M);
-        loss = v[8];
-      }
-      for (int off = 16; off > 0; off >>= 1) {
-        cons += __shfl_down_sync(0xffffffffu, cons, off);
-        loss += __shfl_down_sync(0xffffffffu, loss, off);
-      }
-      if (lane == 0) {
-        red[warp] = cons;
-        red[32 + warp] = loss;
-      }
-      __syncthreads();  // also: every row of the round is written before the next round reads it
-      if (tid == 0) {
-        double a = 0.0, b = 0.0;
-        for (int w = 0; w < nwarps; ++w) {
-          a += (double)red[w];
-          b += (double)red[32 + w];
+      } else {
+        // a thread holds the complete sums of its column group; no thread reads another's rows
+        float cons = (v[4] - v[0] * v[0] * p.inv_M) + (v[5] - v[1] * v[1] * p.inv_M) + (v[6] - v[2] * v[2] * p.inv_M) +
+                     (v[7] - v[3] * v[3] * p.inv_M);
+        float loss = v[8];
+        for (int off = 16; off > 0; off >>= 1) {
+          cons += __shfl_down_sync(0xffffffffu, cons, off);
+          loss += __shfl_down_sync(0xffffffffu, loss, off);
         }
-        double* out = p.partials + ((size_t)k * p.n_tiles + tile) * 2;
-        out[0] = a;
-        out[1] = 0.5 * b;
+        if (nwarps == 1) {
+          if (lane == 0) {
+            out[0] = (double)cons;
+            out[1] = 0.5 * (double)loss;
+          }
+          __syncwarp();  // (the staged draws are overwritten by whichever lane gets there first)
+        } else {
+          float* red = s_red + (k & 1) * 64;
+          if (lane == 0) {
+            red[warp] = cons;
+            red[32 + warp] = loss;
+          }
+          __syncthreads();
+          if (tid == 0) {
+            double a = 0.0, b = 0.0;
+            for (int w = 0; w < nwarps; ++w) {
+              a += (double)red[w];
+              b += (double)red[32 + w];
+            }
+            out[0] = a;
+            out[1] = 0.5 * b;
+          }
+        }
       }
     }
 
