@@ -544,14 +544,15 @@ int plan_round(netmax_ctx* ctx, RoundPlan& plan, int objective) {
   plan.n_tiles = (nq + cg - 1) / cg * rg;
   plan.smem = align_up((size_t)M * 8, 16) + (plan.rl > 1 ? (size_t)kThreads * 32 * ctx->L.halves : 0) + 64 * sizeof(double);
   RoundKernel k = pick_kernel(objective, plan.short_vectors, ctx->L.halves);
-  if (plan.smem > 48 * 1024)
+  // (the kernels also hold a little static shared memory, so the opt-in is needed somewhat below 48 KB of dynamic)
+  if (plan.smem > 40 * 1024)
     NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
   int per_sm = 0;
   NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, plan.smem));
   if (per_sm < 1) return fail(ctx, NETMAX_CUDA_ERROR, "round kernel does not fit on an SM (smem %zu)", plan.smem);
   if (plan.short_vectors && ctx->cooperative) {  // the multi-round kernel needs all of its CTAs resident
     MultiRoundKernel mk = pick_multi_kernel(objective == 2 ? 0 : objective, ctx->L.halves);
-    if (plan.smem > 48 * 1024)
+    if (plan.smem > 40 * 1024)
       NM_CUDA(ctx, cudaFuncSetAttribute(mk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
     int per_sm_multi = 0;
     NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm_multi, mk, kThreads, plan.smem));
@@ -696,7 +697,7 @@ ClusterKernel pick_cluster_kernel(int objective) {
 }
 
 #ifndef NETMAX_CLUSTER_SIZE
-#define NETMAX_CLUSTER_SIZE 8
+#define NETMAX_CLUSTER_SIZE 0  // 0: chosen from the number of workers (cluster_size below); 2, 4, 8: fixed
 #endif
 #ifndef NETMAX_CLUSTER_THREADS
 #define NETMAX_CLUSTER_THREADS 0  // 0: the smallest of 64, 128, 256 threads per CTA whose slabs fit
@@ -707,13 +708,42 @@ size_t cluster_smem(int rpc, int threads) {
          64 * sizeof(double);
 }
 
+// CTAs per cluster for M workers, 0 for "one launch per round instead".  A CTA needs enough rows between
+// two cluster barriers to pay for them and few enough that eight CTAs of 64 threads still fit on an SM:
+// measured on M x 4,000,002 elements (ns per million elements and round; one launch per round: 2,160-2,220)
+//   clusters of 2:  M = 19: 1,880   20: 1,790   22: 1,730   24: 2,010   28: 2,040   32: 1,960   36: 2,460
+//   clusters of 4:  M = 20: 2,180   24: 2,030   28: 1,900   32: 1,830   36: 1,980   40: 1,930   44: 1,860   48: 2,190
+//   clusters of 8:  M = 20: 3,970   32: 2,810   40: 2,470   48: 2,240   52: 2,210   56: 2,070   60: 2,090   64: 1,970
+//                       68: 2,290   72: 2,170   80: 2,120   88: 2,050   96: 2,330
+//   clusters of 16 (not portable): 2,770 or more for M = 64 ... 136
+// `forced` (the caller asked for fused rounds): any M up to 8 x 18 rows gets the cluster whose CTAs hold
+// closest to eight rows.
+int cluster_size(int64_t M, bool forced) {
+  if (NETMAX_CLUSTER_SIZE != 0) return NETMAX_CLUSTER_SIZE;
+  if (M <= 24) return 2;
+  if (M <= 44) return 4;
+  if (M >= 55 && M <= 64) return 8;
+  if (!forced) return 0;
+  int best = 0;
+  int64_t best_gap = 0;
+  for (int c : {2, 4, 8}) {
+    const int64_t rpc = (M + c - 1) / c, gap = rpc > 8 ? rpc - 8 : 8 - rpc;
+    if (rpc <= 18 && (best == 0 || gap < best_gap)) {
+      best = c;
+      best_gap = gap;
+    }
+  }
+  return best;
+}
+
 // Long fp32 vectors with more workers than fused_rounds_kernel can hold per thread (M > 18): the rows
 // of a tile are split over the CTAs of a cluster (cluster_rounds_kernel), up to 18 rows per CTA.
 int plan_cluster_uncached(netmax_ctx* ctx, const RoundPlan& plan, const FusedPlan& fused, ClusterPlan& f) {
   f = ClusterPlan();
   if (ctx->fuse_rounds == 1 || plan.short_vectors || fused.ok || ctx->storage != NETMAX_STORAGE_F32) return NETMAX_OK;
-  const int C = NETMAX_CLUSTER_SIZE;
   const int64_t M = ctx->M;
+  const int C = cluster_size(M, ctx->fuse_rounds >= 2);
+  if (C == 0) return NETMAX_OK;
   const int rpc = (int)((M + C - 1) / C);
   if (rpc > 18) return NETMAX_OK;
   ClusterKernel k = pick_cluster_kernel(ctx->objective);

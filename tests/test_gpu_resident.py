@@ -67,6 +67,31 @@ def test_resident_columns_change_no_bit(nm, M, d, storage):
     res.close()
 
 
+@pytest.mark.parametrize("M,d", [(5048, 146), (5040, 9), (6000, 33)])
+def test_more_workers_than_fit_on_chip(nm, M, d):
+    """Beyond about 4700 workers the columns do not fit a CTA's shared memory and the per-round kernels run; around
+    M = 5040 their table of draws needs just under 48 KB of dynamic shared memory, which with the kernels' static
+    part is over the default limit (such a context once failed to plan its launch)."""
+    rng = np.random.default_rng(M + d)
+    P = random_policy(M, rng, zeros=0.5)
+    kw = dict(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=1, seed=M, trace_rounds=8)
+    one, many = nm.Netmax(fuse_rounds=1, **kw), nm.Netmax(**kw)
+    o = oracle.Sim(M, d, P, full_adj(M), alpha=0.05, rho=one.get_policy()[1], sigma=0.1, objective=1, seed=M)
+    o.init(1.0, 1.0)
+    o.set_x(one.read_replicas())                       # (the two sides' initial normals differ in the last bit)
+    o.set_c(one.read_centres())
+    for n in (1, 5):
+        one.round(n)
+        many.round(n)
+        o.round(n)
+    xa, xb, xo = one.read_replicas(), many.read_replicas(), o.x().astype(np.float64)
+    assert (xa.view(np.uint32) == xb.view(np.uint32)).all()
+    assert (one.peer_trace(0, 6) == o.trace(0, 6)).all() and (many.peer_trace(0, 6) == o.trace(0, 6)).all()
+    assert (np.abs(xa.astype(np.float64) - xo) <= TOL * (1.0 + np.abs(xo))).all()
+    one.close()
+    many.close()
+
+
 @pytest.mark.parametrize("objective", [0, 1])
 @pytest.mark.parametrize("M,d", [(4, 4096), (6, 4099), (64, 515), (130, 37), (1000, 131)])
 def test_resident_columns_match_the_oracle(nm, M, d, objective):
