@@ -511,30 +511,47 @@ int floor_pow2(int64_t v) {
 // (measured optimum on cfg 2-4: wider tiles stream better until the peer reads start to miss).
 // Short vectors (fewer than two such tiles per SM; everything is L2-resident then): 128-byte
 // column segments where M allows, no idle row lanes, and the rows split into rg groups so that
-// about two CTAs per SM have work.
+// about two CTAs per SM have work.  The same shape serves many workers with vectors of any length:
+// beyond 768 rows the 96 KB rule leaves a tile less than 128 bytes of every row, and a stream of
+// 64- or 16-byte pieces costs more than peer rows that come from L2 instead of L1 (4096 x 4096
+// elements: 135 us per round with 16-byte pieces, 34 with 128-byte pieces and two row groups;
+// 1024 x 65536: 250 against 184).
 int plan_round(netmax_ctx* ctx, RoundPlan& plan, int objective) {
   const int64_t M = ctx->M, nq = ctx->L.nq;
   const int64_t target = 2 * (int64_t)ctx->sm_count;  // the short-vector kernel runs 2 CTAs per SM
   int cg = kThreads;
   while (cg > 1 && (int64_t)cg * 16 * M > 96 * 1024) cg >>= 1;
   int rg = 1;
-  if ((nq + cg - 1) / cg < 2 * (int64_t)ctx->sm_count || kThreads / cg > M) {
+  if ((nq + cg - 1) / cg < 2 * (int64_t)ctx->sm_count || kThreads / cg > M || cg < 8) {
     plan.short_vectors = true;
-    static const int order[] = {8, 4, 2, 16, 32, 64, 128, 256, 1};
+    // Candidates in order of preference; the score is the number of CTAs with work, up to the target.
+    // First among segments of at least 128 bytes only: a narrower one that happens to give more CTAs
+    // loses more at the DRAM pins than it wins (8192 x 2048 elements: 144 us per round with 16-byte
+    // pieces and 512 CTAs, 50 with 256-byte pieces and 256 CTAs).  With more workers than resident
+    // columns can hold, this kernel is the one that runs by default, and 256-byte pieces measured
+    // best there (8192 x 2048: 50 against 55 us; 16384 x 1024: 73 against 84).
+    static const int wide_first[] = {8, 16, 32, 64, 128, 256};
+    static const int wide_first_large[] = {16, 8, 32, 64, 128, 256};
+    static const int any_width[] = {8, 4, 2, 16, 32, 64, 128, 256, 1};
     int64_t best_score = -1;
-    for (int cand : order) {
+    auto consider = [&](int cand) {
       const int rl = kThreads / cand;
-      if (rl > M && cand != kThreads) continue;  // row lanes without rows
+      if (rl > M && cand != kThreads) return;  // row lanes without rows
       const int64_t nct = (nq + cand - 1) / cand;
       int g = (int)std::min<int64_t>(std::min<int64_t>(32, std::max<int64_t>(1, M / rl)), floor_pow2(std::max<int64_t>(1, target / nct)));
       while (g > 1 && (size_t)nct * g * cand * 32 * ctx->L.halves > kColPartBytes) g >>= 1;
-      if (nct * g > kMaxGrid) continue;
+      if (nct * g > kMaxGrid) return;
       const int64_t score = std::min<int64_t>(nct * g, target);
       if (score > best_score) {
         best_score = score;
         cg = cand;
         rg = g;
       }
+    };
+    for (int cand : (M > 4700 ? wide_first_large : wide_first)) consider(cand);
+    if (best_score * 20 < target * 17) {  // fewer than 85 % of the CTAs the SMs can hold: narrower pieces may do better
+      best_score = -1;
+      for (int cand : any_width) consider(cand);
     }
   }
   plan.cg = cg;

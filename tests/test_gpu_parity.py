@@ -278,6 +278,35 @@ def test_read_columns_matches_full_read(nm):
     g.close()
 
 
+@pytest.mark.parametrize("M,d", [(1024, 16_387), (2048, 8_195), (4096, 4_099)])
+def test_many_workers_with_longer_vectors(nm, M, d):
+    """So many rows that a tile of all of them would hold less than 128 bytes of each: the rows are split into
+    groups instead (the short-vector launch shape), whatever the length of the vectors."""
+    s = workloads.config(5).link_speeds(0)[:M, :M]
+    P = s / s.sum(axis=1, keepdims=True)
+    cols = np.unique(np.concatenate([np.arange(40), np.random.default_rng(d).integers(0, d, 600), np.arange(d - 40, d)])).astype(np.int64)
+    g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=1, seed=M + d, trace_rounds=16)
+    o = oracle.Sim(M, d, P, full_adj(M), alpha=0.05, rho=g.get_policy()[1], sigma=0.1, objective=1, seed=M + d, cols=cols)
+    o.init(1.0, 1.0)
+    rounds = 6
+    g.round(1)
+    g.round(rounds - 1)
+    o.round(rounds, threads=8)
+    assert (g.peer_trace(0, rounds) == o.trace(0, rounds)).all()
+    assert_replicas_close(g.read_columns(cols), o.x())
+    # telemetry of the last round against its definition on the device buffer of the round before
+    one = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=1, seed=M + d, trace_rounds=16, fuse_rounds=1)
+    one.round(rounds)
+    assert (one.read_replicas().view(np.uint32) == g.read_replicas().view(np.uint32)).all()
+    np.testing.assert_allclose(g.telemetry(0, rounds)[0], one.telemetry(0, rounds)[0], rtol=2e-5)
+    x = one.read_replicas().astype(np.float64)
+    one.round(1)
+    want = ((x - x.mean(axis=0)) ** 2).sum() / M
+    assert one.telemetry(rounds, 1)[0][0] == pytest.approx(want, rel=1e-4)
+    g.close()
+    one.close()
+
+
 def test_many_workers_small_vectors(nm):
     """The sampling-stress shape at reduced round count: M = 4096, d = 1024."""
     w = workloads.config(5)
