@@ -166,7 +166,9 @@ int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
  * drawn ahead in one sampler launch (the draws are counter-based and do not depend on x).
  * Short vectors (a round of a few microseconds) whose M rows of at least one four-element column
  * group fit in a CTA's shared memory (M up to about 4700) run all rounds of a call on
- * shared-memory-resident columns: CTAs own disjoint columns and never exchange anything.
+ * shared-memory-resident columns: CTAs own disjoint columns and never exchange anything.  A call
+ * has to run enough rounds to repay bringing the columns on chip (2 for up to a million elements,
+ * up to 16 for the largest problems); shorter calls take the per-round kernels.
  * Other short-vector shapes (and fuse_rounds = 1) run all rounds of a call in one cooperative
  * launch with a grid-wide barrier per round; its waits are bounded, and one that runs out is
  * reported by the next synchronising call as NETMAX_CUDA_ERROR (the replicas are then not

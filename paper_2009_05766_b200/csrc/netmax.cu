@@ -50,6 +50,7 @@ struct ResidentPlan {  // launch shape of resident_rounds_kernel
   int threads = 0, grid = 0, G = 0, log2G = 0, draw_chunk = 0;
   size_t smem = 0;
   int64_t n_tiles = 0, max_rounds = 0;
+  int64_t min_rounds = 1;  // rounds a call must run to repay loading and storing the tiles
 };
 
 struct FusedPlan {  // launch shape of fused_rounds_kernel
@@ -632,6 +633,14 @@ int plan_resident_uncached(netmax_ctx* ctx, const RoundPlan& plan, ResidentPlan&
   f.smem = resident_smem(M, threads, G);
   f.n_tiles = (nq + G - 1) / G;
   f.max_rounds = std::max<int64_t>(1, std::min<int64_t>(kMaxRoundsPerLaunch, (int64_t)(kColPartBytes / 16) / f.n_tiles));
+  // A call pays once for bringing its tiles on chip and back -- narrow columns of all M rows, which stream
+  // badly (about 1.1 TB/s with one column group per tile) -- and then saves on every round.  Rounds from
+  // which that paid in measurements (us per round, resident columns against the per-round kernels, calls of
+  // 1 / 2 / 4 / many rounds): 4 x 4096 elements 13.4 / 7.0 / 4.1 / 0.9 against 10.3 / 8.2 / 6.0 / 3.8;
+  // 4096 x 1024: 57 / 33 / 21 / 9.5 against 29 / 23 / 19 / 16; 4096 x 4096: 219 / 128 / 80 / 33 against
+  // 66 / 61 / 58 / 54; 4096 x 16384: 837 / 492 / 310 / 136 against 195 / 192 / 190 / 188.
+  const int64_t elements = M * ctx->d;
+  f.min_rounds = elements <= ((int64_t)1 << 20) ? 2 : elements <= ((int64_t)1 << 22) ? 6 : elements <= ((int64_t)1 << 24) ? 8 : 16;
   ResidentKernel k = pick_resident_kernel(ctx->objective, ctx->L.halves);
   NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
   NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)f.smem));
@@ -1277,7 +1286,7 @@ int netmax_round(netmax_ctx* ctx, int64_t n_rounds) {
     rc = launch_sampler(ctx, (uint64_t)ctx->rounds, batch, ctx->trace, ctx->wring, ctx->rounds % ctx->trace_rounds,
                         ctx->trace_rounds);
     if (rc) return rc;
-    if (resident.ok) {
+    if (resident.ok && batch >= resident.min_rounds) {
       // short vectors: every round of the batch on shared-memory-resident columns
       ResidentKernel rk = pick_resident_kernel(ctx->objective, ctx->L.halves);
       int64_t b = 0;
