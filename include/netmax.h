@@ -177,10 +177,11 @@ int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
  * (netmax_config.fuse_rounds): given the draws, Eq. 16 acts on every column separately, so a
  * tile holding all M rows of a column range stays in shared memory for those rounds and HBM
  * sees x and c once per launch instead of once per round.  With 19 to 136 workers (fp32 state)
- * the rows of such a tile are split over the CTAs of a thread-block cluster (2, 4 or 8 of them,
+ * the rows of such a tile are split over the CTAs of a thread-block cluster (2 to 8 of them,
  * by the number of workers) and a pull reads the peer's row from the shared memory of the CTA
  * that holds it; with fuse_rounds = 0 this shape is taken only where it was measured faster than
- * one launch per round (19 to 44 and 55 to 64 workers), with fuse_rounds >= 2 wherever it fits.
+ * one launch per round (19 to 66 workers and most counts up to 88), with fuse_rounds >= 2
+ * wherever it fits.
  * Whatever the launch shape and however a run is split into calls, replicas and peer traces
  * are the same bit for bit; telemetry sums are accumulated in an order that depends on the
  * launch shape and agree to fp32 rounding of their partial sums (2e-5 relative or better).

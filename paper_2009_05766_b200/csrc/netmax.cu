@@ -735,24 +735,27 @@ size_t cluster_smem(int rpc, int threads) {
 }
 
 // CTAs per cluster for M workers, 0 for "one launch per round instead".  A CTA needs enough rows between
-// two cluster barriers to pay for them and few enough that eight CTAs of 64 threads still fit on an SM:
-// measured on M x 4,000,002 elements (ns per million elements and round; one launch per round: 2,160-2,220)
-//   clusters of 2:  M = 19: 1,880   20: 1,790   22: 1,730   24: 2,010   28: 2,040   32: 1,960   36: 2,460
-//   clusters of 4:  M = 20: 2,180   24: 2,030   28: 1,900   32: 1,830   36: 1,980   40: 1,930   44: 1,860   48: 2,190
-//   clusters of 8:  M = 20: 3,970   32: 2,810   40: 2,470   48: 2,240   52: 2,210   56: 2,070   60: 2,090   64: 1,970
-//                       68: 2,290   72: 2,170   80: 2,120   88: 2,050   96: 2,330
-//   clusters of 16 (not portable): 2,770 or more for M = 64 ... 136
-// `forced` (the caller asked for fused rounds): any M up to 8 x 18 rows gets the cluster whose CTAs hold
-// closest to eight rows.
+// two cluster barriers to pay for them (a barrier costs about 1,500 cycles even for the last CTA to arrive)
+// and few enough that eight CTAs of 64 threads still fit on an SM; a ragged last CTA makes the others
+// wait; smaller clusters have cheaper barriers and more pulls that stay in the CTA.  The sweet spot is
+// eight rows per CTA in as few CTAs as possible, but the details do not follow a formula, so the size is
+// the one measured fastest: every size from 2 to 8, M x 2,000,002 elements, four rounds per launch against
+// one launch per round (profiles/cluster_rounds_kernel_cfg4.md has the sweep).  Entered only where the
+// cluster shape took less than 0.97 of the per-round time: 0.73-0.90 for M = 19 ... 66, 0.92-0.97 for most
+// of 68 ... 88, nothing beyond.  Clusters of 16 (not portable) fit too few at a time: 1.3-2.1 x slower.
+// `forced` (the caller asked for fused rounds): any M up to 8 x 18 rows gets the table's size or else the
+// one whose CTAs hold closest to eight rows.
 int cluster_size(int64_t M, bool forced) {
   if (NETMAX_CLUSTER_SIZE != 0) return NETMAX_CLUSTER_SIZE;
-  if (M <= 24) return 2;
-  if (M <= 44) return 4;
-  if (M >= 55 && M <= 64) return 8;
+  static const unsigned char by_workers[] = {
+      // M = 19 ... 88
+      2, 2, 2, 2, 3, 3, 2, 2, 4, 4, 3, 3, 4, 4, 3, 2, 5, 4, 5, 5, 5, 5, 4, 4, 4, 4, 5, 6, 6, 6, 5, 5, 5, 5, 5,
+      5, 5, 7, 6, 6, 6, 6, 8, 8, 8, 8, 6, 6, 0, 4, 7, 7, 0, 7, 7, 7, 7, 7, 7, 0, 0, 8, 0, 0, 0, 8, 8, 8, 8, 8};
+  if (M >= 19 && M < 19 + (int64_t)sizeof by_workers && by_workers[M - 19] != 0) return by_workers[M - 19];
   if (!forced) return 0;
   int best = 0;
   int64_t best_gap = 0;
-  for (int c : {2, 4, 8}) {
+  for (int c = 2; c <= 8; ++c) {
     const int64_t rpc = (M + c - 1) / c, gap = rpc > 8 ? rpc - 8 : 8 - rpc;
     if (rpc <= 18 && (best == 0 || gap < best_gap)) {
       best = c;

@@ -80,10 +80,11 @@ def test_fused_rounds_change_no_bit(nm, M, d, fuse, storage, objective):
 
 
 # more workers than a thread's slab holds: the rows of a tile are split over the CTAs of a cluster
-# (of 2 for M = 19, 20, 24; of 4 for M = 25, 33, 44; of 8 for M = 50, 64, 100, 136; ragged last CTAs, one with no row at all)
+# (every cluster size from 2 to 8: M = 19, 20, 25 -> 2; 24, 33 -> 3; 44 -> 4; 35, 50 -> 5; 47, 57 -> 6; 56, 70 -> 7;
+# 64, 100, 136 -> 8; ragged last CTAs, one with no row at all)
 @pytest.mark.parametrize("M,d,fuse", [(64, 80_003, 0), (20, 303_201, 0), (33, 152_002, 3), (100, 38_001, 4), (136, 40_001, 2),
                                       (19, 310_000, 4), (24, 303_203, 0), (25, 160_001, 0), (44, 160_002, 0), (50, 80_001, 2),
-                                      (57, 80_003, 0)])
+                                      (57, 80_003, 0), (35, 160_003, 0), (47, 160_001, 0), (56, 80_001, 0), (70, 80_002, 0)])
 @pytest.mark.parametrize("objective", [0, 1])
 def test_cluster_resident_rounds_change_no_bit(nm, M, d, fuse, objective):
     rng = np.random.default_rng(M * 7 + d)
@@ -109,11 +110,11 @@ def test_cluster_resident_rounds_change_no_bit(nm, M, d, fuse, objective):
 
 
 def test_cluster_shape_is_taken_only_where_it_pays(nm):
-    """fuse_rounds = 0 fuses rounds over a cluster for 19 ... 44 and 55 ... 64 workers and runs one launch per
-    round for the worker counts in between and beyond; fuse_rounds >= 2 fuses wherever the rows fit (M <= 144)."""
+    """fuse_rounds = 0 fuses rounds over a cluster for the worker counts where that was measured faster (19 ... 66 and
+    most of 68 ... 88) and runs one launch per round elsewhere; fuse_rounds >= 2 fuses wherever the rows fit (M <= 144)."""
     d = 400_001
-    for M, fuse, fused in ((22, 0, True), (40, 0, True), (50, 0, False), (50, 4, True), (60, 0, True), (80, 0, False),
-                           (80, 3, True), (150, 4, False)):
+    for M, fuse, fused in ((22, 0, True), (40, 0, True), (50, 0, True), (67, 0, False), (67, 4, True), (60, 0, True),
+                           (81, 0, False), (81, 3, True), (100, 0, False), (150, 4, False)):
         P = np.full((M, M), 1.0 / (M - 1))
         np.fill_diagonal(P, 0.0)
         g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, seed=1, trace_rounds=16, fuse_rounds=fuse)
