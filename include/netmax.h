@@ -173,14 +173,14 @@ int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
  * launch with a grid-wide barrier per round; its waits are bounded, and one that runs out is
  * reported by the next synchronising call as NETMAX_CUDA_ERROR (the replicas are then not
  * valid).
- * Long vectors with at most 18 workers advance up to four rounds per launch
+ * Long vectors with at most 36 workers advance up to four rounds per launch
  * (netmax_config.fuse_rounds): given the draws, Eq. 16 acts on every column separately, so a
  * tile holding all M rows of a column range stays in shared memory for those rounds and HBM
- * sees x and c once per launch instead of once per round.  With 19 to 136 workers (fp32 state)
- * the rows of such a tile are split over the CTAs of a thread-block cluster (2 to 8 of them,
+ * sees x and c once per launch instead of once per round.  With 37 to 144 workers (fp32 state)
+ * the rows of such a tile are split over the CTAs of a thread-block cluster (4 to 8 of them,
  * by the number of workers) and a pull reads the peer's row from the shared memory of the CTA
  * that holds it; with fuse_rounds = 0 this shape is taken only where it was measured faster than
- * one launch per round (19 to 66 workers and most counts up to 88), with fuse_rounds >= 2
+ * one launch per round (37 to 66 workers and most counts up to 88), with fuse_rounds >= 2
  * wherever it fits.
  * Whatever the launch shape and however a run is split into calls, replicas and peer traces
  * are the same bit for bit; telemetry sums are accumulated in an order that depends on the

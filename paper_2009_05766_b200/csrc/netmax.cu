@@ -676,11 +676,16 @@ int plan_fused_uncached(netmax_ctx* ctx, const RoundPlan& plan, FusedPlan& f) {
   // puts more threads on an SM with at least two CTAs (one loads its tile while the other
   // computes; M = 16: 1 x 256 threads 529 us).  Every thread needs 48 M bytes of shared memory,
   // and the kernel's ~100 registers cap an SM at 16 warps (capping it at 96 or 80 registers for
-  // 18-20 warps measured slower: 135 and 157 us against 128 per cfg2 round).
+  // 18-20 warps measured slower: 135 and 157 us against 128 per cfg2 round).  Beyond 18 workers only
+  // 64-thread CTAs fit, three per SM up to M = 24 and two up to M = 36: four to six warps per SM, and
+  // still 9 to 21 % faster than the same rows split over a cluster (M x 4,000,002 elements, us per round:
+  // M = 20: 132 against 144, 28: 182 against 214, 36: 227 against 287) -- no barrier, no pull that leaves
+  // the CTA.  A single such CTA per SM (M = 37 ... 73) is slower than the cluster shape (M = 40: 330
+  // against 309), so the kernel is used down to 128 threads per SM.
   FusedKernel k = pick_fused_kernel(ctx->objective, ctx->L.halves);
   NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
   int threads = 0, per_sm = 0;
-  for (int cand : {256, 128}) {
+  for (int cand : {256, 128, 64}) {
     const size_t smem = fixed + (size_t)48 * M * cand;
     if (smem > (size_t)227 * 1024) continue;
     NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -689,7 +694,7 @@ int plan_fused_uncached(netmax_ctx* ctx, const RoundPlan& plan, FusedPlan& f) {
     const bool better = (n >= 2) != (per_sm >= 2) ? n >= 2 : n * cand > per_sm * threads;
     if (n >= 1 && (threads == 0 || better)) { threads = cand; per_sm = n; }
   }
-  if (threads == 0 || per_sm * threads < 256) return NETMAX_OK;  // too few warps to hide the arithmetic latency
+  if (threads == 0 || per_sm * threads < 128) return NETMAX_OK;  // too few warps to hide the arithmetic latency
   f.threads = threads;
   f.smem = fixed + (size_t)48 * M * threads;
   f.max_rounds = ctx->fuse_rounds >= 2 ? std::min(ctx->fuse_rounds, kFusedMaxRounds) : kFusedMaxRounds;
@@ -741,17 +746,17 @@ size_t cluster_smem(int rpc, int threads) {
 // eight rows per CTA in as few CTAs as possible, but the details do not follow a formula, so the size is
 // the one measured fastest: every size from 2 to 8, M x 2,000,002 elements, four rounds per launch against
 // one launch per round (profiles/cluster_rounds_kernel_cfg4.md has the sweep).  Entered only where the
-// cluster shape took less than 0.97 of the per-round time: 0.73-0.90 for M = 19 ... 66, 0.92-0.97 for most
+// cluster shape took less than 0.97 of the per-round time: 0.83-0.93 for M = 37 ... 66, 0.92-0.97 for most
 // of 68 ... 88, nothing beyond.  Clusters of 16 (not portable) fit too few at a time: 1.3-2.1 x slower.
 // `forced` (the caller asked for fused rounds): any M up to 8 x 18 rows gets the table's size or else the
 // one whose CTAs hold closest to eight rows.
 int cluster_size(int64_t M, bool forced) {
   if (NETMAX_CLUSTER_SIZE != 0) return NETMAX_CLUSTER_SIZE;
   static const unsigned char by_workers[] = {
-      // M = 19 ... 88
-      2, 2, 2, 2, 3, 3, 2, 2, 4, 4, 3, 3, 4, 4, 3, 2, 5, 4, 5, 5, 5, 5, 4, 4, 4, 4, 5, 6, 6, 6, 5, 5, 5, 5, 5,
-      5, 5, 7, 6, 6, 6, 6, 8, 8, 8, 8, 6, 6, 0, 4, 7, 7, 0, 7, 7, 7, 7, 7, 7, 0, 0, 8, 0, 0, 0, 8, 8, 8, 8, 8};
-  if (M >= 19 && M < 19 + (int64_t)sizeof by_workers && by_workers[M - 19] != 0) return by_workers[M - 19];
+      // M = 37 ... 88 (up to 36 workers fused_rounds_kernel holds all rows in one CTA)
+      5, 5, 5, 5, 4, 4, 4, 4, 5, 6, 6, 6, 5, 5, 5, 5, 5, 5, 5, 7, 6, 6, 6, 6, 8, 8,
+      8, 8, 6, 6, 0, 4, 7, 7, 0, 7, 7, 7, 7, 7, 7, 0, 0, 8, 0, 0, 0, 8, 8, 8, 8, 8};
+  if (M >= 37 && M < 37 + (int64_t)sizeof by_workers && by_workers[M - 37] != 0) return by_workers[M - 37];
   if (!forced) return 0;
   int best = 0;
   int64_t best_gap = 0;
@@ -765,7 +770,7 @@ int cluster_size(int64_t M, bool forced) {
   return best;
 }
 
-// Long fp32 vectors with more workers than fused_rounds_kernel can hold per thread (M > 18): the rows
+// Long fp32 vectors with more workers than fused_rounds_kernel can hold per thread (M > 36): the rows
 // of a tile are split over the CTAs of a cluster (cluster_rounds_kernel), up to 18 rows per CTA.
 int plan_cluster_uncached(netmax_ctx* ctx, const RoundPlan& plan, const FusedPlan& fused, ClusterPlan& f) {
   f = ClusterPlan();

@@ -39,7 +39,8 @@ def random_policy(M, rng, zeros=0.0):
 @pytest.mark.parametrize("M,d,fuse,storage", [(2, 400_003, 0, "f32"), (5, 320_001, 0, "f32"), (8, 400_002, 0, "f32"),
                                               (9, 310_000, 3, "f32"), (8, 400_001, 2, "f32"), (16, 320_001, 4, "f32"),
                                               (18, 310_003, 4, "f32"), (8, 700_003, 0, "bf16"), (3, 650_001, 4, "bf16"),
-                                              (16, 620_006, 3, "bf16")])
+                                              (16, 620_006, 3, "bf16"), (24, 310_001, 0, "f32"), (36, 170_003, 0, "f32"),
+                                              (22, 620_002, 0, "bf16"), (36, 330_001, 2, "bf16")])
 @pytest.mark.parametrize("objective", [0, 1])
 def test_fused_rounds_change_no_bit(nm, M, d, fuse, storage, objective):
     rng = np.random.default_rng(M * 11 + d)
@@ -60,8 +61,9 @@ def test_fused_rounds_change_no_bit(nm, M, d, fuse, storage, objective):
     assert (xa.view(np.uint32) == xb.view(np.uint32)).all()
     assert (one.peer_trace(0, rounds) == many.peer_trace(0, rounds)).all()
     (ca, la), (cb, lb) = one.telemetry(0, rounds), many.telemetry(0, rounds)
-    # (with bfloat16 state the two launch shapes group a thread's fp32 partial sums by 8 and by 4 columns)
-    rtol = 1e-12 if storage == "f32" else 1e-6
+    # (with bfloat16 state the two launch shapes group a thread's fp32 partial sums by 8 and by 4 columns; beyond 24
+    # workers the per-round kernel splits the rows of a column over two row lanes and adds their fp32 sums afterwards)
+    rtol = 1e-12 if storage == "f32" and M <= 24 else 1e-6
     np.testing.assert_allclose(cb, ca, rtol=rtol)
     np.testing.assert_allclose(lb, la, rtol=rtol)
     # padding lanes of the rows stay zero
@@ -79,9 +81,9 @@ def test_fused_rounds_change_no_bit(nm, M, d, fuse, storage, objective):
     many.close()
 
 
-# more workers than a thread's slab holds: the rows of a tile are split over the CTAs of a cluster
-# (every cluster size from 2 to 8: M = 19, 20, 25 -> 2; 24, 33 -> 3; 44 -> 4; 35, 50 -> 5; 47, 57 -> 6; 56, 70 -> 7;
-# 64, 100, 136 -> 8; ragged last CTAs, one with no row at all)
+# more workers than the 128- and 256-thread CTAs hold: 64-thread CTAs of the same kernel up to M = 36 (19, 20, 24: three
+# per SM; 25, 33, 35: two), beyond that the rows of a tile are split over the CTAs of a cluster (M = 44 -> 4 CTAs;
+# 50 -> 5; 47, 57 -> 6; 56, 70 -> 7; 64, 100, 136 -> 8; ragged last CTAs, one with no row at all)
 @pytest.mark.parametrize("M,d,fuse", [(64, 80_003, 0), (20, 303_201, 0), (33, 152_002, 3), (100, 38_001, 4), (136, 40_001, 2),
                                       (19, 310_000, 4), (24, 303_203, 0), (25, 160_001, 0), (44, 160_002, 0), (50, 80_001, 2),
                                       (57, 80_003, 0), (35, 160_003, 0), (47, 160_001, 0), (56, 80_001, 0), (70, 80_002, 0)])
@@ -110,8 +112,9 @@ def test_cluster_resident_rounds_change_no_bit(nm, M, d, fuse, objective):
 
 
 def test_cluster_shape_is_taken_only_where_it_pays(nm):
-    """fuse_rounds = 0 fuses rounds over a cluster for the worker counts where that was measured faster (19 ... 66 and
-    most of 68 ... 88) and runs one launch per round elsewhere; fuse_rounds >= 2 fuses wherever the rows fit (M <= 144)."""
+    """fuse_rounds = 0 fuses rounds for the worker counts where that was measured faster (in one CTA up to 36, over a
+    cluster for 37 ... 66 and most of 68 ... 88) and runs one launch per round elsewhere; fuse_rounds >= 2 fuses
+    wherever the rows fit (M <= 144)."""
     d = 400_001
     for M, fuse, fused in ((22, 0, True), (40, 0, True), (50, 0, True), (67, 0, False), (67, 4, True), (60, 0, True),
                            (81, 0, False), (81, 3, True), (100, 0, False), (150, 4, False)):
