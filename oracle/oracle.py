@@ -183,7 +183,11 @@ class Sim:
             lib().nmo_sim_destroy(self._h)
             self._h = None
 
-    __del__ = close
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:       # (at interpreter exit the module's globals may already be gone)
+            pass
 
     def set_policy(self, P, adj, rho):
         P = np.ascontiguousarray(P, dtype=np.float64)
