@@ -129,8 +129,9 @@ def test_cluster_shape_is_taken_only_where_it_pays(nm):
         g.close()
 
 
-def test_cluster_resident_rounds_match_the_oracle(nm):
-    M, d = 64, 80_003
+# 64-thread CTAs of the single-CTA kernel (M = 28), clusters of 6, 7 and 8 CTAs
+@pytest.mark.parametrize("M,d", [(64, 80_003), (28, 160_003), (48, 80_001), (56, 80_002)])
+def test_cluster_resident_rounds_match_the_oracle(nm, M, d):
     rng = np.random.default_rng(M + d)
     P = random_policy(M, rng, zeros=0.2)
     g = nm.Netmax(M=M, d=d, lr=0.05, prob=P, sigma=0.1, x0_std=1.0, c_std=1.0, objective=1, seed=7, trace_rounds=32)
