@@ -6,9 +6,9 @@
 //                         with Eq. 16 (pull from the round-start snapshot of the peer) and
 //                         with the round's telemetry; reads one buffer, writes the other.
 //   fused_rounds_kernel   the same for up to four rounds per launch on tiles that stay in a
-//                         CTA's shared memory (long vectors, up to 18 workers).
+//                         CTA's shared memory (long vectors, up to 36 workers).
 //   cluster_rounds_kernel the same with the rows of a tile split over the CTAs of a thread-block
-//                         cluster, pulls through distributed shared memory (up to 136 workers).
+//                         cluster, pulls through distributed shared memory (up to 144 workers).
 //   resident_rounds_kernel, multi_round_kernel   short vectors: all rounds of a call in one launch.
 //   step_kernel           the asynchronous timeline: one worker per global step (Eq. 17).
 //   init_normal_kernel    x(0) and c from the seed.

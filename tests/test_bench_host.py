@@ -19,6 +19,15 @@ def test_counter_tables_belong_to_the_current_kernel_sources():
         assert (cfg, "round_kernel") in bench.NCU_COUNTERS
 
 
+def test_source_hash_sees_code_and_not_comments(tmp_path):
+    a, b, c = tmp_path / "a.cuh", tmp_path / "b.cuh", tmp_path / "c.cuh"
+    a.write_text("// header\nint f(int x) {  // doubles\n  return 2 * x;\n}\n")
+    b.write_text("// another header\n\nint f(int x) {\n  return 2 * x;  // twice x\n}\n")
+    c.write_text("int f(int x) {\n  return 3 * x;\n}\n")
+    assert bench.hash_sources([a]) == bench.hash_sources([b]) != bench.hash_sources([c])
+    assert bench.hash_sources([a, c]) != bench.hash_sources([c, a])
+
+
 def test_hbm_roofline_counts_the_bytes_that_must_cross_the_pins():
     elements, ms = 89_391_696, 0.19
     r = bench.hbm_roofline("cfg2_M8_resnet18", "round_kernel", ms, elements, 16, 6537.0, "measured")
