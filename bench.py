@@ -8,9 +8,9 @@ pulls from the peer's round-start replica, over all M x d elements.  The metric 
 GB/s = 16 bytes x M x d x rounds / time (reads of x_i, x_peer and c_i plus the write of x_i',
 4 bytes each).  One JSON line is printed by rank 0.
 
-The library advances up to four rounds per launch where all M rows of a column tile fit in
-shared memory (one CTA's up to 36 workers, a thread-block cluster's beyond); that launch is bound by
-instruction issue, not by HBM,
+The library advances up to eight rounds per launch where all M rows of a column tile fit in
+shared memory (one CTA's up to 36 workers; four rounds over a thread-block cluster's beyond); that launch
+is bound by instruction issue, not by HBM,
 and the line's `roofline` says so.  The same workload with one launch per round (the HBM-bound
 kernel) is timed as well and reported under `one_launch_per_round`.
 
@@ -54,28 +54,28 @@ KERNEL_SOURCES = ("netmax_kernels.cuh", "netmax_rng.cuh")
 # enough to profile, else on the same M and tile shape with a shorter vector (`captured_on`); bytes and
 # instructions per element are what carries over.  Only reported while the kernel sources still hash to
 # the value the capture was taken at.
-NCU_HASH = "1a8b13adfddee6e2"
+NCU_HASH = "a822180d1ad9aa37"
 NCU_COUNTERS = {
     # (workload tag, kernel): dram bytes per element-launch, warp instructions per element-round, captured on
-    ("cfg2_M8_resnet18", "round_kernel"): (1_042_482_000 / 89_391_696, 78_504_733 / 89_391_696, "cfg2"),
-    ("cfg2_M8_resnet18", "fused_rounds_kernel"): (1_040_643_000 / 89_391_696, 314_012_326 / (89_391_696 * 4), "cfg2"),
-    ("cfg2_M8_resnet18/bf16", "round_kernel"): (505_371_000 / 89_391_696, 85_164_099 / 89_391_696, "cfg2"),
-    ("cfg2_M8_resnet18/bf16", "fused_rounds_kernel"): (505_749_000 / 89_391_696, 345_321_682 / (89_391_696 * 4), "cfg2"),
-    ("cfg3_M16_vgg19scale", "fused_rounds_kernel"): (3_805_409_000 / 320_000_000, 1_031_374_061 / (320_000_000 * 4), "cfg3"),
-    ("cfg3_M16_vgg19scale", "round_kernel"): (1_544_043_000 / (16 * 8_000_002), 101_887_293 / (16 * 8_000_002), "cfg3 at d = 8,000,002"),
-    ("cfg4_M64_resnet18", "cluster_rounds_kernel"): (1_503_713_000 / (64 * 2_000_002), 524_126_023 / (64 * 2_000_002 * 4), "cfg4 at d = 2,000,002"),
-    ("cfg4_M64_resnet18", "round_kernel"): (1_544_489_000 / (64 * 2_000_002), 104_626_918 / (64 * 2_000_002), "cfg4 at d = 2,000,002"),
+    ("cfg2_M8_resnet18", "round_kernel"): (1_041_843_000 / 89_391_696, 78_504_733 / 89_391_696, "cfg2"),
+    ("cfg2_M8_resnet18", "fused_rounds_kernel"): (1_041_110_000 / 89_391_696, 612_995_880 / (89_391_696 * 8), "cfg2"),
+    ("cfg2_M8_resnet18/bf16", "round_kernel"): (507_135_000 / 89_391_696, 85_164_099 / 89_391_696, "cfg2"),
+    ("cfg2_M8_resnet18/bf16", "fused_rounds_kernel"): (505_620_000 / 89_391_696, 660_744_326 / (89_391_696 * 8), "cfg2"),
+    ("cfg3_M16_vgg19scale", "fused_rounds_kernel"): (3_805_327_000 / 320_000_000, 2_031_045_889 / (320_000_000 * 8), "cfg3"),
+    ("cfg3_M16_vgg19scale", "round_kernel"): (1_543_966_000 / (16 * 8_000_002), 101_887_293 / (16 * 8_000_002), "cfg3 at d = 8,000,002"),
+    ("cfg4_M64_resnet18", "cluster_rounds_kernel"): (1_503_694_000 / (64 * 2_000_002), 524_126_023 / (64 * 2_000_002 * 4), "cfg4 at d = 2,000,002"),
+    ("cfg4_M64_resnet18", "round_kernel"): (1_545_154_000 / (64 * 2_000_002), 104_626_918 / (64 * 2_000_002), "cfg4 at d = 2,000,002"),
     ("cfg1_M4_d4096", "resident_rounds_kernel"): (None, 49_802_752 / (16_384 * 1024), "cfg1"),
     ("cfg5_M4096_sampling", "resident_rounds_kernel"): (None, 5_822_930_304 / (4_194_304 * 1024), "cfg5"),
 }
 # Busy fractions (of active SM cycles) of the issue slots and of the arithmetic pipes, from the same captures on
 # shorter vectors of the same M: which unit a launch that is bound by instruction issue leans on hardest.
 NCU_PIPES = {
-    ("cfg2_M8_resnet18", "fused_rounds_kernel"): {"issue": 0.601, "fmaheavy": 0.647, "fmalite": 0.282, "alu": 0.359,
+    ("cfg2_M8_resnet18", "fused_rounds_kernel"): {"issue": 0.600, "fmaheavy": 0.657, "fmalite": 0.296, "alu": 0.370,
                                                    "captured_on": "cfg2 at d = 4,000,002"},
-    ("cfg3_M16_vgg19scale", "fused_rounds_kernel"): {"issue": 0.570, "fmaheavy": 0.650, "fmalite": 0.285, "alu": 0.337,
+    ("cfg3_M16_vgg19scale", "fused_rounds_kernel"): {"issue": 0.557, "fmaheavy": 0.639, "fmalite": 0.292, "alu": 0.345,
                                                       "captured_on": "cfg3 at d = 8,000,002"},
-    ("cfg4_M64_resnet18", "cluster_rounds_kernel"): {"issue": 0.486, "fmaheavy": 0.500, "fmalite": 0.197, "alu": 0.339,
+    ("cfg4_M64_resnet18", "cluster_rounds_kernel"): {"issue": 0.486, "fmaheavy": 0.499, "fmalite": 0.197, "alu": 0.339,
                                                       "captured_on": "cfg4 at d = 2,000,002"},
 }
 SM_COUNT, SCHEDULERS_PER_SM = 148, 4     # one warp instruction per scheduler and clock at most
@@ -333,10 +333,10 @@ def launch_shape(g, rounds, ring):
     before = g.kernel_launches
     g.round(rounds)
     per = rounds / max(1, g.kernel_launches - before - (rounds + ring - 1) // ring)      # sampler launches excluded
-    if per > 4.5:
+    if per > 8.5 or (per > 1.5 and g.M * g.d < (1 << 23)):      # (short vectors never take the tile-resident shapes)
         return "all rounds of a call on shared-memory-resident columns", "resident_rounds_kernel", per
     if per > 1.5:
-        if g.M > 18:        # more rows than one CTA's slabs hold: the tile is resident across a cluster of CTAs
+        if g.M > 36:        # more rows than one CTA's slabs hold: the tile is resident across a cluster of CTAs
             return "%d rounds per launch over tiles resident across a thread-block cluster" % round(per), "cluster_rounds_kernel", per
         return "%d rounds per launch over resident tiles" % round(per), "fused_rounds_kernel", per
     return "one launch per round", "round_kernel", per
@@ -358,7 +358,7 @@ def measure_config(torch, binding, wk, args, local, timer, peak, peak_kind, sm_m
     elements = wk.M * wk.d
     tag = wk.name + ("/bf16" if bf16 else "")
     rounds = 200 if elements > 1 << 22 else 2000
-    shape, kernel, per = launch_shape(g, 20, ring)
+    shape, kernel, per = launch_shape(g, 24, ring)
     g.round(20)
     ms = timer.repeats(g, rounds, 3)
     best = min(ms)
@@ -464,8 +464,8 @@ def run_ours(args, w):
     value = bytes_per_element * elements * world * args.steps / sec / 1e9
 
     rounds_per_launch = args.steps / max(1, launches - (args.steps + ring - 1) // ring)   # sampler launches excluded
-    fused = 1.5 < rounds_per_launch <= 4.5
-    resident = rounds_per_launch > 4.5      # short vectors: all rounds of a call on resident columns
+    resident = rounds_per_launch > 8.5 or (rounds_per_launch > 1.5 and elements < (1 << 23))   # short vectors: all rounds
+    fused = rounds_per_launch > 1.5 and not resident                                          # of a call on resident columns
     single_ms = None
     if fused:                       # the same rounds, one launch each: the HBM-bound kernel
         g.set_fuse_rounds(1)
@@ -535,7 +535,7 @@ def run_ours(args, w):
     tag = w.name + ("/bf16" if bf16 else "")
     sm_max_mhz = clocks.summary()["sm_max_mhz"]
     if fused or resident:
-        kernel = (("cluster_rounds_kernel" if w.M > 18 else "fused_rounds_kernel") if fused else
+        kernel = (("cluster_rounds_kernel" if w.M > 36 else "fused_rounds_kernel") if fused else
                   ("multi_round_kernel" if args.fuse_rounds == 1 else "resident_rounds_kernel"))
         roofline = issue_roofline(tag, kernel, per_round_ms, elements, bytes_per_element, rounds_per_launch, sm_max_mhz,
                                   peak, peak_kind)
@@ -676,7 +676,7 @@ def main():
     ap.add_argument("--configs", default="all",
                     help="one GPU: which of cfg1..cfg5 to time into the line's `configs` (all, none, or e.g. 3,4)")
     ap.add_argument("--fuse-rounds", type=int, default=0,
-                    help="rounds per launch over a resident tile: 0 automatic, 1 one launch per round, 2..4")
+                    help="rounds per launch over a resident tile: 0 automatic, 1 one launch per round, 2..8")
     ap.add_argument("--storage", choices=["f32", "bf16"], default="f32",
                     help="precision of the replicas in device memory (arithmetic is fp32 either way)")
     ap.add_argument("--mode", choices=["rounds", "async"], default="rounds",

@@ -112,7 +112,7 @@ typedef struct netmax_config {
   int32_t fuse_rounds;           /* rounds that one launch may advance a tile of long vectors while it is
                                     resident on chip (see netmax_round): 0 (default) automatic, 1 never
                                     (one launch per round; short vectors then do not keep columns in shared
-                                    memory either), 2..4 at most that many.  Replicas and peer traces do
+                                    memory either), 2..8 at most that many (four over a cluster).  Replicas and peer traces do
                                     not depend on it                                                     */
   int64_t first_round;           /* number of the context's first round, 0 <= first_round < 2^56 (default 0).  Rounds are
                                     numbered from here; the round number is a word of every Philox counter, so a run
@@ -173,13 +173,13 @@ int netmax_set_centres(netmax_ctx* ctx, const float* host_c);
  * launch with a grid-wide barrier per round; its waits are bounded, and one that runs out is
  * reported by the next synchronising call as NETMAX_CUDA_ERROR (the replicas are then not
  * valid).
- * Long vectors with at most 36 workers advance up to four rounds per launch
+ * Long vectors with at most 36 workers advance up to eight rounds per launch
  * (netmax_config.fuse_rounds): given the draws, Eq. 16 acts on every column separately, so a
  * tile holding all M rows of a column range stays in shared memory for those rounds and HBM
  * sees x and c once per launch instead of once per round.  With 37 to 144 workers (fp32 state)
  * the rows of such a tile are split over the CTAs of a thread-block cluster (4 to 8 of them,
- * by the number of workers) and a pull reads the peer's row from the shared memory of the CTA
- * that holds it; with fuse_rounds = 0 this shape is taken only where it was measured faster than
+ * by the number of workers), a pull reads the peer's row from the shared memory of the CTA
+ * that holds it, and a launch advances up to four rounds; with fuse_rounds = 0 this shape is taken only where it was measured faster than
  * one launch per round (37 to 66 workers and most counts up to 88), with fuse_rounds >= 2
  * wherever it fits.
  * Whatever the launch shape and however a run is split into calls, replicas and peer traces
@@ -204,7 +204,7 @@ int netmax_round_from_host(netmax_ctx* ctx, const float* host_x, const float* ho
                            int32_t n_chunks);
 
 /* Changes netmax_config.fuse_rounds for the rounds that follow (0 automatic, 1 one launch per
- * round, 2..4 at most that many rounds per launch). */
+ * round, 2..8 at most that many rounds per launch). */
 int netmax_set_fuse_rounds(netmax_ctx* ctx, int32_t fuse_rounds);
 
 /* Number of the next round: netmax_config.first_round plus the rounds enqueued so far. */

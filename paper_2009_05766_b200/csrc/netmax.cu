@@ -56,6 +56,7 @@ struct ResidentPlan {  // launch shape of resident_rounds_kernel
 struct FusedPlan {  // launch shape of fused_rounds_kernel
   bool ok = false;
   int threads = 0, grid = 0, max_rounds = 0;
+  int slots = 0;  // rounds the kernel's table of draws is sized for
   size_t smem = 0;
   int64_t n_tiles = 0;
 };
@@ -101,7 +102,7 @@ Layout make_layout(int64_t M, int64_t d, int64_t trace_rounds, int storage) {
   L.off_trace = take((size_t)trace_rounds * M * sizeof(int32_t));
   L.off_wring = take((size_t)trace_rounds * M * sizeof(float));  // pull weight of every draw in the trace ring
   L.off_tel = take((size_t)trace_rounds * 2 * sizeof(double));
-  L.off_partials = take((size_t)kMaxGrid * 2 * sizeof(double) * 2);  // two sets: multi-round launches alternate
+  L.off_partials = take((size_t)kMaxGrid * 2 * sizeof(double) * kFusedMaxRounds);  // per round of a fused launch; two sets for multi-round launches
   L.off_ticket = take(256);
   L.off_colpart = take(kColPartBytes);
   L.off_coltick = take((size_t)kMaxGrid * sizeof(unsigned int));
@@ -483,9 +484,14 @@ MultiRoundKernel pick_multi_kernel(int objective, int halves) {
 
 using FusedKernel = void (*)(const FusedParams);
 
-FusedKernel pick_fused_kernel(int objective, int halves) {
-  if (halves == 2) return objective == 1 ? fused_rounds_kernel<1, true, true> : fused_rounds_kernel<0, true, true>;
-  return objective == 1 ? fused_rounds_kernel<1, true, false> : fused_rounds_kernel<0, true, false>;
+template <int kRounds>
+FusedKernel pick_fused_kernel_r(int objective, int halves) {
+  if (halves == 2) return objective == 1 ? fused_rounds_kernel<1, true, true, kRounds> : fused_rounds_kernel<0, true, true, kRounds>;
+  return objective == 1 ? fused_rounds_kernel<1, true, false, kRounds> : fused_rounds_kernel<0, true, false, kRounds>;
+}
+// The instance for launches of `rounds` rounds (both instances share one shared-memory layout, FusedParams::slots).
+FusedKernel pick_fused_kernel(int objective, int halves, int rounds) {
+  return rounds <= 4 ? pick_fused_kernel_r<4>(objective, halves) : pick_fused_kernel_r<kFusedMaxRounds>(objective, halves);
 }
 
 using ResidentKernel = void (*)(const ResidentParams);
@@ -669,8 +675,7 @@ int plan_fused_uncached(netmax_ctx* ctx, const RoundPlan& plan, FusedPlan& f) {
   f = FusedPlan();
   if (ctx->fuse_rounds == 1 || plan.short_vectors) return NETMAX_OK;
   const int64_t M = ctx->M;
-  const size_t head = align_up((size_t)kFusedMaxRounds * M * 16, 128);
-  const size_t fixed = head + 64 * sizeof(double);
+  const int want_rounds = ctx->fuse_rounds >= 2 ? std::min(ctx->fuse_rounds, kFusedMaxRounds) : kFusedMaxRounds;
   // 256 or 128 threads per CTA (a multiple of four warps keeps the SM's four schedulers evenly
   // loaded: 3 x 96 threads measured 587 us per cfg3 round against 508 for 2 x 128), whichever
   // puts more threads on an SM with at least two CTAs (one loads its tile while the other
@@ -682,22 +687,39 @@ int plan_fused_uncached(netmax_ctx* ctx, const RoundPlan& plan, FusedPlan& f) {
   // M = 20: 132 against 144, 28: 182 against 214, 36: 227 against 287) -- no barrier, no pull that leaves
   // the CTA.  A single such CTA per SM (M = 37 ... 73) is slower than the cluster shape (M = 40: 330
   // against 309), so the kernel is used down to 128 threads per SM.
-  FusedKernel k = pick_fused_kernel(ctx->objective, ctx->L.halves);
+  FusedKernel k = pick_fused_kernel(ctx->objective, ctx->L.halves, kFusedMaxRounds);  // (the instance with more registers)
   NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
-  int threads = 0, per_sm = 0;
-  for (int cand : {256, 128, 64}) {
-    const size_t smem = fixed + (size_t)48 * M * cand;
-    if (smem > (size_t)227 * 1024) continue;
-    NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int n = 0;
-    NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k, cand, smem));
-    const bool better = (n >= 2) != (per_sm >= 2) ? n >= 2 : n * cand > per_sm * threads;
-    if (n >= 1 && (threads == 0 || better)) { threads = cand; per_sm = n; }
+  NM_CUDA(ctx, cudaFuncSetAttribute(pick_fused_kernel(ctx->objective, ctx->L.halves, 4), cudaFuncAttributePreferredSharedMemoryCarveout,
+                                    (int)cudaSharedmemCarveoutMaxShared));
+  // The table of draws at the head of the shared memory takes 16 M bytes per round of the launch: room for
+  // as many rounds as were asked for, unless the smaller table of four rounds lets more threads live on an SM
+  // (M = 36: the last kilobytes decide between two CTAs and one).
+  int threads = 0, per_sm = 0, slots = 0;
+  size_t fixed = 0;
+  for (int rounds : {want_rounds, std::min(want_rounds, 4)}) {
+    const size_t fixed_r = align_up((size_t)rounds * M * 16, 128) + 64 * sizeof(double);
+    int threads_r = 0, per_sm_r = 0;
+    for (int cand : {256, 128, 64}) {
+      const size_t smem = fixed_r + (size_t)48 * M * cand;
+      if (smem > (size_t)227 * 1024) continue;
+      NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      int n = 0;
+      NM_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k, cand, smem));
+      const bool better = (n >= 2) != (per_sm_r >= 2) ? n >= 2 : n * cand > per_sm_r * threads_r;
+      if (n >= 1 && (threads_r == 0 || better)) { threads_r = cand; per_sm_r = n; }
+    }
+    if (threads_r != 0 && per_sm_r * threads_r > per_sm * threads) {
+      threads = threads_r;
+      per_sm = per_sm_r;
+      slots = rounds;
+      fixed = fixed_r;
+    }
   }
   if (threads == 0 || per_sm * threads < 128) return NETMAX_OK;  // too few warps to hide the arithmetic latency
   f.threads = threads;
+  f.slots = slots;
   f.smem = fixed + (size_t)48 * M * threads;
-  f.max_rounds = ctx->fuse_rounds >= 2 ? std::min(ctx->fuse_rounds, kFusedMaxRounds) : kFusedMaxRounds;
+  f.max_rounds = slots;
   f.n_tiles = ((ctx->d + 3) / 4 + threads - 1) / threads;
   NM_CUDA(ctx, cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)f.smem));
   f.grid = (int)std::min<int64_t>(f.n_tiles, std::min<int64_t>((int64_t)per_sm * ctx->sm_count, kMaxGrid));
@@ -735,7 +757,7 @@ ClusterKernel pick_cluster_kernel(int objective) {
 #endif
 
 size_t cluster_smem(int rpc, int threads) {
-  return align_up((size_t)kFusedMaxRounds * rpc * 16, 128) + (size_t)3 * rpc * threads * 16 + (size_t)2 * threads * 16 +
+  return align_up((size_t)kClusterMaxRounds * rpc * 16, 128) + (size_t)3 * rpc * threads * 16 + (size_t)2 * threads * 16 +
          64 * sizeof(double);
 }
 
@@ -809,7 +831,7 @@ int plan_cluster_uncached(netmax_ctx* ctx, const RoundPlan& plan, const FusedPla
     f.rpc = rpc;
     f.smem = smem;
     f.n_tiles = ((ctx->d + 3) / 4 + cand - 1) / cand;
-    f.max_rounds = ctx->fuse_rounds >= 2 ? std::min(ctx->fuse_rounds, kFusedMaxRounds) : kFusedMaxRounds;
+    f.max_rounds = ctx->fuse_rounds >= 2 ? std::min(ctx->fuse_rounds, kClusterMaxRounds) : kClusterMaxRounds;
     f.grid = (int)std::min<int64_t>(f.n_tiles, (int64_t)clusters) * C;
     f.ok = true;
     break;
@@ -892,7 +914,10 @@ int launch_long_rounds(netmax_ctx* ctx, cudaStream_t stream, const RoundPlan& pl
     const unsigned char* xin = ctx->x[cur] + shift;
     unsigned char* xout = ctx->x[cur ^ 1] + shift;
     if ((fused.ok || cluster.ok) && n - b >= 2) {  // the next rounds in one launch over resident tiles
-      const int chunk = (int)std::min<int64_t>(n - b, fused.ok ? fused.max_rounds : cluster.max_rounds);
+      // launches of even length (20 rounds at 8 per launch: 7 + 7 + 6, not 8 + 8 + 4)
+      const int64_t per_launch = fused.ok ? fused.max_rounds : cluster.max_rounds;
+      const int64_t launches_left = (n - b + per_launch - 1) / per_launch;
+      const int chunk = (int)((n - b + launches_left - 1) / launches_left);
       const int threads = fused.ok ? fused.threads : cluster.threads;
       FusedParams fp;
       fp.x_cur = reinterpret_cast<const float4*>(xin);
@@ -907,6 +932,7 @@ int launch_long_rounds(netmax_ctx* ctx, cudaStream_t stream, const RoundPlan& pl
       fp.ring = ctx->trace_rounds;
       fp.first_round = r;
       fp.n_rounds = chunk;
+      fp.slots = fused.ok ? fused.slots : kClusterMaxRounds;
       fp.nq = range.nq4;
       fp.n_tiles = (range.nq4 + threads - 1) / threads;
       fp.row_bytes = p.row_bytes;
@@ -938,7 +964,8 @@ int launch_long_rounds(netmax_ctx* ctx, cudaStream_t stream, const RoundPlan& pl
         NM_CUDA(ctx, cudaLaunchKernelEx(&lc, ck, cpar));
       } else {
         // (the attribute belongs to the kernel, not to this context: another context may have lowered it)
-        FusedKernel fk = pick_fused_kernel(ctx->objective, ctx->L.halves);
+        // (one instance for all launches of the call: the larger one unless the whole call is four rounds or fewer)
+        FusedKernel fk = pick_fused_kernel(ctx->objective, ctx->L.halves, (int)std::min<int64_t>(n, fused.max_rounds));
         NM_CUDA(ctx, cudaFuncSetAttribute(fk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fused.smem));
         fk<<<(unsigned)std::min<int64_t>(fused.grid, fp.n_tiles), fused.threads, fused.smem, stream>>>(fp);
       }

@@ -674,7 +674,10 @@ __global__ void __launch_bounds__(256, 2) multi_round_kernel(const MultiRoundPar
 // in, and every round's result is rounded to bfloat16 before it is written to the slab, exactly
 // as a store to and a load from the bfloat16 state would.
 #ifndef NETMAX_FUSED_MAX_ROUNDS
-#define NETMAX_FUSED_MAX_ROUNDS 4
+#define NETMAX_FUSED_MAX_ROUNDS 8
+#endif
+#ifndef NETMAX_CLUSTER_MAX_ROUNDS
+#define NETMAX_CLUSTER_MAX_ROUNDS 4
 #endif
 #ifndef NETMAX_FUSED_UNROLL
 #define NETMAX_FUSED_UNROLL 2
@@ -682,7 +685,8 @@ __global__ void __launch_bounds__(256, 2) multi_round_kernel(const MultiRoundPar
 #ifndef NETMAX_FUSED_PREFETCH
 #define NETMAX_FUSED_PREFETCH 1  // fetch the next tile under the last round of the current one (fp32 state)
 #endif
-constexpr int kFusedMaxRounds = NETMAX_FUSED_MAX_ROUNDS;
+constexpr int kFusedMaxRounds = NETMAX_FUSED_MAX_ROUNDS;      // rounds per launch of fused_rounds_kernel, at most
+constexpr int kClusterMaxRounds = NETMAX_CLUSTER_MAX_ROUNDS;  // of cluster_rounds_kernel (16 accumulator registers per four rounds: it has none to spare)
 constexpr int kFusedUnroll = NETMAX_FUSED_UNROLL;  // rows of a round in flight per thread
 
 struct FusedParams {
@@ -696,7 +700,8 @@ struct FusedParams {
   unsigned int* ticket;  // last-CTA-done counter (0 between launches)
   int64_t slot0, ring;   // ring slot of the first round
   uint64_t first_round;
-  int32_t n_rounds;      // 1 .. kFusedMaxRounds
+  int32_t n_rounds;      // 1 .. slots
+  int32_t slots;         // rounds the table of draws at the head of the shared memory has room for (<= kFusedMaxRounds)
   int64_t nq, n_tiles;   // column groups of FOUR elements per row (whatever the storage), tiles of blockDim of them
   uint32_t row_bytes;
   int32_t M, tail;       // tail = d % 4
@@ -705,16 +710,18 @@ struct FusedParams {
   PhiloxKeys keys;
 };
 
-// Dynamic shared memory: (peer row offset, -, -weight, -weight) int4[kFusedMaxRounds][M], then the slabs
+// Dynamic shared memory: (peer row offset, -, -weight, -weight) int4[slots][M], then the slabs
 // float4[3][M][blockDim] (replicas of even rounds, of odd rounds, centres), then 64 doubles.
 // Any block size that is a multiple of 32 up to 256 works.
-template <int kObjective, bool kFastNoise, bool kBf16>
+// kRounds: rounds a launch runs at most (4 or kFusedMaxRounds); a thread keeps two double accumulators per round,
+// and a launch of up to four rounds runs 4 % faster on the instance that holds eight instead of sixteen of them.
+template <int kObjective, bool kFastNoise, bool kBf16, int kRounds>
 __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams p) {
   constexpr uint32_t kGroupBytes = kBf16 ? 8u : 16u;  // four elements in global memory
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int tid = threadIdx.x, T = blockDim.x, M = p.M;
   int4* s_pw = reinterpret_cast<int4*>(smem_raw);  // (byte offset of the peer's row in a slab, unused, -w, -w)
-  const uint32_t head = ((uint32_t)(kFusedMaxRounds * M * 16) + 127u) & ~127u;
+  const uint32_t head = ((uint32_t)(p.slots * M * 16) + 127u) & ~127u;
   const uint32_t stride = (uint32_t)T * 16u;     // bytes between consecutive rows of a slab
   const uint32_t plane = (uint32_t)M * stride;   // bytes of one [M][T] slab
   unsigned char* slab = smem_raw + head + (uint32_t)tid * 16u;  // this thread's column: slabs 0, 1 (replicas), 2 (centres)
@@ -730,9 +737,9 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
   }
   __syncthreads();
 
-  double acc_cons[kFusedMaxRounds], acc_loss[kFusedMaxRounds];
+  double acc_cons[kRounds], acc_loss[kRounds];
 #pragma unroll
-  for (int k = 0; k < kFusedMaxRounds; ++k) acc_cons[k] = acc_loss[k] = 0.0;
+  for (int k = 0; k < kRounds; ++k) acc_cons[k] = acc_loss[k] = 0.0;
 
   // Slab `base` (0 or 1) holds the tile's values at the start of the first round; round k reads
   // slab (base + k) & 1 and writes the other one.  The LAST round of a tile writes its results
@@ -856,7 +863,7 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
                                    (s2.z - s1.z * s1.z * p.inv_M) + (s2.w - s1.w * s1.w * p.inv_M));
       const double loss = (double)((l0 + l1) + (l2 + l3));
 #pragma unroll
-      for (int kk = 0; kk < kFusedMaxRounds; ++kk) {  // acc[k] with k known only at run time: predicated adds keep it in registers
+      for (int kk = 0; kk < kRounds; ++kk) {  // acc[k] with k known only at run time: predicated adds keep it in registers
         if (kk == k) {
           acc_cons[kk] += cons;
           acc_loss[kk] += loss;
@@ -871,7 +878,7 @@ __global__ void __launch_bounds__(256, 2) fused_rounds_kernel(const FusedParams 
 
   // telemetry: per round, CTA partials; the last CTA to finish sums them in index order
 #pragma unroll
-  for (int k = 0; k < kFusedMaxRounds; ++k)
+  for (int k = 0; k < kRounds; ++k)
     if (k < p.n_rounds) block_partials(p.partials + (size_t)k * 2 * gridDim.x, acc_cons[k], acc_loss[k], s_red);
   __shared__ bool s_last;
   if (tid == 0) {
@@ -932,7 +939,7 @@ __device__ __forceinline__ ulonglong2 ld_cluster_16(uint32_t smem_addr, uint32_t
   return v;
 }
 
-// Dynamic shared memory: (peer's local row offset, peer's CTA, -weight, -weight) int4[kFusedMaxRounds][rpc],
+// Dynamic shared memory: (peer's local row offset, peer's CTA, -weight, -weight) int4[kClusterMaxRounds][rpc],
 // then the slabs float4[3][rpc][blockDim], then the exchange area float4[2][blockDim], then 64 doubles.
 template <int kObjective, bool kFastNoise>
 __global__ void __launch_bounds__(256, 2) cluster_rounds_kernel(const ClusterParams cp) {
@@ -942,7 +949,7 @@ __global__ void __launch_bounds__(256, 2) cluster_rounds_kernel(const ClusterPar
   const uint32_t rank = cluster_ctarank(), C = cluster_nctarank();
   const int r0 = min(M, (int)rank * rpc), rows = min(M, r0 + rpc) - r0;  // this CTA's rows [r0, r0 + rows)
   int4* s_pw = reinterpret_cast<int4*>(smem_raw);
-  const uint32_t head = ((uint32_t)(kFusedMaxRounds * rpc * 16) + 127u) & ~127u;
+  const uint32_t head = ((uint32_t)(kClusterMaxRounds * rpc * 16) + 127u) & ~127u;
   const uint32_t stride = (uint32_t)T * 16u;
   const uint32_t plane = (uint32_t)rpc * stride;
   unsigned char* slab = smem_raw + head + (uint32_t)tid * 16u;
@@ -963,9 +970,9 @@ __global__ void __launch_bounds__(256, 2) cluster_rounds_kernel(const ClusterPar
   }
   __syncthreads();
 
-  double acc_cons[kFusedMaxRounds], acc_loss[kFusedMaxRounds];
+  double acc_cons[kClusterMaxRounds], acc_loss[kClusterMaxRounds];
 #pragma unroll
-  for (int k = 0; k < kFusedMaxRounds; ++k) acc_cons[k] = acc_loss[k] = 0.0;
+  for (int k = 0; k < kClusterMaxRounds; ++k) acc_cons[k] = acc_loss[k] = 0.0;
 
   const int64_t n_clusters = gridDim.x / C, cluster_id = blockIdx.x / C;
   const uint64_t row0_bytes = (uint64_t)(uint32_t)r0 * p.row_bytes;
@@ -1094,7 +1101,7 @@ __global__ void __launch_bounds__(256, 2) cluster_rounds_kernel(const ClusterPar
       }
       const double loss = (double)((l0 + l1) + (l2 + l3));
 #pragma unroll
-      for (int kk = 0; kk < kFusedMaxRounds; ++kk) {
+      for (int kk = 0; kk < kClusterMaxRounds; ++kk) {
         if (kk == k) {
           acc_cons[kk] += cons;
           acc_loss[kk] += loss;
@@ -1109,7 +1116,7 @@ __global__ void __launch_bounds__(256, 2) cluster_rounds_kernel(const ClusterPar
   cluster_barrier();  // no CTA leaves while another may still read its exchange area
 
 #pragma unroll
-  for (int k = 0; k < kFusedMaxRounds; ++k)
+  for (int k = 0; k < kClusterMaxRounds; ++k)
     if (k < p.n_rounds) block_partials(p.partials + (size_t)k * 2 * gridDim.x, acc_cons[k], acc_loss[k], s_red);
   __shared__ bool s_last;
   if (tid == 0) {

@@ -35,7 +35,7 @@ def test_hbm_roofline_counts_the_bytes_that_must_cross_the_pins():
     assert r["achieved"] == pytest.approx(12 * elements / (ms / 1e3) / 1e9)
     assert r["frac"] == pytest.approx(r["achieved"] / 6537.0) and r["frac"] < 1.0
     assert r["replica_GBs"] == pytest.approx(16 * elements / (ms / 1e3) / 1e9)
-    assert r["traffic"] == pytest.approx(1_042_482_000)
+    assert r["traffic"] == pytest.approx(1_041_843_000)
     assert r["dram_GBs"] == pytest.approx(r["traffic"] / (ms / 1e3) / 1e9)
     assert r["dram_frac_of_8TBs"] == pytest.approx(r["dram_GBs"] / 8000.0)
     unknown = bench.hbm_roofline("some other workload", "round_kernel", ms, elements, 16, 6537.0, "measured")

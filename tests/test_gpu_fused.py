@@ -40,7 +40,8 @@ def random_policy(M, rng, zeros=0.0):
                                               (9, 310_000, 3, "f32"), (8, 400_001, 2, "f32"), (16, 320_001, 4, "f32"),
                                               (18, 310_003, 4, "f32"), (8, 700_003, 0, "bf16"), (3, 650_001, 4, "bf16"),
                                               (16, 620_006, 3, "bf16"), (24, 310_001, 0, "f32"), (36, 170_003, 0, "f32"),
-                                              (22, 620_002, 0, "bf16"), (36, 330_001, 2, "bf16")])
+                                              (22, 620_002, 0, "bf16"), (36, 330_001, 2, "bf16"), (8, 400_003, 8, "f32"),
+                                              (5, 320_003, 6, "f32"), (16, 620_002, 8, "bf16")])
 @pytest.mark.parametrize("objective", [0, 1])
 def test_fused_rounds_change_no_bit(nm, M, d, fuse, storage, objective):
     rng = np.random.default_rng(M * 11 + d)
@@ -176,5 +177,5 @@ def test_fused_rounds_match_the_oracle(nm, M, d):
 
 def test_fuse_rounds_out_of_range_is_refused(nm):
     with pytest.raises(nm.NetmaxError) as e:
-        nm.Netmax(M=2, d=64, lr=0.1, fuse_rounds=5)
+        nm.Netmax(M=2, d=64, lr=0.1, fuse_rounds=9)
     assert e.value.code == -1
